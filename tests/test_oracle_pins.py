@@ -1,0 +1,324 @@
+"""Pins of the fp64 oracle against what the paper and the mathematics fix.
+
+None of these tests re-types the oracle's own formula: each compares an oracle
+function with a library routine, a closed form, a sampling estimate, an
+explicit per-position computation or brute-force enumeration.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_00636_b200 import inputs
+
+
+def bf16_bits(x):
+    """float array -> (uint16 bit patterns after bf16 rounding, the rounded values as float64)."""
+    t = torch.as_tensor(np.asarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return inputs.bits(t), t.float().numpy().astype(np.float64)
+
+
+def rotate(x, pos, base, layout="half"):
+    """Rotary embedding written with complex numbers (independent of oracle and generator)."""
+    d = x.shape[-1]
+    m = np.arange(d // 2)
+    theta = base ** (-2.0 * m / d)
+    if layout == "half":
+        z = x[..., : d // 2] + 1j * x[..., d // 2:]
+    else:
+        z = x[..., 0::2] + 1j * x[..., 1::2]
+    z = z * np.exp(1j * pos * theta)
+    out = np.empty_like(x)
+    if layout == "half":
+        out[..., : d // 2], out[..., d // 2:] = z.real, z.imag
+    else:
+        out[..., 0::2], out[..., 1::2] = z.real, z.imag
+    return out
+
+
+# ---------------------------------------------------------------- O1 mean / covariance
+@pytest.mark.parametrize("norm", [0, 1])
+def test_mean_cov_matches_numpy(oracle, norm):
+    rng = np.random.default_rng(1)
+    q_bits, q = bf16_bits(rng.normal(size=(3, 2, 40, 16)) * 3 + 1.5)
+    mu, sigma = oracle.mean_cov(q_bits, cov_norm=norm)
+    for u in range(3):
+        for h in range(2):
+            np.testing.assert_allclose(mu[u, h], q[u, h].mean(0), rtol=1e-13, atol=1e-13)
+            ref = np.cov(q[u, h].T, bias=(norm == 0))
+            np.testing.assert_allclose(sigma[u, h], ref, rtol=1e-11, atol=1e-12)
+    # symmetric, positive semi-definite, rank at most W - 1
+    q_bits, q = bf16_bits(rng.normal(size=(1, 1, 5, 12)))
+    _, s = oracle.mean_cov(q_bits)
+    s = s[0, 0]
+    assert np.array_equal(s, s.T)
+    ev = np.linalg.eigvalsh(s)
+    assert ev.min() > -1e-12
+    assert (ev > 1e-10).sum() <= 4
+
+
+# ---------------------------------------------------------------- O2 averaged rotation
+@pytest.mark.parametrize("pos,T,base,d", [(512, 512, 1e4, 64), (8192, 512, 5e5, 128),
+                                          (131072, 1024, 1e6, 256), (0, 1, 1e4, 8), (7, 3, 10.0, 4)])
+def test_rope_average_closed_form(oracle, pos, T, base, d):
+    """Geometric series: (1/T) sum_j e^{i theta (p+j)} = e^{i theta (p+(T-1)/2)} sin(T theta/2) / (T sin(theta/2))."""
+    cbar, sbar = oracle.rope_average(np.array([pos]), T, base, d)
+    theta = base ** (-2.0 * np.arange(d // 2) / d)
+    z = np.exp(1j * theta * (pos + (T - 1) / 2)) * np.sin(T * theta / 2) / (T * np.sin(theta / 2))
+    np.testing.assert_allclose(cbar[0], z.real, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(sbar[0], z.imag, rtol=0, atol=1e-11)
+    assert np.all(cbar ** 2 + sbar ** 2 <= 1 + 1e-12)
+
+
+def test_rope_average_special_cases(oracle):
+    # T = 1: the average is the rotation at pos_next itself (orthogonal blocks)
+    cbar, sbar = oracle.rope_average(np.array([37]), 1, 1e4, 16)
+    np.testing.assert_allclose(cbar ** 2 + sbar ** 2, 1.0, atol=1e-14)
+    theta = 1e4 ** (-2.0 * np.arange(8) / 16)
+    np.testing.assert_allclose(cbar[0], np.cos(37 * theta), atol=1e-14)
+    np.testing.assert_allclose(sbar[0], np.sin(37 * theta), atol=1e-14)
+    # channel 0 has theta = 1: the average over many positions nearly cancels
+    cbar, sbar = oracle.rope_average(np.array([100]), 512, 1e4, 16)
+    assert math.hypot(cbar[0, 0], sbar[0, 0]) < 5e-3
+    # huge base: the slow channels barely rotate, their block stays close to the identity
+    cbar, sbar = oracle.rope_average(np.array([0]), 4, 1e30, 8)
+    np.testing.assert_allclose(cbar[0, 1:], 1.0, atol=1e-6)
+    np.testing.assert_allclose(sbar[0, 1:], 0.0, atol=1e-6)
+    # several units at once
+    c2, s2 = oracle.rope_average(np.array([5, 900]), 16, 1e4, 8)
+    c5, _ = oracle.rope_average(np.array([5]), 16, 1e4, 8)
+    c9, _ = oracle.rope_average(np.array([900]), 16, 1e4, 8)
+    assert np.array_equal(c2[0], c5[0]) and np.array_equal(c2[1], c9[0])
+
+
+# ---------------------------------------------------------------- O3 averaged Gaussian
+@pytest.mark.parametrize("layout", ["half", "interleaved"])
+def test_averaged_gaussian_equals_statistics_of_rotated_samples(oracle, layout):
+    """mu_bar / Sigma_bar must be the mean / covariance of the window queries after each is
+    rotated to every future position and averaged over positions (explicit, sample by sample)."""
+    rng = np.random.default_rng(2)
+    U, Hq, W, d, T, base = 2, 3, 24, 16, 11, 50.0
+    pos = np.array([40, 3])
+    q_bits, q = bf16_bits(rng.normal(size=(U, Hq, W, d)) + 0.7)
+    lay = 0 if layout == "half" else 1
+    mu_bar, sigma_bar = oracle.query_stats(q_bits, pos, T, base, layout=lay)
+    for u in range(U):
+        qbar = np.mean([rotate(q[u], pos[u] + j, base, layout) for j in range(T)], axis=0)
+        for h in range(Hq):
+            np.testing.assert_allclose(mu_bar[u, h], qbar[h].mean(0), atol=1e-12)
+            np.testing.assert_allclose(sigma_bar[u, h], np.cov(qbar[h].T, bias=True), atol=1e-12)
+
+
+def test_rotation_convention_matches_key_generator(oracle):
+    """The generator's rotary embedding of keys and the oracle's averaged rotation of queries
+    use one convention: mean_j (R_{p+j} q) . (R_i k) equals (R_bar q) . (R_i k), and the
+    generator's rotation gives scores that depend on relative position only."""
+    rng = np.random.default_rng(3)
+    d, base, T, p = 32, 1e3, 9, 77
+    q = rng.normal(size=(1, d))
+    k = rng.normal(size=(1, d))
+    kt = lambda pos: inputs.rope_half_split(torch.tensor(k, dtype=torch.float32),
+                                            torch.tensor([pos]), base).double().numpy()
+    qt = lambda pos: inputs.rope_half_split(torch.tensor(q, dtype=torch.float32),
+                                            torch.tensor([pos]), base).double().numpy()
+    # relative-position property of the generator's embedding
+    assert abs((qt(50) @ kt(20).T).item() - (qt(130) @ kt(100).T).item()) < 1e-4
+    np.testing.assert_allclose(kt(20), rotate(k.astype(np.float32).astype(np.float64), 20, base), atol=1e-5)
+    # oracle's R_bar applied to a single "mean" vector with zero covariance
+    cbar, sbar = oracle.rope_average(np.array([p]), T, base, d)
+    mu_bar, sig_bar = oracle.apply_rope_average(q.reshape(1, 1, d), np.zeros((1, 1, d, d)), cbar, sbar)
+    want = np.mean([(rotate(q, p + j, base) @ rotate(k, 5, base).T).item() for j in range(T)])
+    got = (mu_bar[0, 0] @ rotate(k, 5, base).T).item()
+    assert abs(want - got) < 1e-12
+    assert np.all(sig_bar == 0)
+
+
+# ---------------------------------------------------------------- O4 closed-form expectation
+def _small_problem(rng, U=1, Hq=2, Hkv=1, W=32, d=8, n=12, qscale=0.6):
+    q_bits, q = bf16_bits(rng.normal(size=(U, Hq, W, d)) * qscale + 0.2)
+    k_bits, k = bf16_bits(rng.normal(size=(U, Hkv, n, d)))
+    v_bits, v = bf16_bits(rng.normal(size=(U, Hkv, n, d)))
+    return q_bits, q, k_bits, k, v_bits, v
+
+
+def test_logits_match_monte_carlo_expectation(oracle):
+    """exp(s_i) must equal E[exp(q.k_i/sqrt(d))] for q ~ N(mu_bar, Sigma_bar) (Gaussian MGF)."""
+    rng = np.random.default_rng(4)
+    d, n = 8, 12
+    q_bits, q, k_bits, k, _, _ = _small_problem(rng, d=d, n=n)
+    mu_bar, sigma_bar = oracle.query_stats(q_bits, np.array([20]), 6, 100.0)
+    s = oracle.logits(k_bits, mu_bar, sigma_bar)
+    N = 400_000
+    for h in range(2):
+        w, V = np.linalg.eigh(sigma_bar[0, h])
+        L = V * np.sqrt(np.clip(w, 0, None))
+        samples = mu_bar[0, h] + rng.normal(size=(N, d)) @ L.T
+        e = np.exp(samples @ k[0, 0].T / math.sqrt(d))           # [N, n]
+        est, se = e.mean(0), e.std(0, ddof=1) / math.sqrt(N)
+        z = (est - np.exp(s[0, h])) / se
+        assert np.all(np.abs(z) < 4.5), z
+        # the quadratic term matters here: the estimate excludes the mean-only formula
+        lin_only = np.exp(k[0, 0] @ mu_bar[0, h] / math.sqrt(d))
+        assert np.any(np.abs(est - lin_only) / se > 10)
+
+
+def test_logits_zero_covariance_is_dot_product(oracle):
+    """All window queries equal => Sigma = 0 and s_i = (R_bar u) . k_i / sqrt(d)."""
+    rng = np.random.default_rng(5)
+    d, n, W, T, base, p = 16, 20, 10, 7, 1e3, 31
+    u_bits, u = bf16_bits(rng.normal(size=(d,)))
+    q_bits = np.broadcast_to(u_bits, (1, 1, W, d)).copy()
+    k_bits, k = bf16_bits(rng.normal(size=(1, 1, n, d)))
+    mu_bar, sigma_bar = oracle.query_stats(q_bits, np.array([p]), T, base)
+    assert np.abs(sigma_bar).max() < 1e-28
+    s = oracle.logits(k_bits, mu_bar, sigma_bar)
+    ubar = np.mean([rotate(u, p + j, base) for j in range(T)], axis=0)
+    np.testing.assert_allclose(s[0, 0], k[0, 0] @ ubar / math.sqrt(d), atol=1e-12)
+
+
+def test_logits_equal_mean_and_variance_of_projected_window(oracle):
+    """s_i = mean_w(k_i.qbar_w)/sqrt(d) + var_w(k_i.qbar_w)/(2d), qbar_w the averaged-rotated samples."""
+    rng = np.random.default_rng(6)
+    U, Hq, Hkv, W, d, n, T, base = 2, 4, 2, 20, 16, 33, 5, 200.0
+    pos = np.array([33, 64])
+    q_bits, q, k_bits, k, _, _ = _small_problem(rng, U, Hq, Hkv, W, d, n, qscale=2.0)
+    mu_bar, sigma_bar = oracle.query_stats(q_bits, pos, T, base)
+    s = oracle.logits(k_bits, mu_bar, sigma_bar)
+    for u in range(U):
+        qbar = np.mean([rotate(q[u], pos[u] + j, base) for j in range(T)], axis=0)   # [Hq, W, d]
+        for h in range(Hq):
+            proj = k[u, h // 2] @ qbar[h].T                                            # [n, W]
+            want = proj.mean(1) / math.sqrt(d) + proj.var(1) / (2 * d)
+            np.testing.assert_allclose(s[u, h], want, rtol=1e-11, atol=1e-11)
+
+
+# ---------------------------------------------------------------- O5-O7 softmax, GQA, value norm
+def test_scores_invariants(oracle):
+    rng = np.random.default_rng(7)
+    U, Hq, Hkv, n, d = 2, 6, 2, 50, 8
+    s = rng.normal(size=(U, Hq, n)) * 4
+    v_bits, v = bf16_bits(rng.normal(size=(U, Hkv, n, d)))
+    vnorm = np.linalg.norm(v, axis=-1)
+    sc, a = oracle.scores(s, v_bits, 0.02, oracle.GROUP_MEAN_PROB, return_attention=True)
+    np.testing.assert_allclose(a.sum(-1), 1.0, atol=1e-13)
+    np.testing.assert_allclose(sc, (a + 0.02) * vnorm, rtol=1e-13)
+    # scipy's softmax as the library routine for Eq. 8
+    from scipy.special import softmax
+    ref = softmax(s, axis=-1).reshape(U, Hkv, 3, n).mean(2)
+    np.testing.assert_allclose(a, ref, rtol=1e-12, atol=1e-15)
+    _, a_sum = oracle.scores(s, v_bits, 0.0, oracle.GROUP_SUM_PROB, return_attention=True)
+    np.testing.assert_allclose(a_sum, 3 * ref, rtol=1e-12, atol=1e-15)
+    _, a_ml = oracle.scores(s, v_bits, 0.0, oracle.GROUP_MEAN_LOGIT, return_attention=True)
+    np.testing.assert_allclose(a_ml, softmax(s.reshape(U, Hkv, 3, n).mean(2), axis=-1), rtol=1e-12)
+    # adding a per-head constant to the logits changes nothing, even a huge one
+    shift = rng.normal(size=(U, Hq, 1)) * 1e5
+    sc2 = oracle.scores(s + shift, v_bits, 0.02)
+    np.testing.assert_allclose(sc2, sc, rtol=1e-9)
+    # logits far beyond exp's range stay finite
+    big = oracle.scores(s * 1e4, v_bits, 0.02)
+    assert np.all(np.isfinite(big))
+    # scaling V by c scales the scores by c and keeps the kept set
+    v2_bits, _ = bf16_bits(v * 4.0)
+    sc4 = oracle.scores(s, v2_bits, 0.02)
+    np.testing.assert_allclose(sc4, 4 * sc, rtol=1e-13)
+    assert np.array_equal(oracle.select(sc4, 17), oracle.select(sc, 17))
+
+
+def test_group_modes_coincide_without_grouping(oracle):
+    rng = np.random.default_rng(8)
+    s = rng.normal(size=(1, 3, 30)) * 3
+    v_bits, _ = bf16_bits(rng.normal(size=(1, 3, 30, 4)))
+    base = oracle.scores(s, v_bits, 0.02, oracle.GROUP_MEAN_PROB)
+    for mode in (oracle.GROUP_SUM_PROB, oracle.GROUP_MEAN_LOGIT):
+        np.testing.assert_allclose(oracle.scores(s, v_bits, 0.02, mode), base, rtol=1e-13)
+
+
+# ---------------------------------------------------------------- O8-O9 selection and compaction
+def test_select_brute_force(oracle):
+    rng = np.random.default_rng(9)
+    for n, kept in [(1, 1), (6, 0), (9, 4), (12, 12), (13, 5)]:
+        sc = rng.random(size=(3, n))
+        idx = oracle.select(sc, kept)
+        assert idx.shape == (3, kept)
+        for h in range(3):
+            best = max(itertools.combinations(range(n), kept), key=lambda c: sc[h, list(c)].sum())
+            assert list(idx[h]) == sorted(best)
+
+
+def test_select_ties_take_lowest_index(oracle):
+    sc = np.array([[1.0, 3.0, 3.0, 0.5, 3.0, 3.0, 2.0, 3.0]])
+    assert list(oracle.select(sc, 3)[0]) == [1, 2, 4]
+    assert list(oracle.select(sc, 6)[0]) == [1, 2, 4, 5, 6, 7]
+    assert list(oracle.select(np.zeros((1, 7)), 4)[0]) == [0, 1, 2, 3]
+    # every subset of the same total is valid; the rule picks the lexicographically first
+    n, kept = 10, 4
+    sc = np.array([[2.0, 1, 2, 1, 2, 1, 1, 2, 1, 1]])
+    best_sum = max(sc[0, list(c)].sum() for c in itertools.combinations(range(n), kept))
+    ties = [c for c in itertools.combinations(range(n), kept) if sc[0, list(c)].sum() == best_sum]
+    assert list(oracle.select(sc, kept)[0]) == list(min(ties))
+
+
+def test_select_follows_permutation(oracle):
+    rng = np.random.default_rng(10)
+    sc = rng.random(size=(2, 40))
+    perm = rng.permutation(40)
+    a = oracle.select(sc, 11)
+    b = oracle.select(sc[:, perm], 11)
+    for h in range(2):
+        assert sorted(perm[b[h]]) == list(a[h])
+
+
+def test_gather(oracle):
+    rng = np.random.default_rng(11)
+    rows = rng.integers(0, 65535, size=(2, 3, 9, 4), dtype=np.uint16)
+    idx = np.sort(rng.permuted(np.tile(np.arange(9), (2, 3, 1)), axis=-1)[..., :5], axis=-1).astype(np.int32)
+    out = oracle.gather(rows, idx)
+    assert np.array_equal(out, np.take_along_axis(rows, idx[..., None].astype(np.int64), axis=2))
+
+
+def test_n_kept_is_truncated_product(oracle):
+    assert oracle.n_kept(512, 0.5) == 256
+    assert oracle.n_kept(8192, 0.5) == 4096
+    assert oracle.n_kept(32768, 0.75) == 8192
+    assert oracle.n_kept(131072, 0.875) == 16384
+    assert oracle.n_kept(10, 0.0) == 10 and oracle.n_kept(10, 1.0) == 0
+    rng = np.random.default_rng(12)
+    for _ in range(200):
+        n, r = int(rng.integers(0, 10**6)), float(rng.random())
+        assert oracle.n_kept(n, r) == int(n * (1 - r))
+
+
+# ---------------------------------------------------------------- whole path
+def test_whole_path_single_head_against_array_formulation(oracle):
+    """One head, eps = 0: the compression routine written with whole-array library operations
+    (matrix products, softmax, norms, a stable descending sort) selects the same pairs."""
+    from scipy.special import softmax
+    rng = np.random.default_rng(13)
+    W, d, n, T, base, kept = 48, 16, 200, 8, 1e3, 60
+    q_bits, q = bf16_bits(rng.normal(size=(1, 1, W, d)) * 1.5 + 0.3)
+    k_bits, k = bf16_bits(rng.normal(size=(1, 1, n, d)))
+    v_bits, v = bf16_bits(rng.normal(size=(1, 1, n, d)) * np.exp(0.5 * rng.normal(size=(1, 1, n, 1))))
+    out = oracle.compress(q_bits, k_bits, v_bits, np.array([n]), T, base, 0.0, kept)
+    qbar = np.mean([rotate(q[0, 0], n + j, base) for j in range(T)], axis=0)
+    mean_query, cov_query = qbar.mean(0), np.cov(qbar.T, bias=True)
+    keys, values = k[0, 0], v[0, 0]
+    sc = keys @ mean_query / math.sqrt(d) + np.einsum("ni,ij,nj->n", keys, cov_query, keys) / (2 * d)
+    sc = softmax(sc) * np.linalg.norm(values, axis=-1)
+    top = np.sort(np.argsort(-sc, kind="stable")[:kept])
+    assert np.array_equal(out["kept_idx"][0, 0], top)
+    np.testing.assert_allclose(out["scores"][0, 0], sc, rtol=1e-10)
+    assert np.array_equal(out["k_out"][0, 0], k_bits[0, 0][top])
+    assert np.array_equal(out["v_out"][0, 0], v_bits[0, 0][top])
+
+
+def test_oracle_on_tiny_config(oracle):
+    """Config 0 end to end: shapes, finiteness, and the one-hot character of its softmax."""
+    cfg = inputs.CONFIGS[0]
+    q, k, v, pos = inputs.generate_layer(cfg)
+    out = oracle.compress(inputs.bits(q), inputs.bits(k), inputs.bits(v), pos.numpy(), cfg.n_future,
+                          cfg.rope_base, cfg.eps, cfg.n_kept)
+    assert out["kept_idx"].shape == (1, 2, 256)
+    assert np.all(np.isfinite(out["logits"])) and np.all(np.isfinite(out["scores"]))
+    assert np.all(np.diff(out["kept_idx"], axis=-1) > 0)

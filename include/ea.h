@@ -1,0 +1,178 @@
+/*
+ * ea.h - C ABI of the Expected Attention KV-cache scoring and pruning library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the compression routine of the Expected Attention
+ * paper (Sec. 2.2, "Expected Attention: Estimating Attention From Future
+ * Queries"; its compress() pseudo-code) as three asynchronous calls:
+ *
+ *   ea_query_stats     window queries -> position-averaged Gaussian (Eq. 5, 6)
+ *   ea_score           closed-form expected attention of every cached key,
+ *                      softmax over positions, GQA reduction, value-norm
+ *                      weighting (Eq. 7, 8, 9)
+ *   ea_select_compact  keep the n_kept highest-scoring pairs per KV head and
+ *                      gather their K/V rows (the "Compression with Expected
+ *                      Attention" paragraph)
+ *
+ * Conventions
+ *   - One "unit" is one (layer, batch element).  A call handles n_units units
+ *     that share every size; units, and the KV heads inside them, are
+ *     independent problems.
+ *   - Query head h reads KV head h / G, G = n_q_heads / n_kv_heads.
+ *   - All data pointers are DEVICE pointers on the context's device unless a
+ *     comment says HOST.  Tensors are dense, row-major, innermost index last.
+ *     bf16 tensors are passed as const void* / void*.
+ *   - The caller owns every data buffer.  The library never allocates, frees
+ *     or keeps them; the only memory it owns is the context's workspace.
+ *   - Calls enqueue work on cuda_stream (a cudaStream_t passed as void*; NULL
+ *     is the default stream) and return without synchronising.  Work of one
+ *     context must be ordered on one stream at a time (the workspace is
+ *     shared between calls).
+ *   - Errors that the host can detect are returned before anything is
+ *     launched.  No call aborts, throws or traps the device.  A device-side
+ *     wait that runs out of its iteration budget records
+ *     EA_ERR_DEVICE_TIMEOUT, which ea_sync_status reports.
+ *   - There is no CPU fallback: on a machine without an sm_100 GPU ea_create
+ *     fails with EA_ERR_NOT_SM100 or EA_ERR_CUDA.
+ */
+#ifndef EA_H_
+#define EA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum ea_status {
+    EA_OK = 0,
+    EA_ERR_INVALID_ARG = 1,    /* NULL pointer, bad size, misaligned buffer            */
+    EA_ERR_UNSUPPORTED = 2,    /* head_dim or mode not implemented                     */
+    EA_ERR_WORKSPACE = 3,      /* context workspace smaller than ea_workspace_bytes    */
+    EA_ERR_CUDA = 4,           /* a CUDA runtime call failed                           */
+    EA_ERR_NOT_SM100 = 5,      /* device is not compute capability 10.x                */
+    EA_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait gave up                   */
+} ea_status;
+
+/* RoPE channel pairing used when the rotation is averaged (Eq. 6). */
+enum { EA_ROPE_HALF_SPLIT = 0,   /* channel m pairs with m + d/2 (default)             */
+       EA_ROPE_INTERLEAVED = 1 };/* channel 2m pairs with 2m + 1                       */
+/* How the G query heads that share a KV head are combined (the paper only says
+ * the analysis "extends to GQA"). */
+enum { EA_GROUP_MEAN_PROB = 0,   /* softmax per query head, mean over the group (default) */
+       EA_GROUP_SUM_PROB = 1,    /* softmax per query head, sum over the group            */
+       EA_GROUP_MEAN_LOGIT = 2 };/* mean of the log-scores over the group, one softmax    */
+/* Covariance normaliser. */
+enum { EA_COV_POPULATION = 0,    /* 1/W (Gaussian maximum likelihood, default)         */
+       EA_COV_SAMPLE = 1 };      /* 1/(W-1)                                            */
+
+typedef struct ea_shape {
+    int32_t n_units;     /* independent problems in this call: layers * batch          */
+    int32_t n_q_heads;   /* Hq                                                         */
+    int32_t n_kv_heads;  /* Hkv, divides Hq                                            */
+    int32_t head_dim;    /* d: 64, 128 or 256                                          */
+    int32_t n_keys;      /* n: cached keys per KV head (same for every unit)           */
+    int32_t window;      /* W: window queries per query head                           */
+    int32_t rope_layout; /* EA_ROPE_*                                                  */
+    int32_t group_mode;  /* EA_GROUP_*                                                 */
+    int32_t cov_norm;    /* EA_COV_*                                                   */
+} ea_shape;
+
+typedef struct ea_ctx ea_ctx;   /* opaque; owns its workspace and a status word */
+
+/* Library version string, e.g. "ea-b200 0.1". */
+const char* ea_version(void);
+const char* ea_status_string(ea_status s);
+
+/*
+ * Bytes of workspace the three calls need for this shape (the maximum over the
+ * calls; they reuse it).  HOST-only arithmetic, no CUDA call.
+ */
+ea_status ea_workspace_bytes(const ea_shape* shape, size_t* out_bytes);
+
+/*
+ * n_kept = int(n_keys * (1 - compression_ratio)) as the paper's pseudo-code
+ * computes it: product in double, truncated, clamped to [0, n_keys].  HOST-only.
+ */
+int64_t ea_n_kept(int64_t n_keys, double compression_ratio);
+
+/*
+ * Create a context on CUDA device `device` with a workspace of
+ * workspace_bytes (allocated once here with cudaMalloc; 0 is allowed and can
+ * only serve shapes that need none).  May synchronise.  Fails with
+ * EA_ERR_NOT_SM100 unless the device has compute capability 10.x.
+ */
+ea_status ea_create(ea_ctx** out_ctx, int device, size_t workspace_bytes);
+/* Frees the workspace.  The caller must have synchronised the streams used. */
+ea_status ea_destroy(ea_ctx* ctx);
+
+/*
+ * Query statistics with the rotary embedding averaged over the future
+ * positions (Eq. 5 and Eq. 6, queries given directly):
+ *   mu      = (1/W) sum_w u_w                  per query head
+ *   Sigma   = (1/N) sum_w (u_w-mu)(u_w-mu)^T   N = W or W-1 (cov_norm)
+ *   R_bar   = (1/T) sum_{p=pos_next}^{pos_next+T-1} R_p,  R_p the RoPE rotation
+ *             at position p with theta_m = rope_base^(-2m/d)
+ *   mu_bar  = R_bar mu,   sigma_bar = R_bar Sigma R_bar^T
+ *
+ * q_win     bf16 [n_units, Hq, W, d]  PRE-RoPE window queries, 16-byte aligned
+ * pos_next  int64 [n_units] DEVICE: 0-based position of the first future token
+ *           of each unit (n_keys for a prefill cache holding positions 0..n-1)
+ * n_future  T >= 1
+ * mu_bar    fp32 [n_units, Hq, d]      (output)
+ * sigma_bar fp32 [n_units, Hq, d, d]   (output, symmetric)
+ * shape->n_keys is ignored.  Requires W >= 1 (W >= 2 for EA_COV_SAMPLE).
+ */
+ea_status ea_query_stats(ea_ctx* ctx, const ea_shape* shape, const void* q_win,
+                         const int64_t* pos_next, int32_t n_future, double rope_base,
+                         float* mu_bar, float* sigma_bar, void* cuda_stream);
+
+/*
+ * Contribution score of every cached pair (Eq. 7, 8, 9 with ||v|| in place of
+ * ||W_o v||, as the paper's implementation note states):
+ *   s_{h,i}   = mu_bar_h . k_i / sqrt(d) + k_i^T sigma_bar_h k_i / (2d)
+ *   a_{h,i}   = exp(s_{h,i} - logsumexp_i s_{h,.})          softmax over the n keys
+ *   a_{g,i}   = group reduction of a_{h,i} over the G heads of KV head g (group_mode)
+ *   score_{g,i} = (a_{g,i} + epsilon) * ||v_{g,i}||_2
+ * Everything stays in the log domain until the softmax, so outlier-heavy
+ * activations do not overflow.
+ *
+ * k, v       bf16 [n_units, Hkv, n, d]; K is POST-RoPE; 16-byte aligned
+ * mu_bar     fp32 [n_units, Hq, d];  sigma_bar fp32 [n_units, Hq, d, d]
+ * scores     fp32 [n_units, Hkv, n]  (output)
+ * logits_opt fp32 [n_units, Hq, n] or NULL: when given, receives s_{h,i}
+ * shape->window is ignored.  n_keys == 0 or n_units == 0 is a no-op.
+ */
+ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
+                   const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
+                   float* logits_opt, void* cuda_stream);
+
+/*
+ * Eviction and compaction: per (unit, KV head) keep the n_kept pairs with the
+ * highest score; among equal scores the lowest index wins; kept indices are
+ * emitted in ascending order (the cache keeps its temporal order) and the
+ * K/V rows are gathered in that order.
+ *
+ * scores    fp32 [n_units, Hkv, n] (any finite values; -0 is treated as +0)
+ * n_kept    0 <= n_kept <= n_keys (EA_ERR_INVALID_ARG otherwise)
+ * k, v      bf16 [n_units, Hkv, n, d], 16-byte aligned
+ * kept_idx  int32 [n_units, Hkv, n_kept]        (output)
+ * k_out,v_out bf16 [n_units, Hkv, n_kept, d]    (output; must not overlap k, v)
+ *           k_out/v_out may both be NULL to skip the gather (indices only).
+ */
+ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                            int32_t n_kept, const void* k, const void* v, int32_t* kept_idx,
+                            void* k_out, void* v_out, void* cuda_stream);
+
+/*
+ * Synchronises cuda_stream and returns the device-side status recorded since
+ * the last call of this function (EA_OK, EA_ERR_DEVICE_TIMEOUT, or
+ * EA_ERR_CUDA if the stream reports an error), then clears it.
+ */
+ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EA_H_ */

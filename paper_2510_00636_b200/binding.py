@@ -1,0 +1,211 @@
+"""Thin ctypes binding of ``libea.so`` (see ``include/ea.h``).
+
+Argument marshalling only: torch supplies device memory and the current CUDA
+stream; every step of the path runs in the library's kernels.  There is no
+fallback: if the library is missing or the device is not a B200-class GPU the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libea.so")
+
+ROPE_HALF_SPLIT, ROPE_INTERLEAVED = 0, 1
+GROUP_MEAN_PROB, GROUP_SUM_PROB, GROUP_MEAN_LOGIT = 0, 1, 2
+COV_POPULATION, COV_SAMPLE = 0, 1
+
+EXPORTS = (
+    "ea_version", "ea_status_string", "ea_workspace_bytes", "ea_n_kept", "ea_create", "ea_destroy",
+    "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status",
+)
+
+
+class EAError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = lib().ea_status_string(status).decode()
+        super().__init__(f"{where} failed: {name} ({status})")
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "n_units", "n_q_heads", "n_kv_heads", "head_dim", "n_keys", "window", "rope_layout",
+        "group_mode", "cov_norm")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2510_00636_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32, f64 = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float,
+                                  ctypes.c_double)
+        sp = ctypes.POINTER(Shape)
+        L.ea_version.restype = ctypes.c_char_p
+        L.ea_status_string.restype = ctypes.c_char_p
+        L.ea_status_string.argtypes = [ctypes.c_int]
+        L.ea_workspace_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+        L.ea_n_kept.argtypes = [i64, f64]
+        L.ea_n_kept.restype = i64
+        L.ea_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int, ctypes.c_size_t]
+        L.ea_destroy.argtypes = [vp]
+        L.ea_query_stats.argtypes = [vp, sp, vp, vp, i32, f64, vp, vp, vp]
+        L.ea_score.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
+        L.ea_select_compact.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp]
+        L.ea_sync_status.argtypes = [vp, vp]
+        for name in ("ea_workspace_bytes", "ea_create", "ea_destroy", "ea_query_stats", "ea_score",
+                     "ea_select_compact", "ea_sync_status"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise EAError(status, where)
+
+
+def ea_n_kept(n_keys: int, compression_ratio: float) -> int:
+    return int(lib().ea_n_kept(int(n_keys), float(compression_ratio)))
+
+
+def ea_workspace_bytes(shape: Shape) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ea_workspace_bytes(ctypes.byref(shape), ctypes.byref(out)), "ea_workspace_bytes")
+    return int(out.value)
+
+
+def make_shape(n_units, n_q_heads, n_kv_heads, head_dim, n_keys, window, rope_layout=ROPE_HALF_SPLIT,
+               group_mode=GROUP_MEAN_PROB, cov_norm=COV_POPULATION) -> Shape:
+    return Shape(n_units, n_q_heads, n_kv_heads, head_dim, n_keys, window, rope_layout, group_mode,
+                 cov_norm)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _dev_tensor(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+class Context:
+    """Owns an ``ea_ctx`` (its workspace lives on ``device``)."""
+
+    def __init__(self, device: int | torch.device = 0, workspace_bytes: int = 0):
+        self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+        handle = ctypes.c_void_p()
+        _check(lib().ea_create(ctypes.byref(handle), self.device.index or 0, int(workspace_bytes)),
+               "ea_create")
+        self._h = handle
+        self.workspace_bytes = int(workspace_bytes)
+
+    @classmethod
+    def for_shape(cls, shape: Shape, device=0) -> "Context":
+        return cls(device, ea_workspace_bytes(shape))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().ea_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def sync_status(self):
+        _check(lib().ea_sync_status(self._h, _stream(self.device)), "ea_sync_status")
+
+
+def ea_query_stats(ctx: Context, shape: Shape, q_win, pos_next, n_future: int, rope_base: float,
+                   mu_bar=None, sigma_bar=None):
+    """q_win bf16 [U,Hq,W,d], pos_next int64 [U] (device) -> (mu_bar [U,Hq,d], sigma_bar [U,Hq,d,d])."""
+    _dev_tensor(q_win, torch.bfloat16, "q_win")
+    _dev_tensor(pos_next, torch.int64, "pos_next")
+    U, Hq, d = shape.n_units, shape.n_q_heads, shape.head_dim
+    if mu_bar is None:
+        mu_bar = torch.empty((U, Hq, d), dtype=torch.float32, device=q_win.device)
+    if sigma_bar is None:
+        sigma_bar = torch.empty((U, Hq, d, d), dtype=torch.float32, device=q_win.device)
+    _check(lib().ea_query_stats(ctx._h, ctypes.byref(shape), _ptr(q_win), _ptr(pos_next), int(n_future),
+                                float(rope_base), _ptr(mu_bar), _ptr(sigma_bar), _stream(ctx.device)),
+           "ea_query_stats")
+    return mu_bar, sigma_bar
+
+
+def ea_score(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, epsilon: float, scores=None,
+             logits=None, want_logits: bool = False):
+    """k, v bf16 [U,Hkv,n,d] -> scores fp32 [U,Hkv,n] (and the log-scores [U,Hq,n] if asked)."""
+    _dev_tensor(k, torch.bfloat16, "k")
+    _dev_tensor(v, torch.bfloat16, "v")
+    _dev_tensor(mu_bar, torch.float32, "mu_bar")
+    _dev_tensor(sigma_bar, torch.float32, "sigma_bar")
+    U, Hq, Hkv, n = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys
+    if scores is None:
+        scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=k.device)
+    if logits is None and want_logits:
+        logits = torch.empty((U, Hq, n), dtype=torch.float32, device=k.device)
+    _check(lib().ea_score(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(mu_bar), _ptr(sigma_bar),
+                          float(epsilon), _ptr(scores), _ptr(logits), _stream(ctx.device)), "ea_score")
+    return (scores, logits) if (want_logits or logits is not None) else scores
+
+
+def ea_select_compact(ctx: Context, shape: Shape, scores, n_kept: int, k=None, v=None, kept_idx=None,
+                      k_out=None, v_out=None, gather: bool = True):
+    """scores fp32 [U,Hkv,n] -> (kept_idx int32 [U,Hkv,n_kept], k_out, v_out bf16 [U,Hkv,n_kept,d])."""
+    _dev_tensor(scores, torch.float32, "scores")
+    U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
+    if kept_idx is None:
+        kept_idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, device=scores.device)
+    if gather:
+        _dev_tensor(k, torch.bfloat16, "k")
+        _dev_tensor(v, torch.bfloat16, "v")
+        if k_out is None:
+            k_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.bfloat16, device=scores.device)
+        if v_out is None:
+            v_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.bfloat16, device=scores.device)
+    _check(lib().ea_select_compact(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k),
+                                   _ptr(v), _ptr(kept_idx), _ptr(k_out), _ptr(v_out),
+                                   _stream(ctx.device)), "ea_select_compact")
+    return kept_idx, k_out, v_out
+
+
+@dataclass
+class Compressed:
+    mu_bar: torch.Tensor
+    sigma_bar: torch.Tensor
+    scores: torch.Tensor
+    logits: torch.Tensor | None
+    kept_idx: torch.Tensor
+    k_out: torch.Tensor
+    v_out: torch.Tensor
+
+
+def compress(ctx: Context, shape: Shape, q_win, k, v, pos_next, n_future, rope_base, epsilon, n_kept,
+             want_logits: bool = False) -> Compressed:
+    """The three calls back to back on the current stream."""
+    mu_bar, sigma_bar = ea_query_stats(ctx, shape, q_win, pos_next, n_future, rope_base)
+    res = ea_score(ctx, shape, k, v, mu_bar, sigma_bar, epsilon, want_logits=want_logits)
+    scores, logits = res if want_logits else (res, None)
+    kept_idx, k_out, v_out = ea_select_compact(ctx, shape, scores, n_kept, k, v)
+    return Compressed(mu_bar, sigma_bar, scores, logits, kept_idx, k_out, v_out)

@@ -1,0 +1,226 @@
+// Host side of the C ABI: argument validation, workspace planning, context
+// lifetime, and the order of kernel launches of each call.
+#include <new>
+
+#include "ea_internal.h"
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+ea_status check_shape(const ea_shape* s) {
+    if (!s) return EA_ERR_INVALID_ARG;
+    if (s->n_units < 0 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->n_keys < 0 || s->window < 0)
+        return EA_ERR_INVALID_ARG;
+    if (s->n_q_heads % s->n_kv_heads != 0) return EA_ERR_INVALID_ARG;
+    if (s->rope_layout != EA_ROPE_HALF_SPLIT && s->rope_layout != EA_ROPE_INTERLEAVED)
+        return EA_ERR_INVALID_ARG;
+    if (s->group_mode < EA_GROUP_MEAN_PROB || s->group_mode > EA_GROUP_MEAN_LOGIT)
+        return EA_ERR_INVALID_ARG;
+    if (s->cov_norm != EA_COV_POPULATION && s->cov_norm != EA_COV_SAMPLE) return EA_ERR_INVALID_ARG;
+    if (s->head_dim != 64 && s->head_dim != 128 && s->head_dim != 256) return EA_ERR_UNSUPPORTED;
+    // grid dimension limits of the per-head launches
+    if ((long long)s->n_units * s->n_q_heads > 65535LL * 1024) return EA_ERR_UNSUPPORTED;
+    return EA_OK;
+}
+
+}  // namespace
+
+ea_ws_plan ea_plan_workspace(const ea_shape& s) {
+    ea_ws_plan p;
+    size_t off = 0;
+    const size_t U = (size_t)s.n_units, Hq = (size_t)s.n_q_heads, Hkv = (size_t)s.n_kv_heads;
+    const size_t n = (size_t)s.n_keys, d = (size_t)s.head_dim;
+    p.rope_coef = off;  off = ea_align_up(off + U * (d / 2) * 2 * sizeof(float), 256);
+    p.logits = off;     off = ea_align_up(off + U * Hq * n * sizeof(float), 256);
+    p.lse = off;        off = ea_align_up(off + U * Hq * sizeof(float), 256);
+    p.sel_state = off;  off = ea_align_up(off + U * Hkv * 4 * sizeof(uint32_t), 256);
+    p.total = off;
+    return p;
+}
+
+extern "C" {
+
+const char* ea_version(void) { return "ea-b200 0.1"; }
+
+const char* ea_status_string(ea_status s) {
+    switch (s) {
+        case EA_OK: return "EA_OK";
+        case EA_ERR_INVALID_ARG: return "EA_ERR_INVALID_ARG";
+        case EA_ERR_UNSUPPORTED: return "EA_ERR_UNSUPPORTED";
+        case EA_ERR_WORKSPACE: return "EA_ERR_WORKSPACE";
+        case EA_ERR_CUDA: return "EA_ERR_CUDA";
+        case EA_ERR_NOT_SM100: return "EA_ERR_NOT_SM100";
+        case EA_ERR_DEVICE_TIMEOUT: return "EA_ERR_DEVICE_TIMEOUT";
+    }
+    return "EA_ERR_UNKNOWN";
+}
+
+ea_status ea_workspace_bytes(const ea_shape* shape, size_t* out_bytes) {
+    if (!out_bytes) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    *out_bytes = ea_plan_workspace(*shape).total;
+    return EA_OK;
+}
+
+int64_t ea_n_kept(int64_t n_keys, double compression_ratio) {
+    if (n_keys <= 0) return 0;
+    const double x = (double)n_keys * (1.0 - compression_ratio);
+    if (!(x > 0.0)) return 0;
+    if (x >= (double)n_keys) return n_keys;
+    return (int64_t)x;
+}
+
+ea_status ea_create(ea_ctx** out_ctx, int device, size_t workspace_bytes) {
+    if (!out_ctx) return EA_ERR_INVALID_ARG;
+    *out_ctx = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return EA_ERR_CUDA; }
+    if (device < 0 || device >= count) return EA_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    EA_CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return EA_ERR_NOT_SM100;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    EA_CUDA_TRY(cudaSetDevice(device));
+    ea_ctx* ctx = new (std::nothrow) ea_ctx();
+    if (!ctx) { cudaSetDevice(prev); return EA_ERR_CUDA; }
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->workspace = nullptr;
+    ctx->workspace_bytes = workspace_bytes;
+    ctx->status_host = nullptr;
+    ctx->status_dev = nullptr;
+    bool ok = true;
+    if (workspace_bytes > 0) ok = cudaMalloc(&ctx->workspace, workspace_bytes) == cudaSuccess;
+    if (ok) ok = cudaHostAlloc((void**)&ctx->status_host, sizeof(int), cudaHostAllocMapped) == cudaSuccess;
+    if (ok) {
+        *ctx->status_host = 0;
+        ok = cudaHostGetDevicePointer((void**)&ctx->status_dev, ctx->status_host, 0) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        if (ctx->workspace) cudaFree(ctx->workspace);
+        if (ctx->status_host) cudaFreeHost(ctx->status_host);
+        delete ctx;
+        cudaSetDevice(prev);
+        return EA_ERR_CUDA;
+    }
+    cudaSetDevice(prev);
+    *out_ctx = ctx;
+    return EA_OK;
+}
+
+ea_status ea_destroy(ea_ctx* ctx) {
+    if (!ctx) return EA_OK;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->device);
+    if (ctx->workspace) cudaFree(ctx->workspace);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    cudaSetDevice(prev);
+    delete ctx;
+    return EA_OK;
+}
+
+ea_status ea_query_stats(ea_ctx* ctx, const ea_shape* shape, const void* q_win,
+                         const int64_t* pos_next, int32_t n_future, double rope_base,
+                         float* mu_bar, float* sigma_bar, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (shape->n_units == 0) return EA_OK;
+    if (!q_win || !pos_next || !mu_bar || !sigma_bar) return EA_ERR_INVALID_ARG;
+    if (!aligned16(q_win) || !aligned16(mu_bar) || !aligned16(sigma_bar)) return EA_ERR_INVALID_ARG;
+    if (n_future < 1 || !(rope_base > 0.0)) return EA_ERR_INVALID_ARG;
+    if (shape->window < 1 || (shape->cov_norm == EA_COV_SAMPLE && shape->window < 2))
+        return EA_ERR_INVALID_ARG;
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    if (ctx->workspace_bytes < plan.logits /* rope_coef region only */) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    float* coef = reinterpret_cast<float*>(static_cast<char*>(ctx->workspace) + plan.rope_coef);
+    st = ea_launch_stats(ctx, *shape, static_cast<const __nv_bfloat16*>(q_win), pos_next, n_future,
+                         rope_base, coef, mu_bar, sigma_bar, static_cast<cudaStream_t>(cuda_stream));
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
+                   const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
+                   float* logits_opt, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (shape->n_units == 0 || shape->n_keys == 0) return EA_OK;
+    if (!k || !v || !mu_bar || !sigma_bar || !scores) return EA_ERR_INVALID_ARG;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(mu_bar) || !aligned16(sigma_bar) ||
+        !aligned16(scores) || !aligned16(logits_opt))
+        return EA_ERR_INVALID_ARG;
+    if (!(epsilon >= 0.0f)) return EA_ERR_INVALID_ARG;
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    if (ctx->workspace_bytes < plan.total) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    char* ws = static_cast<char*>(ctx->workspace);
+    float* logits = logits_opt ? logits_opt : reinterpret_cast<float*>(ws + plan.logits);
+    float* lse = reinterpret_cast<float*>(ws + plan.lse);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = ea_launch_logits_simt(ctx, *shape, static_cast<const __nv_bfloat16*>(k), mu_bar, sigma_bar,
+                               logits, stream);
+    if (st == EA_OK)
+        st = ea_launch_finalize(ctx, *shape, logits, static_cast<const __nv_bfloat16*>(v), epsilon, lse,
+                                scores, stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                            int32_t n_kept, const void* k, const void* v, int32_t* kept_idx,
+                            void* k_out, void* v_out, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (n_kept < 0 || n_kept > shape->n_keys) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0 || n_kept == 0) return EA_OK;
+    if (!scores || !kept_idx) return EA_ERR_INVALID_ARG;
+    const bool do_gather = k_out != nullptr || v_out != nullptr;
+    if (do_gather && (!k || !v || !k_out || !v_out)) return EA_ERR_INVALID_ARG;
+    if (!aligned16(scores) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+        return EA_ERR_INVALID_ARG;
+    if (do_gather) {
+        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys *
+                                shape->head_dim * sizeof(__nv_bfloat16);
+        const size_t out_bytes = (size_t)shape->n_units * shape->n_kv_heads * n_kept *
+                                 shape->head_dim * sizeof(__nv_bfloat16);
+        const char* ins[2] = {static_cast<const char*>(k), static_cast<const char*>(v)};
+        const char* outs[2] = {static_cast<const char*>(k_out), static_cast<const char*>(v_out)};
+        for (const char* o : outs)
+            for (const char* i : ins)
+                if (o < i + in_bytes && i < o + out_bytes) return EA_ERR_INVALID_ARG;
+    }
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = ea_launch_select(ctx, *shape, scores, n_kept, kept_idx, stream);
+    if (st == EA_OK && do_gather)
+        st = ea_launch_gather(ctx, *shape, n_kept, kept_idx, static_cast<const __nv_bfloat16*>(k),
+                              static_cast<const __nv_bfloat16*>(v), static_cast<__nv_bfloat16*>(k_out),
+                              static_cast<__nv_bfloat16*>(v_out), stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return EA_ERR_CUDA;
+    const int s = *ctx->status_host;
+    *ctx->status_host = 0;
+    return s == 0 ? EA_OK : static_cast<ea_status>(s);
+}
+
+}  // extern "C"

@@ -1,0 +1,58 @@
+// Internal declarations shared by the translation units of libea.so.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "ea.h"
+
+struct ea_ctx {
+    int device;
+    int sm_count;
+    void* workspace;
+    size_t workspace_bytes;
+    int* status_host;    // pinned, mapped: device kernels write EA_ERR_DEVICE_TIMEOUT here
+    int* status_dev;     // device alias of status_host
+};
+
+// Byte offsets of the workspace regions.  Regions of different calls overlap
+// on purpose except where one call's output feeds the next.
+struct ea_ws_plan {
+    size_t rope_coef;    // fp32 [U, d/2, 2]             (ea_query_stats)
+    size_t logits;       // fp32 [U, Hq, n]              (ea_score, when logits_opt == NULL)
+    size_t lse;          // fp32 [U, Hq]                 (ea_score)
+    size_t sel_state;    // uint32 [U*Hkv, 4]            (ea_select_compact)
+    size_t total;
+};
+
+ea_ws_plan ea_plan_workspace(const ea_shape& s);
+
+#define EA_CUDA_TRY(expr)                                   \
+    do {                                                    \
+        cudaError_t err__ = (expr);                         \
+        if (err__ != cudaSuccess) return EA_ERR_CUDA;       \
+    } while (0)
+
+static inline size_t ea_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- launchers (each returns EA_OK or EA_ERR_CUDA from cudaGetLastError) ----
+ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
+                          const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
+                          float* mu_bar, float* sigma_bar, cudaStream_t st);
+
+ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
+                                const float* mu_bar, const float* sigma_bar, float* logits,
+                                cudaStream_t st);
+
+ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
+                             const __nv_bfloat16* v, float epsilon, float* lse, float* scores,
+                             cudaStream_t st);
+
+ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
+                           int32_t* kept_idx, cudaStream_t st);
+
+ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
+                           const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* k_out,
+                           __nv_bfloat16* v_out, cudaStream_t st);

@@ -1,0 +1,155 @@
+// Softmax over positions, GQA reduction and value-norm weighting
+// (Eq. 8 and Eq. 9 of the paper with ||v|| in place of ||W_o v||).
+//
+// lse_kernel: one CTA per softmax row, max-subtracted log-sum-exp with a fixed
+// reduction order (bitwise reproducible).
+// finalize_kernel: one warp per 32 consecutive keys of a KV head.  The warp
+// streams the 32 value rows with 128-bit loads (sum of squares in fp32,
+// shuffle-reduced), then lane r finishes key r: coalesced log-score loads,
+// exp(s - lse) per query head of the group, (a + eps) * ||v||.
+#include "ea_internal.h"
+
+namespace {
+
+constexpr int kLseThreads = 1024;
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float* scratch) {
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        float o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = is_max ? fmaxf(v, o) : v + o;
+    }
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        v = scratch[lane];   // kLseThreads / 32 == 32 partials
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            float o = __shfl_xor_sync(0xffffffffu, v, off);
+            v = is_max ? fmaxf(v, o) : v + o;
+        }
+        if (lane == 0) scratch[0] = v;
+    }
+    __syncthreads();
+    return scratch[0];
+}
+
+// Row r of the softmax is the mean over `g_avg` consecutive log-score rows
+// (g_avg = 1: every query head has its own softmax).
+__global__ void __launch_bounds__(kLseThreads)
+lse_kernel(const float* __restrict__ logits, int n, int g_avg, float* __restrict__ lse) {
+    __shared__ float scratch[32];
+    const float* base = logits + (size_t)blockIdx.x * g_avg * n;
+    const float inv_g = 1.0f / (float)g_avg;
+    float mx = -INFINITY;
+    for (int i = threadIdx.x; i < n; i += kLseThreads) {
+        float x = 0.f;
+        for (int j = 0; j < g_avg; ++j) x += base[(size_t)j * n + i];
+        mx = fmaxf(mx, x * inv_g);
+    }
+    mx = block_reduce(mx, true, scratch);
+    float sum = 0.f;
+    for (int i = threadIdx.x; i < n; i += kLseThreads) {
+        float x = 0.f;
+        for (int j = 0; j < g_avg; ++j) x += base[(size_t)j * n + i];
+        sum += expf(x * inv_g - mx);
+    }
+    sum = block_reduce(sum, false, scratch);
+    if (threadIdx.x == 0) lse[blockIdx.x] = mx + logf(sum);
+}
+
+constexpr int kFinThreads = 256;
+
+template <int D>
+__global__ void __launch_bounds__(kFinThreads)
+finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
+                const __nv_bfloat16* __restrict__ v, int Hq, int Hkv, int n, int group_mode,
+                float epsilon, float* __restrict__ scores) {
+    constexpr int LPR = D / 8;          // lanes per value row (one uint4 = 8 bf16 each)
+    constexpr int RPS = 32 / LPR;       // rows per load step
+    constexpr int STEPS = 32 / RPS;
+    const int G = Hq / Hkv;
+    const int ug = blockIdx.y;
+    const int u = ug / Hkv, g = ug % Hkv;
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int key0 = (blockIdx.x * (kFinThreads / 32) + warp) * 32;
+    if (key0 >= n) return;
+
+    const uint4* vrow = reinterpret_cast<const uint4*>(v + ((size_t)ug * n + key0) * D);
+    float my_sumsq = 0.f;
+#pragma unroll 4
+    for (int t = 0; t < STEPS; ++t) {
+        const int r = t * RPS + lane / LPR;
+        float ss = 0.f;
+        if (key0 + r < n) {
+            const uint4 x = __ldg(vrow + (size_t)r * LPR + lane % LPR);
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float lo = __uint_as_float(w[q] << 16);
+                const float hi = __uint_as_float(w[q] & 0xffff0000u);
+                ss = fmaf(lo, lo, ss);
+                ss = fmaf(hi, hi, ss);
+            }
+        }
+#pragma unroll
+        for (int off = LPR / 2; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        // lane L owns key L: its row was summed in step L / RPS by lane group L % RPS
+        const float mine = __shfl_sync(0xffffffffu, ss, (lane % RPS) * LPR);
+        if (t == lane / RPS) my_sumsq = mine;
+    }
+
+    const int key = key0 + lane;
+    if (key >= n) return;
+    float a;
+    if (group_mode == EA_GROUP_MEAN_LOGIT) {
+        float x = 0.f;
+        for (int j = 0; j < G; ++j) x += logits[((size_t)u * Hq + (size_t)g * G + j) * n + key];
+        a = expf(x * (1.0f / (float)G) - lse[ug]);
+    } else {
+        a = 0.f;
+        for (int j = 0; j < G; ++j) {
+            const size_t uh = (size_t)u * Hq + (size_t)g * G + j;
+            a += expf(logits[uh * n + key] - lse[uh]);
+        }
+        if (group_mode == EA_GROUP_MEAN_PROB) a *= 1.0f / (float)G;
+    }
+    scores[(size_t)ug * n + key] = (a + epsilon) * sqrtf(my_sumsq);
+}
+
+}  // namespace
+
+ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
+                             const __nv_bfloat16* v, float epsilon, float* lse, float* scores,
+                             cudaStream_t st) {
+    (void)ctx;
+    const int G = s.n_q_heads / s.n_kv_heads;
+    if (s.group_mode == EA_GROUP_MEAN_LOGIT)
+        lse_kernel<<<s.n_units * s.n_kv_heads, kLseThreads, 0, st>>>(logits, s.n_keys, G, lse);
+    else
+        lse_kernel<<<s.n_units * s.n_q_heads, kLseThreads, 0, st>>>(logits, s.n_keys, 1, lse);
+    const int keys_per_cta = kFinThreads;   // 8 warps x 32 keys
+    dim3 grid((unsigned)((s.n_keys + keys_per_cta - 1) / keys_per_cta),
+              (unsigned)(s.n_units * s.n_kv_heads));
+    switch (s.head_dim) {
+        case 64:
+            finalize_kernel<64><<<grid, kFinThreads, 0, st>>>(logits, lse, v, s.n_q_heads, s.n_kv_heads,
+                                                             s.n_keys, s.group_mode, epsilon, scores);
+            break;
+        case 128:
+            finalize_kernel<128><<<grid, kFinThreads, 0, st>>>(logits, lse, v, s.n_q_heads,
+                                                              s.n_kv_heads, s.n_keys, s.group_mode,
+                                                              epsilon, scores);
+            break;
+        case 256:
+            finalize_kernel<256><<<grid, kFinThreads, 0, st>>>(logits, lse, v, s.n_q_heads,
+                                                              s.n_kv_heads, s.n_keys, s.group_mode,
+                                                              epsilon, scores);
+            break;
+        default:
+            return EA_ERR_UNSUPPORTED;
+    }
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}

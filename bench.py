@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the Expected Attention scoring + pruning hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 3] [--impl ours|reference]
+
+One step = one pass of the whole path (query statistics, scoring, selection and compaction)
+over every layer of a synthetic, model-shaped KV cache that is already resident in HBM.  The
+default workload is the Gemma3-12B-shaped 128k-token cache (48 layers, 51.5 GB of K+V).  The
+JSON line carries the whole-job throughput in Gkeys/s, the same metric end to end from host
+buffers (``e2e``), the roofline of the dominant kernel, and the fp64 CPU oracle timed on a
+bounded sample of the same workload (``cpu_baseline``).
+
+With N > 1 (torchrun, one rank per GPU) every rank runs its own replica of the workload: units
+are independent, no data-path collective exists.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2510_00636_b200 import inputs  # noqa: E402
+
+METRIC = "kv_keys_scored_and_compacted_per_second"
+UNIT = "Gkeys/s"
+
+
+def measured_peaks():
+    """Roofline denominators: measured on this machine if the file is present, else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), tflops=float(p["bf16_tflops_sustained"]), source="measured")
+    return dict(hbm_gbs=6650.0, tflops=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------- workload
+class Workload:
+    """All layers of one config resident in HBM, plus preallocated outputs."""
+
+    def __init__(self, cfg: inputs.EAConfig, device, ea):
+        self.cfg, self.device, self.ea = cfg, device, ea
+        L, B = cfg.n_layers, cfg.batch
+        U, Hq, Hkv, d, n, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window
+        bf, f32 = torch.bfloat16, torch.float32
+        self.k = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
+        self.v = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
+        self.q = torch.empty((U, Hq, W, d), dtype=bf, device=device)
+        self.pos = torch.empty((U,), dtype=torch.int64, device=device)
+        for layer in range(L):
+            q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device=device)
+            sl = slice(layer * B, (layer + 1) * B)
+            self.q[sl], self.k[sl], self.v[sl], self.pos[sl] = q, k, v, pos.to(device)
+            del q, k, v
+        self.mu = torch.empty((U, Hq, d), dtype=f32, device=device)
+        self.sigma = torch.empty((U, Hq, d, d), dtype=f32, device=device)
+        self.scores = torch.empty((U, Hkv, n), dtype=f32, device=device)
+        self.idx = torch.empty((U, Hkv, cfg.n_kept), dtype=torch.int32, device=device)
+        self.k_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
+        self.v_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
+        self.n_units = U
+
+    def make_ctx(self, units_per_call):
+        cfg = self.cfg
+        shape = self.ea.make_shape(units_per_call, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys,
+                                   cfg.window)
+        return self.ea.Context.for_shape(shape, self.device.index)
+
+    def step(self, ctx, units_per_call):
+        """One pass of the whole path over every unit, `units_per_call` units per library call."""
+        ea, cfg = self.ea, self.cfg
+        for u0 in range(0, self.n_units, units_per_call):
+            u1 = min(self.n_units, u0 + units_per_call)
+            shape = ea.make_shape(u1 - u0, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window)
+            ea.ea_query_stats(ctx, shape, self.q[u0:u1], self.pos[u0:u1], cfg.n_future, cfg.rope_base,
+                              self.mu[u0:u1], self.sigma[u0:u1])
+            ea.ea_score(ctx, shape, self.k[u0:u1], self.v[u0:u1], self.mu[u0:u1], self.sigma[u0:u1], cfg.eps,
+                        self.scores[u0:u1])
+            ea.ea_select_compact(ctx, shape, self.scores[u0:u1], cfg.n_kept, self.k[u0:u1], self.v[u0:u1],
+                                 self.idx[u0:u1], self.k_out[u0:u1], self.v_out[u0:u1])
+
+
+def algorithmic_work(cfg: inputs.EAConfig):
+    """Per step: key-slots, algorithmic HBM bytes (read K, read V, write kept K and V) and the
+    FLOPs of the quadratic form k^T Sigma k for each query head (2 d^2 G per key-slot)."""
+    slots = cfg.key_slots
+    d, G = cfg.head_dim, cfg.group
+    bytes_ = slots * 4 * d + cfg.n_units * cfg.n_kv_heads * cfg.n_kept * 4 * d
+    flops = slots * 2 * d * d * G
+    return slots, bytes_, flops
+
+
+# ------------------------------------------------------------------------------------- distributed
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(cfg: inputs.EAConfig, target_seconds=15.0):
+    """A bounded sample of the workload for the fp64 oracle: layer 0, every head, the first
+    `n_sample` keys, sized for roughly `target_seconds` of CPU work (about 2 GFLOP/s/core)."""
+    cores = len(os.sched_getaffinity(0))
+    per_key = 2.0 * cfg.head_dim ** 2 * cfg.n_q_heads * cfg.batch          # fp64 FLOPs per key index
+    n_sample = int(target_seconds * 2.0e9 * min(cores, cfg.n_q_heads * cfg.batch) / per_key)
+    n_sample = max(256, min(cfg.n_keys, n_sample // 256 * 256))
+    return n_sample
+
+
+def time_oracle(cfg, n_sample, repeats=1):
+    from oracle import ea_oracle
+    q, k, v, pos = inputs.generate_layer(cfg, layer=0, device="cpu", n_keys=n_sample)
+    qb, kb, vb = inputs.bits(q), inputs.bits(k), inputs.bits(v)
+    n_kept = max(1, int(round(n_sample * cfg.n_kept / cfg.n_keys)))
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        ea_oracle.compress(qb, kb, vb, pos.numpy(), cfg.n_future, cfg.rope_base, cfg.eps, n_kept)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    slots = cfg.batch * cfg.n_kv_heads * n_sample
+    return slots, best, ea_oracle.num_threads()
+
+
+def run_reference(args, cfg):
+    """The reference arm: the fp64 CPU oracle, as it stands, on the host cores."""
+    world, rank = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_sample = oracle_sample(cfg, target_seconds=8.0)
+    from oracle import ea_oracle
+    q, k, v, pos = inputs.generate_layer(cfg, layer=0, device="cpu", n_keys=n_sample)
+    qb, kb, vb = inputs.bits(q), inputs.bits(k), inputs.bits(v)
+    n_kept = max(1, int(round(n_sample * cfg.n_kept / cfg.n_keys)))
+    run = lambda: ea_oracle.compress(qb, kb, vb, pos.numpy(), cfg.n_future, cfg.rope_base, cfg.eps, n_kept)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = (time.perf_counter() - t0) / args.steps
+    slots = cfg.batch * cfg.n_kv_heads * n_sample
+    value = slots / dt / 1e9
+    sample = f"layer 0, all {cfg.n_kv_heads} KV heads, first {n_sample} of {cfg.n_keys} keys ({slots} key-slots) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": ea_oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3])
+    ap.add_argument("--units-per-call", type=int, default=0, help="layers per library call (0 = all)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = inputs.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+    if args.warmup < 3:
+        print("note: fewer than 3 warm-up steps requested", file=sys.stderr)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    world, rank, local = dist_setup(args.gpus)
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    from paper_2510_00636_b200 import binding as ea
+    ea.lib()
+
+    wl = Workload(cfg, device, ea)
+    upc = args.units_per_call or wl.n_units
+    ctx = wl.make_ctx(upc)
+    slots, alg_bytes, alg_flops = algorithmic_work(cfg)
+    peaks = measured_peaks()
+
+    for _ in range(args.warmup):
+        wl.step(ctx, upc)
+    ctx.sync_status()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier(world)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ctx.profile_begin()
+    ev0.record()
+    for _ in range(args.steps):
+        wl.step(ctx, upc)
+    ev1.record()
+    score_ms, score_launches, total_launches = ctx.profile_end()
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop()
+    ms_local = ev0.elapsed_time(ev1) / args.steps
+    ms = max_over_ranks(ms_local, world, device)
+    ctx.sync_status()
+
+    # roofline of the dominant kernel (the log-score kernel, Eq. 7)
+    n_calls = (wl.n_units + upc - 1) // upc
+    avg_score_ms = score_ms / max(1, score_launches)
+    flops_per_launch = alg_flops / n_calls
+    bytes_per_launch = slots * 2 * cfg.head_dim / n_calls            # the K rows this kernel must read
+    t_tensor = flops_per_launch / (peaks["tflops"] * 1e12)
+    t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        achieved = flops_per_launch / (avg_score_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["tflops"]}
+    else:
+        achieved = bytes_per_launch / (avg_score_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"]}
+    roofline.update({"traffic": None, "kernel": "log-score kernel (k.mu/sqrt(d) + k'Sigma k/2d)",
+                     "kernel_ms": avg_score_ms, "launches_timed": score_launches,
+                     "peak_source": peaks["source"] + " (sustained bf16 matmul)"})
+    # whole-path roofline: the slower of the K.Sigma FLOPs at tensor peak and the K/V bytes at HBM bandwidth
+    t_path = max(alg_flops / (peaks["tflops"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9))
+    path_frac = t_path / (ms * 1e-3)
+
+    result = {
+        "metric": METRIC, "value": world * slots / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": cfg.n_layers, "batch": cfg.batch,
+                   "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
+                   "n_keys": cfg.n_keys, "window": cfg.window, "n_kept": cfg.n_kept,
+                   "key_slots_per_step": slots, "units_per_call": upc, "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (K+V %.1f GB per step)" % (slots * 4 * cfg.head_dim / 1e9)},
+        "ms_per_128k_compression": ms if cfg.cfg_id == 3 else None,
+        "path_roofline": {"t_roof_ms": t_path * 1e3, "frac": path_frac, "alg_bytes": alg_bytes,
+                          "alg_flops": alg_flops, "peak_source": peaks["source"]},
+        "roofline": roofline,
+        "gpu_launches": int(total_launches),
+        "clocks": clocks,
+    }
+
+    # end to end from host buffers through ea_compress_host (rank-local; max over ranks)
+    if not args.skip_e2e:
+        result["e2e"] = run_e2e(args, cfg, wl, ea, device, world, slots)
+
+    if rank == 0 and world == 1 and not args.skip_cpu_baseline:
+        n_sample = oracle_sample(cfg)
+        o_slots, o_s, cores = time_oracle(cfg, n_sample)
+        result["cpu_baseline"] = {
+            "value": o_slots / o_s / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"layer 0, all {cfg.n_kv_heads} KV heads, first {n_sample} of {cfg.n_keys} keys "
+                      f"({o_slots} key-slots, {o_s:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_e2e(args, cfg, wl, ea, device, world, slots):
+    """Same metric with HOST buffers: every step copies each layer's Q/K/V host->device and the
+    kept indices and compacted K/V device->host inside the timed region (ea_compress_host, one
+    layer per chunk).  The pinned host pool holds `pool` distinct layers that the 48 layers
+    cycle through, so the bytes moved per step are those of the full cache."""
+    L, B = cfg.n_layers, cfg.batch
+    pool = min(L, 4)
+    U = pool * B
+    shape = ea.make_shape(U, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window)
+    hq = wl.q[:U].cpu().pin_memory()
+    hk = wl.k[:U].cpu().pin_memory()
+    hv = wl.v[:U].cpu().pin_memory()
+    hpos = wl.pos[:U].cpu().pin_memory()
+    hidx = torch.empty((U, cfg.n_kv_heads, cfg.n_kept), dtype=torch.int32).pin_memory()
+    hko = torch.empty((U, cfg.n_kv_heads, cfg.n_kept, cfg.head_dim), dtype=torch.bfloat16).pin_memory()
+    hvo = torch.empty_like(hko).pin_memory()
+    ctx = ea.Context(device.index, ea.ea_host_workspace_bytes(shape, cfg.n_kept, B))
+    rounds = (L + pool - 1) // pool            # passes over the pool per step
+    h2d = rounds * (hq.numel() + hk.numel() + hv.numel()) * 2 + rounds * hpos.numel() * 8
+    d2h = rounds * (hidx.numel() * 4 + (hko.numel() + hvo.numel()) * 2)
+    units_done = rounds * U
+
+    def one_step():
+        for _ in range(rounds):
+            ea.ea_compress_host(ctx, shape, hq, hk, hv, hpos, cfg.n_future, cfg.rope_base, cfg.eps, cfg.n_kept,
+                                B, hidx, hko, hvo)
+
+    one_step()
+    ctx.sync_status()
+    barrier(world)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.e2e_steps):
+        one_step()
+    ev1.record()
+    torch.cuda.synchronize()
+    ctx.sync_status()
+    ms = max_over_ranks(ev0.elapsed_time(ev1) / args.e2e_steps, world, device)
+    # the device result of the same layers must be what came back
+    ok = bool(torch.equal(hidx[:B], wl.idx[:B].cpu()))
+    e_slots = units_done * cfg.n_kv_heads * cfg.n_keys
+    return {"value": world * e_slots / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
+            "host_pool_layers": pool, "key_slots_per_step": e_slots, "matches_device_path": ok}
+
+
+if __name__ == "__main__":
+    main()

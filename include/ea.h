@@ -172,6 +172,50 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
  */
 ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream);
 
+/*
+ * The whole routine on HOST buffers: compress(queries, keys, values) ->
+ * (kept indices, keys[idx], values[idx]) as in the paper's pseudo-code, for
+ * callers whose cache lives in host memory.  Units are processed in chunks of
+ * units_per_chunk; each chunk is copied to the device, run through
+ * ea_query_stats, ea_score and ea_select_compact, and its results copied
+ * back, with the copies of neighbouring chunks overlapping the kernels (two
+ * staging buffers, two internal copy streams).  Every pointer here is a HOST
+ * pointer; pinned memory (cudaHostAlloc / cudaHostRegister) is needed for the
+ * copies to overlap, pageable memory works but serialises.  The call returns
+ * after enqueuing; the host buffers must stay valid and untouched until
+ * cuda_stream has been synchronised (ea_sync_status does that).
+ *
+ * shape            sizes of the WHOLE problem (n_units = all units)
+ * q_win,k,v        bf16 host arrays shaped as for the device calls
+ * pos_next         int64 [n_units] host
+ * kept_idx         int32 [n_units, Hkv, n_kept] host (output)
+ * k_out, v_out     bf16 [n_units, Hkv, n_kept, d] host (output)
+ * scores_opt       fp32 [n_units, Hkv, n] host or NULL (output)
+ * The context's workspace must hold ea_host_workspace_bytes(shape, n_kept,
+ * units_per_chunk) bytes (staging for two chunks plus the kernels' workspace).
+ */
+ea_status ea_host_workspace_bytes(const ea_shape* shape, int32_t n_kept, int32_t units_per_chunk,
+                                  size_t* out_bytes);
+ea_status ea_compress_host(ea_ctx* ctx, const ea_shape* shape, const void* q_win, const void* k,
+                           const void* v, const int64_t* pos_next, int32_t n_future,
+                           double rope_base, float epsilon, int32_t n_kept, int32_t units_per_chunk,
+                           int32_t* kept_idx, void* k_out, void* v_out, float* scores_opt,
+                           void* cuda_stream);
+
+/*
+ * Instrumentation for benchmarks (the paper has no counterpart).  Between
+ * ea_profile_begin and ea_profile_end the context counts every kernel it
+ * launches and brackets each launch of the log-score kernel (Eq. 7, the
+ * dominant kernel) with CUDA events on the caller's stream.  ea_profile_end
+ * synchronises cuda_stream and reports the summed device time of those
+ * launches in milliseconds, how many there were, and the total number of
+ * kernel launches.  At most 4096 log-score launches are timed per window;
+ * later ones are counted but not timed (timed_launches tells how many were).
+ */
+ea_status ea_profile_begin(ea_ctx* ctx);
+ea_status ea_profile_end(ea_ctx* ctx, void* cuda_stream, double* score_kernel_ms,
+                         int64_t* timed_launches, int64_t* total_kernel_launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ COV_POPULATION, COV_SAMPLE = 0, 1
 
 EXPORTS = (
     "ea_version", "ea_status_string", "ea_workspace_bytes", "ea_n_kept", "ea_create", "ea_destroy",
-    "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status",
+    "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
+    "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host",
 )
 
 
@@ -65,8 +66,13 @@ def lib() -> ctypes.CDLL:
         L.ea_score.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
         L.ea_select_compact.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.ea_sync_status.argtypes = [vp, vp]
+        L.ea_host_workspace_bytes.argtypes = [sp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.ea_compress_host.argtypes = [vp, sp, vp, vp, vp, vp, i32, f64, f32, i32, i32, vp, vp, vp, vp, vp]
+        L.ea_profile_begin.argtypes = [vp]
+        L.ea_profile_end.argtypes = [vp, vp, ctypes.POINTER(f64), ctypes.POINTER(i64), ctypes.POINTER(i64)]
         for name in ("ea_workspace_bytes", "ea_create", "ea_destroy", "ea_query_stats", "ea_score",
-                     "ea_select_compact", "ea_sync_status"):
+                     "ea_select_compact", "ea_sync_status", "ea_profile_begin", "ea_profile_end",
+                     "ea_host_workspace_bytes", "ea_compress_host"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -136,6 +142,16 @@ class Context:
     def sync_status(self):
         _check(lib().ea_sync_status(self._h, _stream(self.device)), "ea_sync_status")
 
+    def profile_begin(self):
+        _check(lib().ea_profile_begin(self._h), "ea_profile_begin")
+
+    def profile_end(self):
+        """-> (device ms summed over the timed log-score launches, their count, all kernel launches)."""
+        ms, timed, total = ctypes.c_double(0), ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib().ea_profile_end(self._h, _stream(self.device), ctypes.byref(ms), ctypes.byref(timed),
+                                    ctypes.byref(total)), "ea_profile_end")
+        return ms.value, timed.value, total.value
+
 
 def ea_query_stats(ctx: Context, shape: Shape, q_win, pos_next, n_future: int, rope_base: float,
                    mu_bar=None, sigma_bar=None):
@@ -176,14 +192,14 @@ def ea_select_compact(ctx: Context, shape: Shape, scores, n_kept: int, k=None, v
     _dev_tensor(scores, torch.float32, "scores")
     U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
     if kept_idx is None:
-        kept_idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, device=scores.device)
+        kept_idx = torch.empty((U, Hkv, max(n_kept, 0)), dtype=torch.int32, device=scores.device)
     if gather:
         _dev_tensor(k, torch.bfloat16, "k")
         _dev_tensor(v, torch.bfloat16, "v")
         if k_out is None:
-            k_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.bfloat16, device=scores.device)
+            k_out = torch.empty((U, Hkv, max(n_kept, 0), d), dtype=torch.bfloat16, device=scores.device)
         if v_out is None:
-            v_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.bfloat16, device=scores.device)
+            v_out = torch.empty((U, Hkv, max(n_kept, 0), d), dtype=torch.bfloat16, device=scores.device)
     _check(lib().ea_select_compact(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k),
                                    _ptr(v), _ptr(kept_idx), _ptr(k_out), _ptr(v_out),
                                    _stream(ctx.device)), "ea_select_compact")
@@ -209,3 +225,40 @@ def compress(ctx: Context, shape: Shape, q_win, k, v, pos_next, n_future, rope_b
     scores, logits = res if want_logits else (res, None)
     kept_idx, k_out, v_out = ea_select_compact(ctx, shape, scores, n_kept, k, v)
     return Compressed(mu_bar, sigma_bar, scores, logits, kept_idx, k_out, v_out)
+
+
+def ea_host_workspace_bytes(shape: Shape, n_kept: int, units_per_chunk: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ea_host_workspace_bytes(ctypes.byref(shape), int(n_kept), int(units_per_chunk),
+                                         ctypes.byref(out)), "ea_host_workspace_bytes")
+    return int(out.value)
+
+
+def _host_tensor(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CPU tensor of {dtype}")
+    return t
+
+
+def ea_compress_host(ctx: Context, shape: Shape, q_win, k, v, pos_next, n_future, rope_base, epsilon,
+                     n_kept: int, units_per_chunk: int = 1, kept_idx=None, k_out=None, v_out=None,
+                     scores=None):
+    """Whole routine on HOST tensors (pin them for overlapped copies).  Asynchronous: call
+    ``ctx.sync_status()`` before reading the returned host tensors."""
+    _host_tensor(q_win, torch.bfloat16, "q_win")
+    _host_tensor(k, torch.bfloat16, "k")
+    _host_tensor(v, torch.bfloat16, "v")
+    _host_tensor(pos_next, torch.int64, "pos_next")
+    U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
+    pin = k.is_pinned()
+    if kept_idx is None:
+        kept_idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, pin_memory=pin)
+    if k_out is None:
+        k_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.bfloat16, pin_memory=pin)
+    if v_out is None:
+        v_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.bfloat16, pin_memory=pin)
+    _check(lib().ea_compress_host(ctx._h, ctypes.byref(shape), _ptr(q_win), _ptr(k), _ptr(v),
+                                  _ptr(pos_next), int(n_future), float(rope_base), float(epsilon),
+                                  int(n_kept), int(units_per_chunk), _ptr(kept_idx), _ptr(k_out),
+                                  _ptr(v_out), _ptr(scores), _stream(ctx.device)), "ea_compress_host")
+    return kept_idx, k_out, v_out

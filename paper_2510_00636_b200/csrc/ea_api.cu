@@ -92,8 +92,15 @@ ea_status ea_create(ea_ctx** out_ctx, int device, size_t workspace_bytes) {
     ctx->workspace_bytes = workspace_bytes;
     ctx->status_host = nullptr;
     ctx->status_dev = nullptr;
-    bool ok = true;
-    if (workspace_bytes > 0) ok = cudaMalloc(&ctx->workspace, workspace_bytes) == cudaSuccess;
+    ctx->host_ready = false;
+    ctx->profiling = false;
+    ctx->launches = 0;
+    ctx->n_events = 0;
+    ctx->n_events_created = 0;
+    ctx->ev_start = new (std::nothrow) cudaEvent_t[kMaxProfileEvents];
+    ctx->ev_stop = new (std::nothrow) cudaEvent_t[kMaxProfileEvents];
+    bool ok = ctx->ev_start && ctx->ev_stop;
+    if (ok && workspace_bytes > 0) ok = cudaMalloc(&ctx->workspace, workspace_bytes) == cudaSuccess;
     if (ok) ok = cudaHostAlloc((void**)&ctx->status_host, sizeof(int), cudaHostAllocMapped) == cudaSuccess;
     if (ok) {
         *ctx->status_host = 0;
@@ -103,6 +110,8 @@ ea_status ea_create(ea_ctx** out_ctx, int device, size_t workspace_bytes) {
         cudaGetLastError();
         if (ctx->workspace) cudaFree(ctx->workspace);
         if (ctx->status_host) cudaFreeHost(ctx->status_host);
+        delete[] ctx->ev_start;
+        delete[] ctx->ev_stop;
         delete ctx;
         cudaSetDevice(prev);
         return EA_ERR_CUDA;
@@ -119,6 +128,22 @@ ea_status ea_destroy(ea_ctx* ctx) {
     cudaSetDevice(ctx->device);
     if (ctx->workspace) cudaFree(ctx->workspace);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    if (ctx->host_ready) {
+        cudaStreamDestroy(ctx->st_h2d);
+        cudaStreamDestroy(ctx->st_d2h);
+        cudaEventDestroy(ctx->ev_entry);
+        for (int b = 0; b < 2; ++b) {
+            cudaEventDestroy(ctx->ev_h2d[b]);
+            cudaEventDestroy(ctx->ev_comp[b]);
+            cudaEventDestroy(ctx->ev_d2h[b]);
+        }
+    }
+    for (int i = 0; i < ctx->n_events_created; ++i) {
+        cudaEventDestroy(ctx->ev_start[i]);
+        cudaEventDestroy(ctx->ev_stop[i]);
+    }
+    delete[] ctx->ev_start;
+    delete[] ctx->ev_stop;
     cudaSetDevice(prev);
     delete ctx;
     return EA_OK;
@@ -223,4 +248,48 @@ ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream) {
     return s == 0 ? EA_OK : static_cast<ea_status>(s);
 }
 
+ea_status ea_profile_begin(ea_ctx* ctx) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ctx->profiling = true;
+    ctx->launches = 0;
+    ctx->n_events = 0;
+    return EA_OK;
+}
+
+ea_status ea_profile_end(ea_ctx* ctx, void* cuda_stream, double* score_kernel_ms,
+                         int64_t* timed_launches, int64_t* total_kernel_launches) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ctx->profiling = false;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return EA_ERR_CUDA;
+    double total = 0.0;
+    for (int i = 0; i < ctx->n_events; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ctx->ev_start[i], ctx->ev_stop[i]) != cudaSuccess) return EA_ERR_CUDA;
+        total += (double)ms;
+    }
+    if (score_kernel_ms) *score_kernel_ms = total;
+    if (timed_launches) *timed_launches = ctx->n_events;
+    if (total_kernel_launches) *total_kernel_launches = ctx->launches;
+    return EA_OK;
+}
+
 }  // extern "C"
+
+cudaEvent_t ea_profile_mark_start(const ea_ctx* cctx, cudaStream_t st) {
+    ea_ctx* ctx = const_cast<ea_ctx*>(cctx);
+    if (!ctx->profiling || ctx->n_events >= kMaxProfileEvents) return nullptr;
+    const int i = ctx->n_events;
+    if (i >= ctx->n_events_created) {
+        if (cudaEventCreate(&ctx->ev_start[i]) != cudaSuccess) return nullptr;
+        if (cudaEventCreate(&ctx->ev_stop[i]) != cudaSuccess) { cudaEventDestroy(ctx->ev_start[i]); return nullptr; }
+        ctx->n_events_created = i + 1;
+    }
+    cudaEventRecord(ctx->ev_start[i], st);
+    ctx->n_events = i + 1;
+    return ctx->ev_stop[i];
+}
+
+void ea_profile_mark_stop(const ea_ctx* ctx, cudaEvent_t stop, cudaStream_t st) {
+    (void)ctx;
+    if (stop) cudaEventRecord(stop, st);
+}

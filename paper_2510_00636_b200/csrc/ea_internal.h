@@ -15,7 +15,28 @@ struct ea_ctx {
     size_t workspace_bytes;
     int* status_host;    // pinned, mapped: device kernels write EA_ERR_DEVICE_TIMEOUT here
     int* status_dev;     // device alias of status_host
+    // benchmark instrumentation (ea_profile_begin / ea_profile_end)
+    bool profiling;
+    long long launches;          // kernels launched since ea_profile_begin
+    int n_events;                // event pairs recorded in this window
+    int n_events_created;        // event pairs that exist
+    cudaEvent_t* ev_start;       // [kMaxProfileEvents]
+    cudaEvent_t* ev_stop;
+    // host-buffer pipeline (ea_compress_host), created on first use
+    bool host_ready;
+    cudaStream_t st_h2d, st_d2h;
+    cudaEvent_t ev_entry, ev_h2d[2], ev_comp[2], ev_d2h[2];
 };
+
+constexpr int kMaxProfileEvents = 4096;
+
+// Count `n` kernel launches made on behalf of `ctx`.
+static inline void ea_count_launches(const ea_ctx* ctx, int n) {
+    const_cast<ea_ctx*>(ctx)->launches += n;
+}
+// Bracket the dominant kernel with events while profiling; returns the stop event or nullptr.
+cudaEvent_t ea_profile_mark_start(const ea_ctx* ctx, cudaStream_t st);
+void ea_profile_mark_stop(const ea_ctx* ctx, cudaEvent_t stop, cudaStream_t st);
 
 // Byte offsets of the workspace regions.  Regions of different calls overlap
 // on purpose except where one call's output feeds the next.

@@ -124,7 +124,6 @@ finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
                              const __nv_bfloat16* v, float epsilon, float* lse, float* scores,
                              cudaStream_t st) {
-    (void)ctx;
     const int G = s.n_q_heads / s.n_kv_heads;
     if (s.group_mode == EA_GROUP_MEAN_LOGIT)
         lse_kernel<<<s.n_units * s.n_kv_heads, kLseThreads, 0, st>>>(logits, s.n_keys, G, lse);
@@ -151,5 +150,6 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
         default:
             return EA_ERR_UNSUPPORTED;
     }
+    ea_count_launches(ctx, 2);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

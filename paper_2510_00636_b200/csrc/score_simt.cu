@@ -75,7 +75,8 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const float* __restrict_
 ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                 const float* mu_bar, const float* sigma_bar, float* logits,
                                 cudaStream_t st) {
-    (void)ctx;
+    ea_count_launches(ctx, 1);
+    cudaEvent_t stop = ea_profile_mark_start(ctx, st);
     dim3 grid((unsigned)((s.n_keys + kKeysPerCta - 1) / kKeysPerCta),
               (unsigned)(s.n_units * s.n_q_heads));
     switch (s.head_dim) {
@@ -96,5 +97,6 @@ ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv
         default:
             return EA_ERR_UNSUPPORTED;
     }
+    ea_profile_mark_stop(ctx, stop, st);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

@@ -149,8 +149,8 @@ __global__ void gather_kernel(const int32_t* __restrict__ kept_idx, long long n_
 
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
                            int32_t* kept_idx, cudaStream_t st) {
-    (void)ctx;
     if (n_kept <= 0) return EA_OK;
+    ea_count_launches(ctx, 1);
     select_kernel<<<s.n_units * s.n_kv_heads, kSelThreads, 0, st>>>(scores, s.n_keys, n_kept, kept_idx);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }
@@ -159,6 +159,7 @@ ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, con
                            const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* k_out,
                            __nv_bfloat16* v_out, cudaStream_t st) {
     if (n_kept <= 0) return EA_OK;
+    ea_count_launches(ctx, 1);
     const long long rows = (long long)s.n_units * s.n_kv_heads * n_kept;
     const int threads = 256;
     const long long pieces = rows * (s.head_dim / 8);

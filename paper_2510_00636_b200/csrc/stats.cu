@@ -124,7 +124,6 @@ stats_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restrict__ 
 ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
                           const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
                           float* mu_bar, float* sigma_bar, cudaStream_t st) {
-    (void)ctx;
     const int d = s.head_dim, half = d / 2;
     const int n_coef = s.n_units * half;
     rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, st>>>(pos_next, s.n_units, half, d, n_future,
@@ -148,5 +147,6 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
         default:
             return EA_ERR_UNSUPPORTED;
     }
+    ea_count_launches(ctx, 2);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

@@ -32,10 +32,14 @@ def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
 def logit_error_bound(k_bits, mu_bar, sigma_bar, sigma_operand_bits: int):
     """Per (unit, query head, key) bound on the CUDA path's log-score error.
 
-    fp32 accumulation contributes 2^-20 of the sum of the magnitudes of the terms.  When the
-    covariance operand is rounded to ``sigma_operand_bits`` significant bits (8 for bf16, 24
-    for fp32) each product k_a k_b Sigma_ab carries an independent relative error of at most
-    2^-bits; six standard deviations of their sum bound the quadratic term's error.
+    Three sources, added:
+      * fp32 accumulation of the score: 2^-20 of the sum of the magnitudes of its terms;
+      * the covariance operand rounded to ``sigma_operand_bits`` significant bits (8 for bf16,
+        24 for fp32): each product k_a k_b Sigma_ab carries an independent relative error of at
+        most 2^-bits, and six standard deviations of their sum bound the total;
+      * the fp32 statistics themselves: each Sigma_ab is off by about 2^-20 sqrt(Sigma_aa
+        Sigma_bb) (W fp32 additions), again six standard deviations of the summed effect,
+        6 * 2^-20 * sum_a k_a^2 Sigma_aa / (2d).
     """
     k = bf16_to_f64(k_bits)                                  # [U, Hkv, n, d]
     U, Hkv, n, d = k.shape
@@ -50,7 +54,9 @@ def logit_error_bound(k_bits, mu_bar, sigma_bar, sigma_operand_bits: int):
             absl = ak @ np.abs(mu_bar[u, h]) / np.sqrt(d)
             k2 = kk ** 2
             rnd = np.sqrt(((k2 @ sigma_bar[u, h] ** 2) * k2).sum(-1)) / (2 * d)
-            out[u, h] = 2.0 ** -20 * (absq + absl) + 6.0 * 2.0 ** (-sigma_operand_bits) / np.sqrt(3) * rnd
+            stat = 6.0 * 2.0 ** -20 * (k2 @ np.diag(sigma_bar[u, h])) / (2 * d)
+            out[u, h] = (2.0 ** -20 * (absq + absl) + 6.0 * 2.0 ** (-sigma_operand_bits) / np.sqrt(3) * rnd
+                         + stat)
     return out
 
 

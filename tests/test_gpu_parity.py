@@ -229,3 +229,35 @@ def test_empty_inputs_are_noops(ea):
     assert ea.lib().ea_score(ctx._h, __import__("ctypes").byref(shape), None, None, None, None, 0.02,
                              None, None, None) == 0
     ctx.sync_status()
+
+
+@pytest.mark.parametrize("chunk", [1, 2, 5])
+def test_host_buffer_entry_point_matches_device_calls(ea, chunk):
+    """ea_compress_host (host pointers, chunked, copies overlapped) returns the device path's bits."""
+    cfg = inputs.CONFIGS[0]
+    U = 3
+    qs, ks, vs = [], [], []
+    for layer in range(U):
+        q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device="cuda")
+        qs.append(q), ks.append(k), vs.append(v)
+    q, k, v = torch.cat(qs), torch.cat(ks), torch.cat(vs)
+    pos = torch.tensor([512, 600, 5], dtype=torch.int64)
+    shape = _shape(ea, cfg, n_units=U)
+    ctx = ea.Context.for_shape(shape)
+    want = ea.compress(ctx, shape, q, k, v, pos.cuda(), cfg.n_future, cfg.rope_base, cfg.eps, cfg.n_kept)
+    ctx.sync_status()
+    hctx = ea.Context(0, ea.ea_host_workspace_bytes(shape, cfg.n_kept, chunk))
+    hq, hk, hv = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+    hs = torch.empty((U, cfg.n_kv_heads, cfg.n_keys), dtype=torch.float32).pin_memory()
+    for _ in range(2):      # twice: staging buffers and events are reused
+        idx, ko, vo = ea.ea_compress_host(hctx, shape, hq, hk, hv, pos, cfg.n_future, cfg.rope_base, cfg.eps,
+                                          cfg.n_kept, chunk, scores=hs)
+        hctx.sync_status()
+        assert torch.equal(idx, want.kept_idx.cpu())
+        assert torch.equal(ko.view(torch.int16), want.k_out.cpu().view(torch.int16))
+        assert torch.equal(vo.view(torch.int16), want.v_out.cpu().view(torch.int16))
+        assert torch.equal(hs, want.scores.cpu())
+    small = ea.Context(0, 1024)
+    with pytest.raises(ea.EAError) as e:
+        ea.ea_compress_host(small, shape, hq, hk, hv, pos, cfg.n_future, cfg.rope_base, cfg.eps, cfg.n_kept, chunk)
+    assert e.value.status == 3

@@ -35,6 +35,9 @@ ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     p.logits = off;     off = ea_align_up(off + U * Hq * n * sizeof(float), 256);
     p.lse = off;        off = ea_align_up(off + U * Hq * sizeof(float), 256);
     p.sel_state = off;  off = ea_align_up(off + U * Hkv * 4 * sizeof(uint32_t), 256);
+    const bool mma = ea_mma_path_supported(s);
+    p.image = off;      off = ea_align_up(off + (mma ? ea_mma_image_bytes(s) : 0), 1024);
+    p.vec = off;        off = ea_align_up(off + (mma ? ea_mma_vec_bytes(s) : 0), 256);
     p.total = off;
     return p;
 }
@@ -194,8 +197,12 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     float* logits = logits_opt ? logits_opt : reinterpret_cast<float*>(ws + plan.logits);
     float* lse = reinterpret_cast<float*>(ws + plan.lse);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    st = ea_launch_logits_simt(ctx, *shape, static_cast<const __nv_bfloat16*>(k), mu_bar, sigma_bar,
-                               logits, stream);
+    if (ea_mma_path_supported(*shape))
+        st = ea_launch_logits_mma(ctx, *shape, static_cast<const __nv_bfloat16*>(k), mu_bar, sigma_bar,
+                                  ws + plan.image, reinterpret_cast<float*>(ws + plan.vec), logits, stream);
+    else
+        st = ea_launch_logits_simt(ctx, *shape, static_cast<const __nv_bfloat16*>(k), mu_bar, sigma_bar,
+                                   logits, stream);
     if (st == EA_OK)
         st = ea_launch_finalize(ctx, *shape, logits, static_cast<const __nv_bfloat16*>(v), epsilon, lse,
                                 scores, stream);

@@ -45,6 +45,8 @@ struct ea_ws_plan {
     size_t logits;       // fp32 [U, Hq, n]              (ea_score, when logits_opt == NULL)
     size_t lse;          // fp32 [U, Hq]                 (ea_score)
     size_t sel_state;    // uint32 [U*Hkv, 4]            (ea_select_compact)
+    size_t image;        // bf16 covariance images of the tensor-core log-score kernel (ea_score)
+    size_t vec;          // fp32 [U*Hq, 2, d] epilogue vectors of that kernel            (ea_score)
     size_t total;
 };
 
@@ -66,6 +68,14 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
 ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                 const float* mu_bar, const float* sigma_bar, float* logits,
                                 cudaStream_t st);
+
+// Tensor-core log-score kernel (tcgen05): available for some shapes only.
+bool ea_mma_path_supported(const ea_shape& s);
+size_t ea_mma_image_bytes(const ea_shape& s);
+size_t ea_mma_vec_bytes(const ea_shape& s);
+ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
+                               const float* mu_bar, const float* sigma_bar, void* image, float* vec,
+                               float* logits, cudaStream_t st);
 
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
                              const __nv_bfloat16* v, float epsilon, float* lse, float* scores,

@@ -23,7 +23,7 @@ def _shape(ea, cfg, n_units=None, n_keys=None, **kw):
                          cfg.head_dim, cfg.n_keys if n_keys is None else n_keys, cfg.window, **kw)
 
 
-def _run_whole_path(ea, oracle, cfg, group_mode=0, sigma_bits=24, layer=0):
+def _run_whole_path(ea, oracle, cfg, group_mode=0, sigma_bits=16, layer=0):
     q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device="cuda")
     shape = _shape(ea, cfg, n_units=cfg.batch, group_mode=group_mode)
     ctx = ea.Context.for_shape(shape)

@@ -129,6 +129,43 @@ ea_status ea_query_stats(ea_ctx* ctx, const ea_shape* shape, const void* q_win,
                          float* mu_bar, float* sigma_bar, void* cuda_stream);
 
 /*
+ * ea_query_stats for callers that cannot allocate device memory (the paper has
+ * no counterpart: this is a packaging variant, the arithmetic and the outputs
+ * are those of ea_query_stats).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a
+ * serving loop whose memory is fully handed to a caching allocator, in a
+ * plugin whose host forbids driver allocations after start-up, or on a
+ * latency path where an allocation's implicit device synchronisation is not
+ * acceptable.  ea_create allocates (the workspace and a pinned status word),
+ * so this call takes no context: it uses the CURRENT device and only launches
+ * kernels on cuda_stream.
+ *
+ * The one piece of scratch the statistics need, the averaged-rotation
+ * coefficients (one fp32 cos/sin pair per unit and channel pair), lives in a
+ * fixed array inside the library: EA_STATIC_MAX_ROPE_PAIRS pairs, 128 KiB,
+ * held by every GPU that loads the library until the process exits.  A shape
+ * with n_units * head_dim / 2 > EA_STATIC_MAX_ROPE_PAIRS is refused with
+ * EA_ERR_WORKSPACE before anything is launched (split the units over several
+ * calls on the same stream).
+ *
+ * The first call on each device looks up the array's device address (no
+ * allocation, but a runtime query): make that first call before starting any
+ * stream capture.  All calls on a device share the array.  Each call rewrites
+ * every coefficient it later reads, so nothing left by an earlier call can
+ * leak into the result and nothing needs clearing; but two calls whose kernels
+ * overlap on the GPU (different streams, no ordering between them) race on
+ * it.  Order them on one stream or with events.
+ *
+ * Arguments as for ea_query_stats (pos_next is a DEVICE pointer); n_keys,
+ * n_kv_heads and group_mode of the shape are ignored.
+ */
+#define EA_STATIC_MAX_ROPE_PAIRS 16384
+ea_status ea_query_stats_static(const ea_shape* shape, const void* q_win, const int64_t* pos_next,
+                                int32_t n_future, double rope_base, float* mu_bar, float* sigma_bar,
+                                void* cuda_stream);
+
+/*
  * Contribution score of every cached pair (Eq. 7, 8, 9 with ||v|| in place of
  * ||W_o v||, as the paper's implementation note states):
  *   s_{h,i}   = mu_bar_h . k_i / sqrt(d) + k_i^T sigma_bar_h k_i / (2d)

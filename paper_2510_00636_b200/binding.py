@@ -23,8 +23,9 @@ COV_POPULATION, COV_SAMPLE = 0, 1
 EXPORTS = (
     "ea_version", "ea_status_string", "ea_workspace_bytes", "ea_n_kept", "ea_create", "ea_destroy",
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
-    "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host",
+    "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
 )
+STATIC_MAX_ROPE_PAIRS = 16384
 
 
 class EAError(RuntimeError):
@@ -63,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.ea_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int, ctypes.c_size_t]
         L.ea_destroy.argtypes = [vp]
         L.ea_query_stats.argtypes = [vp, sp, vp, vp, i32, f64, vp, vp, vp]
+        L.ea_query_stats_static.argtypes = [sp, vp, vp, i32, f64, vp, vp, vp]
+        L.ea_query_stats_static.restype = ctypes.c_int
         L.ea_score.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
         L.ea_select_compact.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.ea_sync_status.argtypes = [vp, vp]
@@ -166,6 +169,25 @@ def ea_query_stats(ctx: Context, shape: Shape, q_win, pos_next, n_future: int, r
     _check(lib().ea_query_stats(ctx._h, ctypes.byref(shape), _ptr(q_win), _ptr(pos_next), int(n_future),
                                 float(rope_base), _ptr(mu_bar), _ptr(sigma_bar), _stream(ctx.device)),
            "ea_query_stats")
+    return mu_bar, sigma_bar
+
+
+def ea_query_stats_static(shape: Shape, q_win, pos_next, n_future: int, rope_base: float, mu_bar, sigma_bar):
+    """``ea_query_stats`` without a context: for callers that must not allocate device memory.
+
+    The library call itself allocates nothing, so the outputs are NOT created here: the caller
+    hands in ``mu_bar`` [U,Hq,d] and ``sigma_bar`` [U,Hq,d,d] (fp32, on the device of ``q_win``).
+    Works on the tensors' device, which must be the current one; at most
+    ``STATIC_MAX_ROPE_PAIRS`` (unit, channel pair) combinations per call.
+    """
+    _dev_tensor(q_win, torch.bfloat16, "q_win")
+    _dev_tensor(pos_next, torch.int64, "pos_next")
+    _dev_tensor(mu_bar, torch.float32, "mu_bar")
+    _dev_tensor(sigma_bar, torch.float32, "sigma_bar")
+    with torch.cuda.device(q_win.device):
+        _check(lib().ea_query_stats_static(ctypes.byref(shape), _ptr(q_win), _ptr(pos_next), int(n_future),
+                                           float(rope_base), _ptr(mu_bar), _ptr(sigma_bar),
+                                           _stream(q_win.device)), "ea_query_stats_static")
     return mu_bar, sigma_bar
 
 

@@ -150,3 +150,86 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
     ea_count_launches(ctx, 2);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------------
+// ea_query_stats_static: the same two kernels, with the averaged-rotation coefficients kept in a
+// fixed device array of this library instead of a context workspace.  Nothing is allocated here
+// or on first use; the array is part of the loaded module on every GPU that loads the library.
+#include <mutex>
+
+namespace {
+
+// fp32 (cos, sin) pairs: n_units * head_dim / 2 of them per call.
+static __device__ __align__(256) float g_static_rope_coef[2 * EA_STATIC_MAX_ROPE_PAIRS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float* g_static_coef_addr[kMaxDevices];   // device address of the array, per device, once resolved
+
+// Device address of g_static_rope_coef on the CURRENT device.  The symbol's name is only a
+// host-side handle; kernels must be given the address the runtime reports for it.
+ea_status static_coef_address(float** out) {
+    int dev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return EA_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_coef_addr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_rope_coef) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return EA_ERR_CUDA;
+        }
+        g_static_coef_addr[dev] = static_cast<float*>(ptr);
+    }
+    *out = g_static_coef_addr[dev];
+    return EA_OK;
+}
+
+}  // namespace
+
+extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win, const int64_t* pos_next,
+                                           int32_t n_future, double rope_base, float* mu_bar,
+                                           float* sigma_bar, void* cuda_stream) {
+    if (!s) return EA_ERR_INVALID_ARG;
+    if (s->n_units < 0 || s->n_q_heads < 1 || s->window < 1) return EA_ERR_INVALID_ARG;
+    if (s->rope_layout != EA_ROPE_HALF_SPLIT && s->rope_layout != EA_ROPE_INTERLEAVED) return EA_ERR_INVALID_ARG;
+    if (s->cov_norm != EA_COV_POPULATION && s->cov_norm != EA_COV_SAMPLE) return EA_ERR_INVALID_ARG;
+    if (s->cov_norm == EA_COV_SAMPLE && s->window < 2) return EA_ERR_INVALID_ARG;
+    if (s->head_dim != 64 && s->head_dim != 128 && s->head_dim != 256) return EA_ERR_UNSUPPORTED;
+    if (n_future < 1 || !(rope_base > 0.0)) return EA_ERR_INVALID_ARG;
+    const int d = s->head_dim, half = d / 2;
+    // the fixed array bounds the problem size: refuse anything that would not fit
+    if ((long long)s->n_units * half > (long long)EA_STATIC_MAX_ROPE_PAIRS) return EA_ERR_WORKSPACE;
+    if ((long long)s->n_units * s->n_q_heads > 0x7fffffffLL) return EA_ERR_UNSUPPORTED;
+    if (s->n_units == 0) return EA_OK;
+    if (!q_win || !pos_next || !mu_bar || !sigma_bar) return EA_ERR_INVALID_ARG;
+    if (((uintptr_t)q_win | (uintptr_t)mu_bar | (uintptr_t)sigma_bar) & 15u) return EA_ERR_INVALID_ARG;
+
+    float* coef = nullptr;
+    ea_status st = static_coef_address(&coef);
+    if (st != EA_OK) return st;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(q_win);
+    const int n_coef = s->n_units * half;
+    // every coefficient this call reads is written first, so stale contents of earlier calls are harmless
+    rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, stream>>>(pos_next, s->n_units, half, d, n_future,
+                                                               rope_base, coef);
+    const float inv_norm = 1.0f / (float)(s->cov_norm == EA_COV_SAMPLE ? s->window - 1 : s->window);
+    dim3 grid((unsigned)(s->n_units * s->n_q_heads), (unsigned)(d / kRowBlock));
+    switch (d) {
+        case 64:
+            stats_kernel<64><<<grid, kStatsThreads, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+                                                                 s->rope_layout, inv_norm, mu_bar, sigma_bar);
+            break;
+        case 128:
+            stats_kernel<128><<<grid, kStatsThreads, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+                                                                  s->rope_layout, inv_norm, mu_bar, sigma_bar);
+            break;
+        default:
+            stats_kernel<256><<<grid, kStatsThreads, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+                                                                  s->rope_layout, inv_norm, mu_bar, sigma_bar);
+            break;
+    }
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}

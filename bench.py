@@ -248,11 +248,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3])
     ap.add_argument("--units-per-call", type=int, default=0, help="layers per library call (0 = all)")
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: only the first N layers of the stack")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = inputs.CONFIGS[args.config]
+    if args.layers:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, n_layers=args.layers, name=f"{cfg.name}-first{args.layers}layers")
 
     if args.impl == "reference":
         run_reference(args, cfg)

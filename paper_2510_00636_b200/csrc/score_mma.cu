@@ -4,19 +4,23 @@
 // The dense part is the product K . B^T of a tile of 128 cached keys with a bf16 image B of
 // the covariance; the row-wise quadratic form is finished in the epilogue:
 //     D[i, c]  = sum_a K[i, a] B[c, a]                      (tcgen05.mma, fp32 in tensor memory)
-//     s_{h,i}  = sum_c k_{i,c} ( D[i, c]/(2d) + mu_bar_c/sqrt(d) + Sigma_bar_cc k_{i,c}/(2d) )
-// B carries the off-diagonal of Sigma_bar at twice bf16 precision for the price of one bf16
+//     s_{h,i}  = sum_c k_{i,c} ( D[i, c] + mu_bar_c/sqrt(d) + Sigma_bar_cc k_{i,c}/(2d) )
+// B carries the off-diagonal of Sigma_bar/(2d) at twice bf16 precision for the price of one bf16
 // matrix: the quadratic form only sees B[c,a] + B[a,c], so for a < c the entry B[c,a] holds
-// bf16(2 Sigma_ac) and the mirrored entry B[a,c] holds the bf16 rounding of what that left over.
+// bf16(Sigma_ac/d) and the mirrored entry B[a,c] holds the bf16 rounding of what that left over.
 // The diagonal stays out of B and enters in fp32 in the epilogue together with the linear term.
 //
-// One CTA keeps the image of `hpc` query heads of one KV head resident in shared memory
+// A CTA keeps the image of `hpc` query heads of one KV head resident in shared memory
 // (hpc * d = 256 accumulator columns at most) and streams key tiles through a TMA ring:
-//   warp 0    TMA producer (one lane): covariance image (bulk copy) and key tiles (tiled, 128B swizzle)
-//   warp 1    MMA issuer (one lane); owns the tensor-memory allocation
-//   warps 2-5 epilogue: thread <-> accumulator lane <-> key; reads its key row from the staged tile
-// Tensor memory holds two accumulator stages so the epilogue of one tile overlaps the MMAs of
-// the next.  Every wait is bounded; a wait that gives up raises the context's status word.
+//   warp 0     TMA producer (one lane): covariance image (bulk copy) and key tiles (tiled, 128B swizzle)
+//   warp 1     MMA issuer (one lane); owns the tensor-memory allocation
+//   warps 2-9  epilogue, two warps per tensor-memory lane quarter: thread <-> accumulator lane <-> key;
+//              each reads its key row from the staged tile and half of the accumulator columns
+// Tensor memory holds two accumulator stages so the epilogue of one tile overlaps the MMAs of the
+// next.  With PAIR, two CTAs of a cluster work as one (cta_group::2): each stages its own 128 keys
+// and half of the image rows, the leader issues M = 256 MMAs for both, and each CTA runs the
+// epilogue of its own keys; this is what lets head_dim 256 fit in shared memory.
+// Every wait is bounded; a wait that gives up raises the context's status word.
 #include "ea_internal.h"
 #include "ptx_sm100.cuh"
 
@@ -24,36 +28,47 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kTileKeys = 128;
-constexpr int kEpiWarps = 4;
+constexpr int kTileKeys = 128;                     // keys per CTA per step
+constexpr int kEpiWarps = 8;
 constexpr int kMmaThreads = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
-constexpr int kAccCols = 256;          // columns of one accumulator stage
+constexpr int kAccCols = 256;                      // columns of one accumulator stage
+constexpr int kChunkA = kTileKeys * 128;           // bytes of one 64-channel chunk of a key tile
 
-template <int D>
+template <int D, bool PAIR>
 struct Geo {
-    static constexpr int HPC = 256 / D;                  // query heads per CTA pass (1, 2 or 4)
+    static constexpr int HPC = 256 / D;                  // query heads per pass (1, 2 or 4)
     static constexpr int KCH = D / 64;                   // 64-channel (128-byte) chunks per row
-    static constexpr int CHUNK_A = kTileKeys * 128;      // bytes of one chunk of a key tile
-    static constexpr int STAGE = KCH * CHUNK_A;          // bytes of one key tile
-    static constexpr int IMG_ROWS = HPC * D;             // rows (accumulator columns) of the image
-    static constexpr int CHUNK_B = IMG_ROWS * 128;       // bytes of one chunk of the image
-    static constexpr int IMG = KCH * CHUNK_B;            // bytes of the image of one head subset
-    static constexpr int STAGES = 4;
-    static constexpr int VEC = HPC * D * 2 * sizeof(float);   // mu' and diagonal vectors
-    static constexpr int SMEM = IMG + STAGES * STAGE + VEC + 256 + 1024;
+    static constexpr int STAGE = KCH * kChunkA;          // bytes of one key tile
+    static constexpr int IMG_ROWS = HPC * D;             // rows of a whole image (accumulator columns)
+    static constexpr int CHUNK_B_FULL = IMG_ROWS * 128;  // bytes of one chunk of a whole image (global)
+    static constexpr int IMG_FULL = KCH * CHUNK_B_FULL;  // bytes of a whole image (global)
+    static constexpr int ROWS_CTA = PAIR ? IMG_ROWS / 2 : IMG_ROWS;   // image rows one CTA keeps
+    static constexpr int CHUNK_B = ROWS_CTA * 128;
+    static constexpr int IMG_CTA = KCH * CHUNK_B;
+    static constexpr int STAGES = D == 256 ? 2 : 4;
+    static constexpr int NSLOT = STAGES * KCH;           // ring of 16 KiB chunk slots
+    static constexpr int VEC = HPC * D * 2 * (int)sizeof(float);   // mu' and diagonal vectors
+    static constexpr int PART = 2 * kTileKeys * (int)sizeof(float);
+    static constexpr int NBAR = 2 * NSLOT + 6;
+    static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
+    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + VEC + PART + CTRL + 1024;
+    // warps that must release a chunk slot before it is refilled
+    static constexpr int SLOT_RELEASERS = D == 256 ? kEpiWarps / 2 : kEpiWarps;
+    static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
+    static_assert(SMEM <= 232448, "shared memory budget");
 };
 
 struct MmaParams {
     const float* vec;        // fp32 [U*Hq][2][D]: mu_bar/sqrt(d), diag(Sigma_bar)/(2d)
-    const uint8_t* image;    // bf16 images, Geo::IMG bytes per (unit, kv head, head subset)
+    const uint8_t* image;    // bf16 images, IMG_FULL bytes per (unit, kv head, head subset)
     float* logits;           // fp32 [U, Hq, n]
     int* status;             // device-visible status word
     int Hq, Hkv, n;
     int n_subsets;           // head subsets per KV head
-    int n_tiles;             // key tiles per head
-    int chunk_tiles;         // tiles per work item
-    int n_chunks;            // work items per (head subset)
+    int n_tiles;             // steps per head (128 keys per step, 256 with PAIR)
+    int chunk_tiles;         // steps per work item
+    int n_chunks;            // work items per head subset
     long long n_items;
 };
 
@@ -63,7 +78,7 @@ template <int D>
 __global__ void __launch_bounds__(256)
 sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ sigma_bar, int Hq, int Hkv,
                    uint8_t* __restrict__ image, float* __restrict__ vec) {
-    using G = Geo<D>;
+    using G = Geo<D, true>;
     const int uh = blockIdx.x;
     const int u = uh / Hq, h = uh % Hq;
     const int Gq = Hq / Hkv;
@@ -71,7 +86,8 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
     const int n_subsets = (Gq + G::HPC - 1) / G::HPC;
     const int hs = hg / G::HPC, j = hg % G::HPC;
     const float* S = sigma_bar + (size_t)uh * D * D;
-    uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG;
+    uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG_FULL;
+    const float inv_d = 1.0f / (float)D;       // a power of two: the scaling is exact
 
     // one 16-byte unit (8 consecutive a) of one row c per thread step
     for (int e = threadIdx.x; e < D * (D / 8); e += blockDim.x) {
@@ -85,9 +101,11 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
                 const int a = a0 + 2 * p + q;
                 float val = 0.f;
                 if (a != c) {
-                    const float two_s = S[(size_t)c * D + a] + S[(size_t)a * D + c];
-                    const float hi = __bfloat162float(__float2bfloat16_rn(two_s));
-                    val = a < c ? hi : two_s - hi;
+                    // Sigma_ac / d (the two mirrored entries together carry 2 Sigma_ac / (2d)),
+                    // split into a bf16 and the bf16 rounding of its remainder
+                    const float x = (S[(size_t)c * D + a] + S[(size_t)a * D + c]) * (0.5f * inv_d);
+                    const float hi = __bfloat162float(__float2bfloat16_rn(x));
+                    val = a < c ? hi : x - hi;
                 }
                 half[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(val));
             }
@@ -95,7 +113,7 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
         }
         const int row = j * D + c;
         const int kc = a0 / 64, unit = (a0 % 64) / 8;
-        uint4* dst = reinterpret_cast<uint4*>(img + (size_t)kc * G::CHUNK_B + (size_t)row * 128 +
+        uint4* dst = reinterpret_cast<uint4*>(img + (size_t)kc * G::CHUNK_B_FULL + (size_t)row * 128 +
                                               ((unit ^ (row & 7)) << 4));
         *dst = make_uint4(w[0], w[1], w[2], w[3]);
     }
@@ -124,107 +142,146 @@ __device__ __forceinline__ Item decode_item(long long item, const MmaParams& p, 
     return it;
 }
 
-template <int D>
+// AND of `ok` over all epilogue threads (named barrier 1): keeps their control flow identical.
+__device__ __forceinline__ bool epi_all(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)ok), "n"(32 * kEpiWarps)
+        : "memory");
+    return r != 0;
+}
+
+template <int D, bool PAIR>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) {
-    using G = Geo<D>;
+    using G = Geo<D, PAIR>;
     extern __shared__ uint8_t smem_raw[];
     // carve shared memory: 1024-byte aligned operand tiles first
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_img = base;
-    const uint32_t s_k = s_img + G::IMG;
-    const uint32_t s_vec = s_k + G::STAGES * G::STAGE;
-    const float* vec_gen = reinterpret_cast<const float*>(gen_base + G::IMG + G::STAGES * G::STAGE);
-    const uint32_t s_bar = s_vec + G::VEC;
-    uint8_t* bar_gen = gen_base + G::IMG + G::STAGES * G::STAGE + G::VEC;
-    // barriers: full_k[S], empty_k[S], tmem_full[2], tmem_empty[2], img_full
-    auto full_k = [&](int s) { return s_bar + 8u * s; };
-    auto empty_k = [&](int s) { return s_bar + 8u * (G::STAGES + s); };
-    auto tmem_full = [&](int a) { return s_bar + 8u * (2 * G::STAGES + a); };
-    auto tmem_empty = [&](int a) { return s_bar + 8u * (2 * G::STAGES + 2 + a); };
-    const uint32_t img_full = s_bar + 8u * (2 * G::STAGES + 4);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * G::STAGES + 5));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * G::STAGES + 5) + 4);
+    const uint32_t s_k = s_img + G::IMG_CTA;
+    constexpr int kOffVec = G::IMG_CTA + G::STAGES * G::STAGE;
+    const uint32_t s_vec = base + kOffVec;
+    const float* vec_gen = reinterpret_cast<const float*>(gen_base + kOffVec);
+    float* part_gen = reinterpret_cast<float*>(gen_base + kOffVec + G::VEC);
+    const uint32_t s_bar = base + kOffVec + G::VEC + G::PART;
+    uint8_t* bar_gen = gen_base + kOffVec + G::VEC + G::PART;
+    auto full_k = [&](int slot) { return s_bar + 8u * slot; };
+    auto empty_k = [&](int slot) { return s_bar + 8u * (G::NSLOT + slot); };
+    auto tmem_full = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + a); };
+    auto tmem_empty = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + 2 + a); };
+    const uint32_t img_full = s_bar + 8u * (2 * G::NSLOT + 4);
+    const uint32_t img_peer = s_bar + 8u * (2 * G::NSLOT + 5);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * G::NBAR);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * G::NBAR + 4);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;     // 0 = leader
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < G::STAGES; ++s) {
+        for (int s = 0; s < G::NSLOT; ++s) {
             mbar_init(full_k(s), 1);
-            mbar_init(empty_k(s), kEpiWarps);
+            mbar_init(empty_k(s), G::SLOT_RELEASERS);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
-            mbar_init(tmem_empty(a), kEpiWarps);
+            mbar_init(tmem_empty(a), PAIR ? 2 * kEpiWarps : kEpiWarps);
         }
         mbar_init(img_full, 1);
+        mbar_init(img_peer, 1);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&k_map);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-        tmem_relinquish();
+        if (PAIR) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+            tmem_relinquish();
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (PAIR) cluster_sync();          // the peer's barriers exist before anything signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const long long first = blockIdx.x, stride = gridDim.x;
+    const long long first = PAIR ? blockIdx.x / 2 : blockIdx.x;
+    const long long stride = PAIR ? gridDim.x / 2 : gridDim.x;
+    constexpr int kKeysPerStep = PAIR ? 2 * kTileKeys : kTileKeys;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            int fills[G::STAGES];
-#pragma unroll
-            for (int s = 0; s < G::STAGES; ++s) fills[s] = 0;
-            long long tile_no = 0;
-            long long cur_img = -1;
+            long long tile_no = 0, cur_img = -1;
             bool ok = true;
             for (long long item = first; ok && item < p.n_items; item += stride) {
                 const Item it = decode_item(item, p, G::HPC);
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
                     // every tile that used the resident image must have left the epilogue
-#pragma unroll
-                    for (int s = 0; s < G::STAGES; ++s)
-                        if (ok && fills[s] > 0) ok = mbar_wait(empty_k(s), (fills[s] - 1) & 1, abort_flag);
+                    for (int back = 1; ok && back <= G::STAGES && back <= tile_no; ++back) {
+                        const long long tn = tile_no - back;
+                        const int stage = (int)(tn % G::STAGES);
+                        const uint32_t fill = (uint32_t)(tn / G::STAGES);
+                        for (int kc = 0; ok && kc < G::KCH; ++kc)
+                            ok = mbar_wait(empty_k(stage * G::KCH + kc), fill & 1, abort_flag);
+                    }
                     if (!ok) break;
-                    const int rows = it.hpc * D;
+                    const int rows_total = it.hpc * D;
+                    const int rows = PAIR ? rows_total / 2 : rows_total;
                     const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
                     const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
                     const uint32_t vec_bytes = (uint32_t)(it.hpc * 2 * D * sizeof(float));
                     mbar_arrive_expect_tx(img_full, (uint32_t)(G::KCH * rows * 128) + vec_bytes);
-                    const uint8_t* src = p.image + (size_t)img_id * G::IMG;
+                    const uint8_t* src = p.image + (size_t)img_id * G::IMG_FULL + (size_t)rank * rows * 128;
                     for (int kc = 0; kc < G::KCH; ++kc)
-                        bulk_load(s_img + kc * G::CHUNK_B, src + (size_t)kc * G::CHUNK_B, rows * 128, img_full);
+                        bulk_load(s_img + kc * G::CHUNK_B, src + (size_t)kc * G::CHUNK_B_FULL, rows * 128, img_full);
                     bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * 2 * D, vec_bytes, img_full);
                     cur_img = img_id;
                 }
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                    const int s = (int)(tile_no % G::STAGES);
-                    ok = mbar_wait(empty_k(s), (fills[s] & 1) ^ 1, abort_flag);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(full_k(s), G::STAGE);
-                    for (int kc = 0; kc < G::KCH; ++kc)
-                        tma_load_3d(s_k + s * G::STAGE + kc * G::CHUNK_A, &k_map, full_k(s), kc * 64,
-                                    t * kTileKeys, it.ug);
-                    ++fills[s];
+                    const int stage = (int)(tile_no % G::STAGES);
+                    const uint32_t fill = (uint32_t)(tile_no / G::STAGES);
+                    const int key0 = t * kKeysPerStep + (int)rank * kTileKeys;
+                    for (int kc = 0; ok && kc < G::KCH; ++kc) {
+                        const int slot = stage * G::KCH + kc;
+                        ok = mbar_wait(empty_k(slot), (fill & 1) ^ 1, abort_flag);
+                        if (!ok) break;
+                        if (PAIR) {
+                            if (leader) mbar_arrive_expect_tx(full_k(slot), 2 * kChunkA);
+                            tma_load_3d_pair(s_k + slot * kChunkA, &k_map, mapa(full_k(slot), 0), kc * 64, key0,
+                                             it.ug);
+                        } else {
+                            mbar_arrive_expect_tx(full_k(slot), kChunkA);
+                            tma_load_3d(s_k + slot * kChunkA, &k_map, full_k(slot), kc * 64, key0, it.ug);
+                        }
+                    }
                 }
             }
-            if (!ok) {
+            if (!ok && !PAIR) {
                 // let the copies already in flight land before the CTA's shared memory goes away
-#pragma unroll
-                for (int s = 0; s < G::STAGES; ++s)
-                    if (fills[s] > 0) mbar_wait(full_k(s), (fills[s] - 1) & 1, abort_flag);
+                for (int back = 1; back <= G::STAGES && back <= tile_no; ++back) {
+                    const long long tn = tile_no - back;
+                    for (int kc = 0; kc < G::KCH; ++kc)
+                        mbar_wait(full_k((int)(tn % G::STAGES) * G::KCH + kc), (uint32_t)(tn / G::STAGES) & 1,
+                                  abort_flag);
+                }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && leader) {
+            // -------------------------------------------------------------- MMA issuer
             long long tile_no = 0, cur_img = -1;
             int img_loads = 0;
             bool ok = true;
@@ -233,38 +290,70 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
                     ok = mbar_wait(img_full, img_loads & 1, abort_flag);
+                    if (ok && PAIR) ok = mbar_wait<true>(img_peer, img_loads & 1, abort_flag);
                     if (!ok) break;
                     ++img_loads;
                     cur_img = img_id;
                 }
-                const uint32_t idesc = umma_idesc_bf16_m128((uint32_t)(it.hpc * D));
+                const uint32_t n_cols = (uint32_t)(it.hpc * D);
+                const uint32_t idesc = PAIR ? umma_idesc_bf16_m256(n_cols) : umma_idesc_bf16_m128(n_cols);
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                    const int s = (int)(tile_no % G::STAGES);
+                    const int stage = (int)(tile_no % G::STAGES);
+                    const uint32_t fill = (uint32_t)(tile_no / G::STAGES);
                     const int a = (int)(tile_no & 1);
                     const uint32_t use = (uint32_t)(tile_no >> 1);
-                    ok = mbar_wait(full_k(s), (uint32_t)((tile_no / G::STAGES) & 1), abort_flag) &&
-                         mbar_wait(tmem_empty(a), (use & 1) ^ 1, abort_flag);
+                    ok = mbar_wait<PAIR>(tmem_empty(a), (use & 1) ^ 1, abort_flag);
                     if (!ok) break;
-                    tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(a * kAccCols);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off = (uint32_t)((ks % 4) * 32);
-                        const uint64_t da = umma_desc_k_sw128(s_k + s * G::STAGE + (ks / 4) * G::CHUNK_A + off);
-                        const uint64_t db = umma_desc_k_sw128(s_img + (ks / 4) * G::CHUNK_B + off);
-                        umma_bf16(d_tmem, da, db, idesc, ks > 0 ? 1u : 0u);
+                    for (int kc = 0; kc < G::KCH; ++kc) {
+                        const int slot = stage * G::KCH + kc;
+                        ok = ok && mbar_wait<PAIR>(full_k(slot), fill & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t da = umma_desc_k_sw128(s_k + slot * kChunkA + ks * 32);
+                            const uint64_t db = umma_desc_k_sw128(s_img + kc * G::CHUNK_B + ks * 32);
+                            const uint32_t acc = (kc | ks) ? 1u : 0u;
+                            if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, acc);
+                            else umma_bf16(d_tmem, da, db, idesc, acc);
+                        }
                     }
-                    umma_commit(tmem_full(a));
+                    if (!ok) break;
+                    if (PAIR) umma_commit_pair(tmem_full(a), 3);
+                    else umma_commit(tmem_full(a));
+                }
+            }
+        } else if (PAIR && lane == 0) {
+            // ---------------------------------------------- peer: report each landed image half
+            long long cur_img = -1;
+            int img_loads = 0;
+            bool ok = true;
+            for (long long item = first; ok && item < p.n_items; item += stride) {
+                const Item it = decode_item(item, p, G::HPC);
+                const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
+                if (img_id != cur_img) {
+                    ok = mbar_wait(img_full, img_loads & 1, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_cluster(mapa(img_peer, 0));
+                    ++img_loads;
+                    cur_img = img_id;
                 }
             }
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ epilogue
+        const int ew = warp - 2;
         const int quarter = warp % 4;              // the TMEM lanes this warp may read
+        const int half = ew / 4;                   // which half of the accumulator columns
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const float inv_2d = 0.5f / (float)D;
+        constexpr int CB = D / 32;                                 // 32-column blocks per head
+        constexpr int HPH = G::HPC >= 2 ? G::HPC / 2 : 1;          // heads per half
+        constexpr int NBH = G::HPC >= 2 ? HPH * CB : CB / 2;       // blocks per half
+        const uint32_t empty_remote = PAIR ? mapa(tmem_empty(0), 0) : 0u;
         long long tile_no = 0, cur_img = -1;
         int img_loads = 0;
         bool ok = true;
@@ -273,6 +362,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
             if (img_id != cur_img) {
                 ok = __all_sync(0xffffffffu, mbar_wait(img_full, img_loads & 1, abort_flag));
+                if (G::HPC == 1) ok = epi_all(ok);
                 if (!ok) break;
                 ++img_loads;
                 cur_img = img_id;
@@ -280,66 +370,99 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
             const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
             for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                const int s = (int)(tile_no % G::STAGES);
+                const int stage = (int)(tile_no % G::STAGES);
                 const int a = (int)(tile_no & 1);
-                ok = __all_sync(0xffffffffu, mbar_wait(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait<PAIR>(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag));
+                if (G::HPC == 1) ok = epi_all(ok);     // the halves meet at a named barrier below
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t k_row = s_k + s * G::STAGE + row * 128;
-                float2 acc[G::HPC];
+                const uint32_t k_row = s_k + stage * G::STAGE + row * 128;
+                float2 acc[HPH][4];
 #pragma unroll
-                for (int j = 0; j < G::HPC; ++j) acc[j] = make_float2(0.f, 0.f);
+                for (int jl = 0; jl < HPH; ++jl)
 #pragma unroll
-                for (int cb = 0; cb < D / 32; ++cb) {
+                    for (int q = 0; q < 4; ++q) acc[jl][q] = make_float2(0.f, 0.f);
+
+                // block bi of this half: local head jl, head j, 32-column block cb
+                auto head_of = [&](int bi) { return G::HPC >= 2 ? half * HPH + bi / CB : 0; };
+                auto cb_of = [&](int bi) { return G::HPC >= 2 ? bi % CB : half * NBH + bi; };
+                uint32_t dv[2][32];
+                if (head_of(0) < it.hpc)
+                    tmem_ld_x32(t_lane + (uint32_t)(a * kAccCols + head_of(0) * D + cb_of(0) * 32), dv[0]);
+#pragma unroll
+                for (int bi = 0; bi < NBH; ++bi) {
+                    const int jl = G::HPC >= 2 ? bi / CB : 0;
+                    const int j = head_of(bi), cb = cb_of(bi);
                     const int c0 = cb * 32;
-                    float2 kf[16];
+                    const bool active = j < it.hpc;
+                    tmem_ld_wait();
+                    if (bi + 1 < NBH && head_of(bi + 1) < it.hpc)
+                        tmem_ld_x32(t_lane + (uint32_t)(a * kAccCols + head_of(bi + 1) * D + cb_of(bi + 1) * 32),
+                                    dv[(bi + 1) & 1]);
+                    if (active) {
+                        float2 kf[16];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int unit = (c0 % 64) / 8 + q;
-                        const uint4 w = lds128(k_row + (c0 / 64) * G::CHUNK_A + ((unit ^ (row & 7)) << 4));
-                        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                        for (int q = 0; q < 4; ++q) {
+                            const int unit = (c0 % 64) / 8 + q;
+                            const uint4 w = lds128(k_row + (c0 / 64) * kChunkA + ((unit ^ (row & 7)) << 4));
+                            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
-                                                        __uint_as_float(ww[e] & 0xffff0000u));
-                    }
+                            for (int e = 0; e < 4; ++e)
+                                kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
+                                                            __uint_as_float(ww[e] & 0xffff0000u));
+                        }
+                        const float4* mu4 = reinterpret_cast<const float4*>(vec_gen + (j * 2 + 0) * D + c0);
+                        const float4* dg4 = reinterpret_cast<const float4*>(vec_gen + (j * 2 + 1) * D + c0);
+                        const uint32_t* dd = dv[bi & 1];
 #pragma unroll
-                    for (int j = 0; j < G::HPC; ++j) {
-                        if (j < it.hpc) {
-                            uint32_t dv[32];
-                            tmem_ld_x32(t_lane + (uint32_t)(a * kAccCols + j * D + c0), dv);
-                            tmem_ld_wait();
-                            const float4* mu4 = reinterpret_cast<const float4*>(vec_gen + (j * 2 + 0) * D + c0);
-                            const float4* dg4 = reinterpret_cast<const float4*>(vec_gen + (j * 2 + 1) * D + c0);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const float4 m = mu4[q], dg = dg4[q];
-                                const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
-                                float2 t0 = fma2(make_float2(dg.x, dg.y), k0, make_float2(m.x, m.y));
-                                float2 t1 = fma2(make_float2(dg.z, dg.w), k1, make_float2(m.z, m.w));
-                                t0 = fma2(make_float2(__uint_as_float(dv[4 * q]), __uint_as_float(dv[4 * q + 1])),
-                                          make_float2(inv_2d, inv_2d), t0);
-                                t1 = fma2(make_float2(__uint_as_float(dv[4 * q + 2]), __uint_as_float(dv[4 * q + 3])),
-                                          make_float2(inv_2d, inv_2d), t1);
-                                acc[j] = fma2(k0, t0, acc[j]);
-                                acc[j] = fma2(k1, t1, acc[j]);
-                            }
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 m = mu4[q], dg = dg4[q];
+                            const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
+                            float2 t0 = fma2(make_float2(dg.x, dg.y), k0, make_float2(m.x, m.y));
+                            float2 t1 = fma2(make_float2(dg.z, dg.w), k1, make_float2(m.z, m.w));
+                            t0.x += __uint_as_float(dd[4 * q]);
+                            t0.y += __uint_as_float(dd[4 * q + 1]);
+                            t1.x += __uint_as_float(dd[4 * q + 2]);
+                            t1.y += __uint_as_float(dd[4 * q + 3]);
+                            acc[jl][(2 * q) & 3] = fma2(k0, t0, acc[jl][(2 * q) & 3]);
+                            acc[jl][(2 * q + 1) & 3] = fma2(k1, t1, acc[jl][(2 * q + 1) & 3]);
                         }
                     }
+                    // hand the 64-channel chunk back to the producer once this warp is done with it
+                    const bool last_use = D == 64 ? bi == NBH - 1 : (bi & 1) == 1;
+                    if (last_use) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(empty_k(stage * G::KCH + (D == 64 ? 0 : cb / 2)));
+                    }
                 }
-                // the accumulator stage and the key tile are free again
+                // the accumulator stage is free again
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(tmem_empty(a));
-                    mbar_arrive(empty_k(s));
+                    if (PAIR && !leader) mbar_arrive_cluster(empty_remote + 8u * a);
+                    else mbar_arrive(tmem_empty(a));
                 }
-                const int key = t * kTileKeys + row;
-                if (key < p.n) {
+                float s_out[HPH];
 #pragma unroll
-                    for (int j = 0; j < G::HPC; ++j)
-                        if (j < it.hpc)
-                            p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] = acc[j].x + acc[j].y;
+                for (int jl = 0; jl < HPH; ++jl) {
+                    const float2 s01 = make_float2(acc[jl][0].x + acc[jl][1].x, acc[jl][0].y + acc[jl][1].y);
+                    const float2 s23 = make_float2(acc[jl][2].x + acc[jl][3].x, acc[jl][2].y + acc[jl][3].y);
+                    s_out[jl] = (s01.x + s23.x) + (s01.y + s23.y);
+                }
+                const int key = t * kKeysPerStep + (int)rank * kTileKeys + row;
+                if (G::HPC == 1) {
+                    // the two halves of the columns meet in shared memory (double-buffered by tile parity)
+                    float* slot = part_gen + (tile_no & 1) * kTileKeys + row;
+                    if (half == 1) *slot = s_out[0];
+                    asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+                    if (half == 0 && key < p.n)
+                        p.logits[((size_t)u * p.Hq + h0) * (size_t)p.n + key] = s_out[0] + *slot;
+                } else if (key < p.n) {
+#pragma unroll
+                    for (int jl = 0; jl < HPH; ++jl) {
+                        const int j = half * HPH + jl;
+                        if (j < it.hpc) p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] = s_out[jl];
+                    }
                 }
             }
         }
@@ -348,9 +471,11 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     // ---------------------------------------------------------------------- teardown
     tc_fence_before_sync();
     __syncthreads();
+    if (PAIR) cluster_sync();          // the peer may still read this CTA's shared memory until here
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, kTmemCols);
+        if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols);
+        else tmem_dealloc(tmem_base, kTmemCols);
     }
     if (threadIdx.x == 0 && *abort_flag) *p.status = (int)EA_ERR_DEVICE_TIMEOUT;
 }
@@ -391,11 +516,13 @@ bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, long lon
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, bool PAIR>
 ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k, const float* mu_bar,
                      const float* sigma_bar, uint8_t* image, float* vec, float* logits, cudaStream_t st) {
-    using G = Geo<D>;
+    using G = Geo<D, PAIR>;
     const int Gq = s.n_q_heads / s.n_kv_heads;
+    constexpr int keys_per_step = PAIR ? 2 * kTileKeys : kTileKeys;
+    const int workers = PAIR ? ctx->sm_count / 2 : ctx->sm_count;     // CTAs or CTA pairs
     MmaParams p;
     p.vec = vec;
     p.image = image;
@@ -405,11 +532,11 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     p.Hkv = s.n_kv_heads;
     p.n = s.n_keys;
     p.n_subsets = (Gq + G::HPC - 1) / G::HPC;
-    p.n_tiles = (s.n_keys + kTileKeys - 1) / kTileKeys;
+    p.n_tiles = (s.n_keys + keys_per_step - 1) / keys_per_step;
     // Work items: enough of them to balance the SMs, long enough to amortise the image load.
     const long long combos = (long long)s.n_units * s.n_kv_heads * p.n_subsets;
     int chunk = p.n_tiles;
-    const long long want_items = 6LL * ctx->sm_count;
+    const long long want_items = 6LL * workers;
     while (chunk > 16 && combos * ((p.n_tiles + chunk - 1) / chunk) < want_items) chunk = (chunk + 1) / 2;
     p.chunk_tiles = chunk;
     p.n_chunks = (p.n_tiles + chunk - 1) / chunk;
@@ -420,20 +547,34 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
 
     sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(mu_bar, sigma_bar, s.n_q_heads, s.n_kv_heads,
                                                                  image, vec);
-    if (cudaFuncSetAttribute(logits_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM) !=
-        cudaSuccess)
+    auto kern = logits_mma_kernel<D, PAIR>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM) != cudaSuccess)
         return EA_ERR_CUDA;
-    const unsigned grid = (unsigned)(p.n_items < ctx->sm_count ? p.n_items : ctx->sm_count);
+    const long long want = p.n_items < workers ? p.n_items : workers;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(PAIR ? 2 * want : want));
+    cfg.blockDim = dim3(kMmaThreads);
+    cfg.dynamicSmemBytes = G::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     ea_count_launches(ctx, 2);
     cudaEvent_t stop = ea_profile_mark_start(ctx, st);
-    logits_mma_kernel<D><<<grid, kMmaThreads, G::SMEM, st>>>(k_map, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, k_map, p);
     ea_profile_mark_stop(ctx, stop, st);
+    if (err != cudaSuccess) return EA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }
 
 }  // namespace
 
 bool ea_mma_path_supported(const ea_shape& s) {
+    if (s.head_dim == 256) return s.n_keys >= 2 * kTileKeys;
     return (s.head_dim == 64 || s.head_dim == 128) && s.n_keys >= kTileKeys;
 }
 
@@ -451,11 +592,14 @@ size_t ea_mma_vec_bytes(const ea_shape& s) {
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                const float* mu_bar, const float* sigma_bar, void* image, float* vec,
                                float* logits, cudaStream_t st) {
+    uint8_t* img = static_cast<uint8_t*>(image);
     switch (s.head_dim) {
         case 64:
-            return launch_mma<64>(ctx, s, k, mu_bar, sigma_bar, static_cast<uint8_t*>(image), vec, logits, st);
+            return launch_mma<64, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, st);
         case 128:
-            return launch_mma<128>(ctx, s, k, mu_bar, sigma_bar, static_cast<uint8_t*>(image), vec, logits, st);
+            return launch_mma<128, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, st);
+        case 256:
+            return launch_mma<256, true>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, st);
         default:
             return EA_ERR_UNSUPPORTED;
     }

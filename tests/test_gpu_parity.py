@@ -87,6 +87,18 @@ def test_whole_path_tempered(ea, oracle, cfg_id, scale, eps):
     assert rep["score_unstable"] == 0
 
 
+@pytest.mark.parametrize("n,scale,eps", [(3000, 20.0, 0.02), (3000, 2.0, 0.02), (4096, 3.0, 0.0), (300, 2.0, 0.02)])
+def test_whole_path_head_dim_256(ea, oracle, n, scale, eps):
+    """The 128k-context config's geometry (head_dim 256, two query heads per KV head) on a short,
+    ragged cache: several key tiles, a partial last tile, and the paired-CTA tensor-core path."""
+    import dataclasses
+    cfg = dataclasses.replace(inputs.CONFIGS[3].tempered(scale, eps), n_layers=1, n_keys=n, n_kept=n // 8)
+    rep = _run_whole_path(ea, oracle, cfg)
+    print(rep)
+    if scale <= 3.0:
+        assert rep["score_unstable"] == 0
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 def test_group_modes(ea, oracle, mode):
     print(_run_whole_path(ea, oracle, inputs.CONFIGS[0].tempered(2.0), group_mode=mode))

@@ -47,22 +47,25 @@ def measured_peaks():
 
 # ------------------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons with nvidia-smi in the background.  It is started
+    before the warm-up (nvidia-smi needs a moment to come up) and reports the samples whose
+    timestamps fall inside the timed region."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu_index = gpu_index
+    def __init__(self, gpu_index: int, period_ms: int = 25):
+        self.gpu_index, self.period_ms = gpu_index, period_ms
         self.proc = None
         self.lines = []
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms",
+                 str(self.period_ms), "-i", str(self.gpu_index)], stdout=subprocess.PIPE,
+                stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except OSError:
@@ -72,31 +75,39 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
-    def stop(self):
+    def stop(self, t0: float, t1: float):
+        """Summary of the samples taken between host times t0 and t1 (time.time())."""
+        import datetime
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(2.5 * self.period_ms / 1e3)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
+        sm, power, mx, reasons = [], [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        pad = 0.5 * self.period_ms / 1e3
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 6:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx = float(parts[1])
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if not (t0 - pad <= ts <= t1 + pad):
+                    continue
+                sm.append(float(parts[1]))
+                mx = float(parts[2])
+                power.append(float(parts[3]))
             except ValueError:
                 continue
-            for name, val in zip(names, parts[2:6]):
+            for name, val in zip(names, parts[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         sm.sort()
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "power_w_max": max(power) if power else None}
 
 
 # ------------------------------------------------------------------------------------- workload
@@ -278,24 +289,26 @@ def main():
     slots, alg_bytes, alg_flops = algorithmic_work(cfg)
     peaks = measured_peaks()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         wl.step(ctx, upc)
     ctx.sync_status()
 
-    sampler = ClockSampler(local)
-    sampler.start()
     barrier(world)
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ctx.profile_begin()
+    t_host0 = time.time()
     ev0.record()
     for _ in range(args.steps):
         wl.step(ctx, upc)
     ev1.record()
     score_ms, score_launches, total_launches = ctx.profile_end()
     torch.cuda.synchronize()
+    t_host1 = time.time()
     barrier(world)
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_host0, t_host1)
     ms_local = ev0.elapsed_time(ev1) / args.steps
     ms = max_over_ranks(ms_local, world, device)
     ctx.sync_status()

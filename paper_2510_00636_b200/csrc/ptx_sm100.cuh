@@ -148,6 +148,19 @@ __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr)
         : "memory");
 }
+// 16 lanes x 32 columns starting at (lane, column) of taddr, in the 16x256b fragment layout:
+// thread t = 4 r + q receives, for jj = 0..3, r[4 jj + 2 s + e] = element (lane r + 8 s,
+// column 8 jj + 2 q + e): two adjacent columns of two rows per 8-column group.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -164,6 +177,17 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t addr) {
     d |= static_cast<uint64_t>(1024 >> 4) << 32;          // stride byte offset: next 8-row group
     d |= static_cast<uint64_t>(1) << 46;                  // descriptor version of sm_100
     d |= static_cast<uint64_t>(2) << 61;                  // layout: 128-byte swizzle
+    return d;
+}
+// Descriptor of a K-major bf16 operand of one K = 16 step stored WITHOUT swizzle as core matrices
+// of 8 rows x 16 bytes (128 contiguous bytes each): K columns 8..15 sit 128 bytes after columns
+// 0..7 (leading byte offset), the next 8 rows 256 bytes on (stride byte offset).
+__device__ __forceinline__ uint64_t umma_desc_k_plain(uint32_t addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(128 >> 4) << 16;
+    d |= static_cast<uint64_t>(256 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
     return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
@@ -243,6 +267,16 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask
 }
 
 // ------------------------------------------------------------------ small helpers
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float2 lds_f2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
@@ -256,6 +290,13 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
         : "=l"(reinterpret_cast<uint64_t&>(d))
         : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)),
           "l"(reinterpret_cast<uint64_t&>(c)));
+    return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+    float2 d;
+    asm("add.rn.f32x2 %0, %1, %2;"
+        : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
     return d;
 }
 __device__ __forceinline__ bool elect_one() {

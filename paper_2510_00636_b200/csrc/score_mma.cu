@@ -4,18 +4,19 @@
 // The dense part is the product K . B^T of a tile of 128 cached keys with a bf16 image B of
 // the covariance; the row-wise quadratic form is finished in the epilogue:
 //     D[i, c]  = sum_a K[i, a] B[c, a]                      (tcgen05.mma, fp32 in tensor memory)
-//     s_{h,i}  = sum_c k_{i,c} ( D[i, c] + mu_bar_c/sqrt(d) + Sigma_bar_cc k_{i,c}/(2d) )
+//                + mu_bar_c / sqrt(d)                        (one more MMA step: ones x (hi, lo) of the term)
+//     s_{h,i}  = sum_c k_{i,c} ( D[i, c] + Sigma_bar_cc k_{i,c}/(2d) )
 // B carries the off-diagonal of Sigma_bar/(2d) at twice bf16 precision for the price of one bf16
 // matrix: the quadratic form only sees B[c,a] + B[a,c], so for a < c the entry B[c,a] holds
 // bf16(Sigma_ac/d) and the mirrored entry B[a,c] holds the bf16 rounding of what that left over.
-// The diagonal stays out of B and enters in fp32 in the epilogue together with the linear term.
+// The diagonal stays out of B and enters in fp32 in the epilogue: two FMAs per accumulator element.
 //
 // A CTA keeps the image of `hpc` query heads of one KV head resident in shared memory
 // (hpc * d = 256 accumulator columns at most) and streams key tiles through a TMA ring:
 //   warp 0     TMA producer (one lane): covariance image (bulk copy) and key tiles (tiled, 128B swizzle)
 //   warp 1     MMA issuer (one lane); owns the tensor-memory allocation
 //   warps 2-9  epilogue, two warps per tensor-memory lane quarter: thread <-> accumulator lane <-> key;
-//              each reads its key row from the staged tile and half of the accumulator columns
+//              each reads half of its key row from the staged tile and the matching accumulator columns
 // Tensor memory holds two accumulator stages so the epilogue of one tile overlaps the MMAs of the
 // next.  With PAIR, two CTAs of a cluster work as one (cta_group::2): each stages its own 128 keys
 // and half of the image rows, the leader issues M = 256 MMAs for both, and each CTA runs the
@@ -42,25 +43,31 @@ struct Geo {
     static constexpr int STAGE = KCH * kChunkA;          // bytes of one key tile
     static constexpr int IMG_ROWS = HPC * D;             // rows of a whole image (accumulator columns)
     static constexpr int CHUNK_B_FULL = IMG_ROWS * 128;  // bytes of one chunk of a whole image (global)
-    static constexpr int IMG_FULL = KCH * CHUNK_B_FULL;  // bytes of a whole image (global)
+    static constexpr int IMG_MAIN = KCH * CHUNK_B_FULL;  // bytes of the covariance part of a whole image (global)
     static constexpr int ROWS_CTA = PAIR ? IMG_ROWS / 2 : IMG_ROWS;   // image rows one CTA keeps
     static constexpr int CHUNK_B = ROWS_CTA * 128;
     static constexpr int IMG_CTA = KCH * CHUNK_B;
     static constexpr int STAGES = D == 256 ? 2 : 4;
     static constexpr int NSLOT = STAGES * KCH;           // ring of 16 KiB chunk slots
-    static constexpr int VEC = HPC * D * 2 * (int)sizeof(float);   // mu' and diagonal vectors
-    static constexpr int PART = 2 * kTileKeys * (int)sizeof(float);
+    static constexpr int VEC = HPC * D * (int)sizeof(float);       // diagonal vectors of the resident heads
+    // linear term: one extra K = 16 MMA step, a constant block of ones times (hi, lo) of mu' per column,
+    // both as unswizzled K-major core matrices (8 rows x 16 bytes; 128 bytes on along K, 256 on along rows)
+    static constexpr int ONES = kTileKeys * 32;
+    static constexpr int LIN_FULL = IMG_ROWS * 32;       // bytes of the mu' operand of a whole image (global)
+    static constexpr int LIN_CTA = ROWS_CTA * 32;
+    static constexpr int IMG_FULL = IMG_MAIN + LIN_FULL; // bytes of a whole image (global)
+    static constexpr int PART = 2 * HPC * kTileKeys * (int)sizeof(float);   // partial sums of the two column halves
     static constexpr int NBAR = 2 * NSLOT + 6;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + VEC + PART + CTRL + 1024;
+    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + ONES + LIN_CTA + VEC + PART + CTRL + 1024;
     // warps that must release a chunk slot before it is refilled
-    static constexpr int SLOT_RELEASERS = D == 256 ? kEpiWarps / 2 : kEpiWarps;
+    static constexpr int SLOT_RELEASERS = D == 64 ? kEpiWarps : kEpiWarps / 2;
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
 struct MmaParams {
-    const float* vec;        // fp32 [U*Hq][2][D]: mu_bar/sqrt(d), diag(Sigma_bar)/(2d)
+    const float* vec;        // fp32 [U*Hq][D]: diag(Sigma_bar)/(2d)
     const uint8_t* image;    // bf16 images, IMG_FULL bytes per (unit, kv head, head subset)
     float* logits;           // fp32 [U, Hq, n]
     int* status;             // device-visible status word
@@ -86,7 +93,7 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
     const int n_subsets = (Gq + G::HPC - 1) / G::HPC;
     const int hs = hg / G::HPC, j = hg % G::HPC;
     const float* S = sigma_bar + (size_t)uh * D * D;
-    uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG_FULL;
+    uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG_FULL;   // 16-byte aligned
     const float inv_d = 1.0f / (float)D;       // a power of two: the scaling is exact
 
     // one 16-byte unit (8 consecutive a) of one row c per thread step
@@ -117,10 +124,20 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
                                               ((unit ^ (row & 7)) << 4));
         *dst = make_uint4(w[0], w[1], w[2], w[3]);
     }
+    // linear-term operand: row (j, c) holds mu_bar_c / sqrt(d) as a bf16 and the bf16 of its remainder in
+    // K columns 0 and 1, zeros elsewhere; unswizzled core-matrix layout (8 rows x 16 bytes, K columns
+    // 8..15 another 128 bytes on, next 8 rows 256 bytes on)
     const float inv_sqrt_d = rsqrtf((float)D), inv_2d = 0.5f / (float)D;
     for (int c = threadIdx.x; c < D; c += blockDim.x) {
-        vec[((size_t)uh * 2 + 0) * D + c] = mu_bar[(size_t)uh * D + c] * inv_sqrt_d;
-        vec[((size_t)uh * 2 + 1) * D + c] = S[(size_t)c * D + c] * inv_2d;
+        const float m = mu_bar[(size_t)uh * D + c] * inv_sqrt_d;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(m);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(m - __bfloat162float(hi));
+        const int row = j * D + c;
+        uint8_t* dst = img + G::IMG_MAIN + (size_t)(row / 8) * 256 + (row % 8) * 16;
+        *reinterpret_cast<uint4*>(dst) =
+            make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
+        vec[(size_t)uh * D + c] = S[(size_t)c * D + c] * inv_2d;
     }
 }
 
@@ -166,7 +183,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_img = base;
     const uint32_t s_k = s_img + G::IMG_CTA;
-    constexpr int kOffVec = G::IMG_CTA + G::STAGES * G::STAGE;
+    constexpr int kOffOnes = G::IMG_CTA + G::STAGES * G::STAGE;
+    const uint32_t s_ones = base + kOffOnes;
+    const uint32_t s_lin = s_ones + G::ONES;
+    constexpr int kOffVec = kOffOnes + G::ONES + G::LIN_CTA;
     const uint32_t s_vec = base + kOffVec;
     const float* vec_gen = reinterpret_cast<const float*>(gen_base + kOffVec);
     float* part_gen = reinterpret_cast<float*>(gen_base + kOffVec + G::VEC);
@@ -200,6 +220,14 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         fence_mbar_init();
         prefetch_tensormap(&k_map);
     }
+    // constant A operand of the linear-term step: K columns 0 and 1 are one, the rest zero
+    // (row r of the tile at (r / 8) * 256 + (r % 8) * 16, K columns 8..15 another 128 bytes on)
+    for (int e = threadIdx.x; e < G::ONES / 16; e += kMmaThreads) {
+        const int piece = e % 16;                       // 16-byte pieces of a 256-byte group of 8 rows
+        uint4 v = make_uint4(piece < 8 ? 0x3f803f80u : 0u, 0u, 0u, 0u);   // two bf16 ones, then zeros
+        *reinterpret_cast<uint4*>(gen_base + kOffOnes + e * 16) = v;
+    }
+    fence_proxy_async_smem();
     if (warp == 1) {
         if (PAIR) {
             tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -241,12 +269,14 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     const int rows = PAIR ? rows_total / 2 : rows_total;
                     const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
                     const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
-                    const uint32_t vec_bytes = (uint32_t)(it.hpc * 2 * D * sizeof(float));
-                    mbar_arrive_expect_tx(img_full, (uint32_t)(G::KCH * rows * 128) + vec_bytes);
-                    const uint8_t* src = p.image + (size_t)img_id * G::IMG_FULL + (size_t)rank * rows * 128;
+                    const uint32_t vec_bytes = (uint32_t)(it.hpc * D * sizeof(float));
+                    mbar_arrive_expect_tx(img_full, (uint32_t)(G::KCH * rows * 128 + rows * 32) + vec_bytes);
+                    const uint8_t* img = p.image + (size_t)img_id * G::IMG_FULL;
+                    const uint8_t* src = img + (size_t)rank * rows * 128;
                     for (int kc = 0; kc < G::KCH; ++kc)
                         bulk_load(s_img + kc * G::CHUNK_B, src + (size_t)kc * G::CHUNK_B_FULL, rows * 128, img_full);
-                    bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * 2 * D, vec_bytes, img_full);
+                    bulk_load(s_lin, img + G::IMG_MAIN + (size_t)rank * rows * 32, rows * 32, img_full);
+                    bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
                     cur_img = img_id;
                 }
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
@@ -321,6 +351,12 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         }
                     }
                     if (!ok) break;
+                    {   // linear term: D += ones . (hi, lo of mu')^T
+                        const uint64_t da = umma_desc_k_plain(s_ones);
+                        const uint64_t db = umma_desc_k_plain(s_lin);
+                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, 1u);
+                        else umma_bf16(d_tmem, da, db, idesc, 1u);
+                    }
                     if (PAIR) umma_commit_pair(tmem_full(a), 3);
                     else umma_commit(tmem_full(a));
                 }
@@ -345,25 +381,28 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ epilogue
+        // Warp (quarter, half): accumulator lanes 32*quarter.. (thread <-> lane <-> key) and the
+        // 32-column blocks [half*CB/2, (half+1)*CB/2) of every head of the pass.  The two halves of
+        // a key meet in shared memory; head j is finished and stored by half j % 2.
         const int ew = warp - 2;
         const int quarter = warp % 4;              // the TMEM lanes this warp may read
-        const int half = ew / 4;                   // which half of the accumulator columns
+        const int half = ew / 4;
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        constexpr int CB = D / 32;                                 // 32-column blocks per head
-        constexpr int HPH = G::HPC >= 2 ? G::HPC / 2 : 1;          // heads per half
-        constexpr int NBH = G::HPC >= 2 ? HPH * CB : CB / 2;       // blocks per half
+        constexpr int CB = D / 32;                 // 32-column blocks per head
+        constexpr int CBH = CB / 2;                // of which this warp handles half
+        constexpr int NB = CBH * G::HPC;           // blocks per tile for this warp
         const uint32_t empty_remote = PAIR ? mapa(tmem_empty(0), 0) : 0u;
+        const float4* dg_base = reinterpret_cast<const float4*>(vec_gen);
         long long tile_no = 0, cur_img = -1;
         int img_loads = 0;
         bool ok = true;
         for (long long item = first; ok && item < p.n_items; item += stride) {
             const Item it = decode_item(item, p, G::HPC);
             const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
+            bool img_ok = true;
             if (img_id != cur_img) {
-                ok = __all_sync(0xffffffffu, mbar_wait(img_full, img_loads & 1, abort_flag));
-                if (G::HPC == 1) ok = epi_all(ok);
-                if (!ok) break;
+                img_ok = mbar_wait(img_full, img_loads & 1, abort_flag);
                 ++img_loads;
                 cur_img = img_id;
             }
@@ -372,97 +411,92 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
                 const int stage = (int)(tile_no % G::STAGES);
                 const int a = (int)(tile_no & 1);
-                ok = __all_sync(0xffffffffu, mbar_wait<PAIR>(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag));
-                if (G::HPC == 1) ok = epi_all(ok);     // the halves meet at a named barrier below
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t k_row = s_k + stage * G::STAGE + row * 128;
-                float2 acc[HPH][4];
+                bool my_ok = img_ok && mbar_wait<PAIR>(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag);
+                my_ok = __all_sync(0xffffffffu, my_ok);
+                float s_out[G::HPC];
+                float* part = part_gen + (tile_no & 1) * (G::HPC * kTileKeys);
+                if (my_ok) {
+                    tc_fence_after_sync();
+                    const uint32_t k_row = s_k + stage * G::STAGE + row * 128;
+                    float2 acc[G::HPC][2];
 #pragma unroll
-                for (int jl = 0; jl < HPH; ++jl)
+                    for (int j = 0; j < G::HPC; ++j) acc[j][0] = acc[j][1] = make_float2(0.f, 0.f);
+                    // block b -> (cb, j): heads innermost so the unpacked key values are reused
+                    auto cb_of = [&](int b) { return half * CBH + b / G::HPC; };
+                    auto addr_of = [&](int b) {
+                        return t_lane + (uint32_t)(a * kAccCols + (b % G::HPC) * D + cb_of(b) * 32);
+                    };
+                    uint32_t dv[2][32];
+                    tmem_ld_x32(addr_of(0), dv[0]);      // head 0 always exists
+                    float2 kf[16];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) acc[jl][q] = make_float2(0.f, 0.f);
-
-                // block bi of this half: local head jl, head j, 32-column block cb
-                auto head_of = [&](int bi) { return G::HPC >= 2 ? half * HPH + bi / CB : 0; };
-                auto cb_of = [&](int bi) { return G::HPC >= 2 ? bi % CB : half * NBH + bi; };
-                uint32_t dv[2][32];
-                if (head_of(0) < it.hpc)
-                    tmem_ld_x32(t_lane + (uint32_t)(a * kAccCols + head_of(0) * D + cb_of(0) * 32), dv[0]);
+                    for (int b = 0; b < NB; ++b) {
+                        const int j = b % G::HPC;
+                        const int cb = cb_of(b);
+                        const int c0 = cb * 32;
+                        if (j == 0) {
 #pragma unroll
-                for (int bi = 0; bi < NBH; ++bi) {
-                    const int jl = G::HPC >= 2 ? bi / CB : 0;
-                    const int j = head_of(bi), cb = cb_of(bi);
-                    const int c0 = cb * 32;
-                    const bool active = j < it.hpc;
-                    tmem_ld_wait();
-                    if (bi + 1 < NBH && head_of(bi + 1) < it.hpc)
-                        tmem_ld_x32(t_lane + (uint32_t)(a * kAccCols + head_of(bi + 1) * D + cb_of(bi + 1) * 32),
-                                    dv[(bi + 1) & 1]);
-                    if (active) {
-                        float2 kf[16];
+                            for (int q = 0; q < 4; ++q) {
+                                const int unit = (c0 % 64) / 8 + q;
+                                const uint4 w = lds128(k_row + (c0 / 64) * kChunkA + ((unit ^ (row & 7)) << 4));
+                                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int unit = (c0 % 64) / 8 + q;
-                            const uint4 w = lds128(k_row + (c0 / 64) * kChunkA + ((unit ^ (row & 7)) << 4));
-                            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
-                                                            __uint_as_float(ww[e] & 0xffff0000u));
+                                for (int e = 0; e < 4; ++e)
+                                    kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
+                                                                __uint_as_float(ww[e] & 0xffff0000u));
+                            }
                         }
-                        const float4* mu4 = reinterpret_cast<const float4*>(vec_gen + (j * 2 + 0) * D + c0);
-                        const float4* dg4 = reinterpret_cast<const float4*>(vec_gen + (j * 2 + 1) * D + c0);
-                        const uint32_t* dd = dv[bi & 1];
+                        tmem_ld_wait();
+                        if (b + 1 < NB && (b + 1) % G::HPC < it.hpc) tmem_ld_x32(addr_of(b + 1), dv[(b + 1) & 1]);
+                        if (j < it.hpc) {
+                            // accumulator = K.B^T + mu' (the linear term rode in on the extra MMA step)
+                            const float4* dg4 = dg_base + (j * D + c0) / 4;
+                            const uint32_t* dd = dv[b & 1];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const float4 m = mu4[q], dg = dg4[q];
-                            const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
-                            float2 t0 = fma2(make_float2(dg.x, dg.y), k0, make_float2(m.x, m.y));
-                            float2 t1 = fma2(make_float2(dg.z, dg.w), k1, make_float2(m.z, m.w));
-                            t0.x += __uint_as_float(dd[4 * q]);
-                            t0.y += __uint_as_float(dd[4 * q + 1]);
-                            t1.x += __uint_as_float(dd[4 * q + 2]);
-                            t1.y += __uint_as_float(dd[4 * q + 3]);
-                            acc[jl][(2 * q) & 3] = fma2(k0, t0, acc[jl][(2 * q) & 3]);
-                            acc[jl][(2 * q + 1) & 3] = fma2(k1, t1, acc[jl][(2 * q + 1) & 3]);
+                            for (int q = 0; q < 8; ++q) {
+                                const float4 dg = dg4[q];
+                                const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
+                                const float2 t0 = fma2(make_float2(dg.x, dg.y), k0,
+                                                       make_float2(__uint_as_float(dd[4 * q]), __uint_as_float(dd[4 * q + 1])));
+                                const float2 t1 = fma2(make_float2(dg.z, dg.w), k1,
+                                                       make_float2(__uint_as_float(dd[4 * q + 2]), __uint_as_float(dd[4 * q + 3])));
+                                acc[j][0] = fma2(k0, t0, acc[j][0]);
+                                acc[j][1] = fma2(k1, t1, acc[j][1]);
+                            }
+                        }
+                        // hand the 64-channel chunk back to the producer once this warp is done with it
+                        const bool chunk_done = j == G::HPC - 1 && (D == 64 || (cb & 1) == 1);
+                        if (chunk_done) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(empty_k(stage * G::KCH + cb / 2));
                         }
                     }
-                    // hand the 64-channel chunk back to the producer once this warp is done with it
-                    const bool last_use = D == 64 ? bi == NBH - 1 : (bi & 1) == 1;
-                    if (last_use) {
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(empty_k(stage * G::KCH + (D == 64 ? 0 : cb / 2)));
+                    // the accumulator stage is free again
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (PAIR && !leader) mbar_arrive_cluster(empty_remote + 8u * a);
+                        else mbar_arrive(tmem_empty(a));
+                    }
+#pragma unroll
+                    for (int j = 0; j < G::HPC; ++j) {
+                        s_out[j] = (acc[j][0].x + acc[j][1].x) + (acc[j][0].y + acc[j][1].y);
+                        if ((j & 1) != half) part[j * kTileKeys + row] = s_out[j];   // finished by the other half
                     }
                 }
-                // the accumulator stage is free again
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) {
-                    if (PAIR && !leader) mbar_arrive_cluster(empty_remote + 8u * a);
-                    else mbar_arrive(tmem_empty(a));
-                }
-                float s_out[HPH];
-#pragma unroll
-                for (int jl = 0; jl < HPH; ++jl) {
-                    const float2 s01 = make_float2(acc[jl][0].x + acc[jl][1].x, acc[jl][0].y + acc[jl][1].y);
-                    const float2 s23 = make_float2(acc[jl][2].x + acc[jl][3].x, acc[jl][2].y + acc[jl][3].y);
-                    s_out[jl] = (s01.x + s23.x) + (s01.y + s23.y);
+                // one named barrier per tile: the halves exchange their partial sums, and a wait
+                // that gave up anywhere stops every epilogue warp at the same tile
+                if (!epi_all(my_ok)) {
+                    ok = false;
+                    break;
                 }
                 const int key = t * kKeysPerStep + (int)rank * kTileKeys + row;
-                if (G::HPC == 1) {
-                    // the two halves of the columns meet in shared memory (double-buffered by tile parity)
-                    float* slot = part_gen + (tile_no & 1) * kTileKeys + row;
-                    if (half == 1) *slot = s_out[0];
-                    asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
-                    if (half == 0 && key < p.n)
-                        p.logits[((size_t)u * p.Hq + h0) * (size_t)p.n + key] = s_out[0] + *slot;
-                } else if (key < p.n) {
+                if (key < p.n) {
 #pragma unroll
-                    for (int jl = 0; jl < HPH; ++jl) {
-                        const int j = half * HPH + jl;
-                        if (j < it.hpc) p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] = s_out[jl];
-                    }
+                    for (int j = 0; j < G::HPC; ++j)
+                        if ((j & 1) == half && j < it.hpc)
+                            p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] =
+                                s_out[j] + part[j * kTileKeys + row];
                 }
             }
         }
@@ -582,11 +616,11 @@ size_t ea_mma_image_bytes(const ea_shape& s) {
     const int Gq = s.n_q_heads / s.n_kv_heads;
     const int hpc = 256 / s.head_dim;
     const size_t subsets = (size_t)((Gq + hpc - 1) / hpc);
-    return (size_t)s.n_units * s.n_kv_heads * subsets * hpc * s.head_dim * s.head_dim * 2;
+    return (size_t)s.n_units * s.n_kv_heads * subsets * ((size_t)hpc * s.head_dim * s.head_dim * 2 + (size_t)hpc * s.head_dim * 32);
 }
 
 size_t ea_mma_vec_bytes(const ea_shape& s) {
-    return (size_t)s.n_units * s.n_q_heads * 2 * s.head_dim * sizeof(float);
+    return (size_t)s.n_units * s.n_q_heads * s.head_dim * sizeof(float);
 }
 
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,

@@ -74,9 +74,10 @@ struct MmaParams {
     int Hq, Hkv, n;
     int n_subsets;           // head subsets per KV head
     int n_tiles;             // steps per head (128 keys per step, 256 with PAIR)
-    int chunk_tiles;         // steps per work item
-    int n_chunks;            // work items per head subset
-    long long n_items;
+    int chunk_tiles;         // steps per work unit
+    int n_chunks;            // work units per (unit, kv head)
+    int n_groups;            // groups of n_subsets workers; a group walks a contiguous range of work units
+    long long n_work;        // work units in all: (unit, kv head, chunk)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -146,12 +147,14 @@ struct Item {
     int ug, hs, tile0, tile1, hpc;
 };
 
-__device__ __forceinline__ Item decode_item(long long item, const MmaParams& p, int hpc_max) {
+// Work unit w of head subset hs: a run of key tiles of one (unit, kv head).  The workers of a group
+// (one per head subset) walk the same units at the same time, so the key tiles they share are
+// fetched from HBM once, and a worker changes its covariance image only when the head changes.
+__device__ __forceinline__ Item decode_item(long long w, int hs, const MmaParams& p, int hpc_max) {
     Item it;
-    it.hs = (int)(item % p.n_subsets);
-    const long long r = item / p.n_subsets;
-    const int chunk = (int)(r % p.n_chunks);
-    it.ug = (int)(r / p.n_chunks);
+    it.hs = hs;
+    const int chunk = (int)(w % p.n_chunks);
+    it.ug = (int)(w / p.n_chunks);
     it.tile0 = chunk * p.chunk_tiles;
     it.tile1 = min(p.n_tiles, it.tile0 + p.chunk_tiles);
     const int Gq = p.Hq / p.Hkv;
@@ -243,8 +246,11 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const long long first = PAIR ? blockIdx.x / 2 : blockIdx.x;
-    const long long stride = PAIR ? gridDim.x / 2 : gridDim.x;
+    const int worker = PAIR ? blockIdx.x / 2 : blockIdx.x;
+    const int my_hs = worker % p.n_subsets;
+    const long long my_group = worker / p.n_subsets;
+    const long long first = p.n_work * my_group / p.n_groups;
+    const long long last = p.n_work * (my_group + 1) / p.n_groups;
     constexpr int kKeysPerStep = PAIR ? 2 * kTileKeys : kTileKeys;
 
     if (warp == 0) {
@@ -252,8 +258,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         if (lane == 0) {
             long long tile_no = 0, cur_img = -1;
             bool ok = true;
-            for (long long item = first; ok && item < p.n_items; item += stride) {
-                const Item it = decode_item(item, p, G::HPC);
+            for (long long item = first; ok && item < last; ++item) {
+                const Item it = decode_item(item, my_hs, p, G::HPC);
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
                     // every tile that used the resident image must have left the epilogue
@@ -315,8 +321,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             long long tile_no = 0, cur_img = -1;
             int img_loads = 0;
             bool ok = true;
-            for (long long item = first; ok && item < p.n_items; item += stride) {
-                const Item it = decode_item(item, p, G::HPC);
+            for (long long item = first; ok && item < last; ++item) {
+                const Item it = decode_item(item, my_hs, p, G::HPC);
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
                     ok = mbar_wait(img_full, img_loads & 1, abort_flag);
@@ -366,8 +372,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             long long cur_img = -1;
             int img_loads = 0;
             bool ok = true;
-            for (long long item = first; ok && item < p.n_items; item += stride) {
-                const Item it = decode_item(item, p, G::HPC);
+            for (long long item = first; ok && item < last; ++item) {
+                const Item it = decode_item(item, my_hs, p, G::HPC);
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
                     ok = mbar_wait(img_full, img_loads & 1, abort_flag);
@@ -393,12 +399,11 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         constexpr int CBH = CB / 2;                // of which this warp handles half
         constexpr int NB = CBH * G::HPC;           // blocks per tile for this warp
         const uint32_t empty_remote = PAIR ? mapa(tmem_empty(0), 0) : 0u;
-        const float4* dg_base = reinterpret_cast<const float4*>(vec_gen);
         long long tile_no = 0, cur_img = -1;
         int img_loads = 0;
         bool ok = true;
-        for (long long item = first; ok && item < p.n_items; item += stride) {
-            const Item it = decode_item(item, p, G::HPC);
+        for (long long item = first; ok && item < last; ++item) {
+            const Item it = decode_item(item, my_hs, p, G::HPC);
             const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
             bool img_ok = true;
             if (img_id != cur_img) {
@@ -446,15 +451,22 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                                                                 __uint_as_float(ww[e] & 0xffff0000u));
                             }
                         }
+                        // the block's diagonal constants, requested before the accumulator wait so that
+                        // their latency is not paid inside the arithmetic
+                        uint4 dgv[8];
+                        if (j < it.hpc) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) dgv[q] = lds128(s_vec + (uint32_t)((j * D + c0 + 4 * q) * 4));
+                        }
                         tmem_ld_wait();
                         if (b + 1 < NB && (b + 1) % G::HPC < it.hpc) tmem_ld_x32(addr_of(b + 1), dv[(b + 1) & 1]);
                         if (j < it.hpc) {
                             // accumulator = K.B^T + mu' (the linear term rode in on the extra MMA step)
-                            const float4* dg4 = dg_base + (j * D + c0) / 4;
                             const uint32_t* dd = dv[b & 1];
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
-                                const float4 dg = dg4[q];
+                                const float4 dg = make_float4(__uint_as_float(dgv[q].x), __uint_as_float(dgv[q].y),
+                                                              __uint_as_float(dgv[q].z), __uint_as_float(dgv[q].w));
                                 const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
                                 const float2 t0 = fma2(make_float2(dg.x, dg.y), k0,
                                                        make_float2(__uint_as_float(dd[4 * q]), __uint_as_float(dd[4 * q + 1])));
@@ -567,14 +579,17 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     p.n = s.n_keys;
     p.n_subsets = (Gq + G::HPC - 1) / G::HPC;
     p.n_tiles = (s.n_keys + keys_per_step - 1) / keys_per_step;
-    // Work items: enough of them to balance the SMs, long enough to amortise the image load.
-    const long long combos = (long long)s.n_units * s.n_kv_heads * p.n_subsets;
+    // Workers come in groups of n_subsets (one per head subset); every group gets an equal,
+    // contiguous share of the work units, which are cut fine enough to balance the groups.
+    const long long heads = (long long)s.n_units * s.n_kv_heads;
+    p.n_groups = workers / p.n_subsets;
+    if (p.n_groups < 1) return EA_ERR_UNSUPPORTED;
+    if (p.n_groups > heads * p.n_tiles) p.n_groups = (int)(heads * p.n_tiles);
     int chunk = p.n_tiles;
-    const long long want_items = 6LL * workers;
-    while (chunk > 16 && combos * ((p.n_tiles + chunk - 1) / chunk) < want_items) chunk = (chunk + 1) / 2;
+    while (chunk > 4 && heads * ((p.n_tiles + chunk - 1) / chunk) < 32LL * p.n_groups) chunk = (chunk + 1) / 2;
     p.chunk_tiles = chunk;
     p.n_chunks = (p.n_tiles + chunk - 1) / chunk;
-    p.n_items = combos * p.n_chunks;
+    p.n_work = heads * p.n_chunks;
 
     CUtensorMap k_map;
     if (!make_k_map(&k_map, k, D, s.n_keys, (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
@@ -584,7 +599,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     auto kern = logits_mma_kernel<D, PAIR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM) != cudaSuccess)
         return EA_ERR_CUDA;
-    const long long want = p.n_items < workers ? p.n_items : workers;
+    const long long want = (long long)p.n_groups * p.n_subsets;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * want : want));
     cfg.blockDim = dim3(kMmaThreads);

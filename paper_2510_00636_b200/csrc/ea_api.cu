@@ -38,6 +38,7 @@ ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     const bool mma = ea_mma_path_supported(s);
     p.image = off;      off = ea_align_up(off + (mma ? ea_mma_image_bytes(s) : 0), 1024);
     p.vec = off;        off = ea_align_up(off + (mma ? ea_mma_vec_bytes(s) : 0), 256);
+    p.lse_part = off;   off = ea_align_up(off + (mma ? ea_mma_lse_part_bytes(s) : 0), 256);
     p.total = off;
     return p;
 }
@@ -197,15 +198,27 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     float* logits = logits_opt ? logits_opt : reinterpret_cast<float*>(ws + plan.logits);
     float* lse = reinterpret_cast<float*>(ws + plan.lse);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (ea_mma_path_supported(*shape))
-        st = ea_launch_logits_mma(ctx, *shape, static_cast<const __nv_bfloat16*>(k), mu_bar, sigma_bar,
-                                  ws + plan.image, reinterpret_cast<float*>(ws + plan.vec), logits, stream);
-    else
-        st = ea_launch_logits_simt(ctx, *shape, static_cast<const __nv_bfloat16*>(k), mu_bar, sigma_bar,
-                                   logits, stream);
-    if (st == EA_OK)
-        st = ea_launch_finalize(ctx, *shape, logits, static_cast<const __nv_bfloat16*>(v), epsilon, lse,
-                                scores, stream);
+    const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+    const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
+    if (ea_mma_path_supported(*shape) && shape->group_mode != EA_GROUP_MEAN_LOGIT) {
+        // tensor-core log-scores with the log-sum-exp partials from their epilogue
+        float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
+        int n_chunks = 0;
+        st = ea_launch_logits_mma(ctx, *shape, kb, mu_bar, sigma_bar, ws + plan.image,
+                                  reinterpret_cast<float*>(ws + plan.vec), logits, lse_part, &n_chunks, stream);
+        if (st == EA_OK) st = ea_launch_lse_combine(ctx, *shape, lse_part, n_chunks, lse, stream);
+        if (st == EA_OK) st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, true, scores, stream);
+    } else {
+        if (ea_mma_path_supported(*shape)) {
+            int n_chunks = 0;
+            st = ea_launch_logits_mma(ctx, *shape, kb, mu_bar, sigma_bar, ws + plan.image,
+                                      reinterpret_cast<float*>(ws + plan.vec), logits,
+                                      reinterpret_cast<float*>(ws + plan.lse_part), &n_chunks, stream);
+        } else {
+            st = ea_launch_logits_simt(ctx, *shape, kb, mu_bar, sigma_bar, logits, stream);
+        }
+        if (st == EA_OK) st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, false, scores, stream);
+    }
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

@@ -46,7 +46,8 @@ struct ea_ws_plan {
     size_t lse;          // fp32 [U, Hq]                 (ea_score)
     size_t sel_state;    // uint32 [U*Hkv, 4]            (ea_select_compact)
     size_t image;        // bf16 covariance images of the tensor-core log-score kernel (ea_score)
-    size_t vec;          // fp32 [U*Hq, 2, d] epilogue vectors of that kernel            (ea_score)
+    size_t vec;          // fp32 [U*Hq, d] epilogue vectors of that kernel               (ea_score)
+    size_t lse_part;     // fp32 [U*Hq, chunks, 2] log-sum-exp partials of that kernel    (ea_score)
     size_t total;
 };
 
@@ -73,12 +74,16 @@ ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv
 bool ea_mma_path_supported(const ea_shape& s);
 size_t ea_mma_image_bytes(const ea_shape& s);
 size_t ea_mma_vec_bytes(const ea_shape& s);
+size_t ea_mma_lse_part_bytes(const ea_shape& s);
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                const float* mu_bar, const float* sigma_bar, void* image, float* vec,
-                               float* logits, cudaStream_t st);
+                               float* logits, float* lse_part, int* n_chunks, cudaStream_t st);
+// log-sum-exp per softmax row from the per-work-unit partials of the tensor-core kernel
+ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const float* lse_part, int n_chunks,
+                                float* lse, cudaStream_t st);
 
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
-                             const __nv_bfloat16* v, float epsilon, float* lse, float* scores,
+                             const __nv_bfloat16* v, float epsilon, float* lse, bool lse_ready, float* scores,
                              cudaStream_t st);
 
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,

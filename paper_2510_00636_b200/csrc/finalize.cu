@@ -119,13 +119,32 @@ finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
     scores[(size_t)ug * n + key] = (a + epsilon) * sqrtf(my_sumsq);
 }
 
+
+// One thread per softmax row: combine the (max, sum of exp) partials of its work units in order.
+__global__ void lse_combine_kernel(const float* __restrict__ lse_part, int n_rows, int n_chunks,
+                                   float* __restrict__ lse) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n_rows) return;
+    const float* pp = lse_part + (size_t)r * n_chunks * 2;
+    float m = -INFINITY, l = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+        const float mo = pp[2 * c], lo = pp[2 * c + 1];
+        const float mn = fmaxf(m, mo);
+        l = mn == -INFINITY ? 0.f : l * expf(m - mn) + lo * expf(mo - mn);
+        m = mn;
+    }
+    lse[r] = m + logf(l);
+}
+
 }  // namespace
 
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
-                             const __nv_bfloat16* v, float epsilon, float* lse, float* scores,
+                             const __nv_bfloat16* v, float epsilon, float* lse, bool lse_ready, float* scores,
                              cudaStream_t st) {
     const int G = s.n_q_heads / s.n_kv_heads;
-    if (s.group_mode == EA_GROUP_MEAN_LOGIT)
+    if (lse_ready) {
+        // the log-sum-exp of every softmax row was assembled from the log-score kernel's partials
+    } else if (s.group_mode == EA_GROUP_MEAN_LOGIT)
         lse_kernel<<<s.n_units * s.n_kv_heads, kLseThreads, 0, st>>>(logits, s.n_keys, G, lse);
     else
         lse_kernel<<<s.n_units * s.n_q_heads, kLseThreads, 0, st>>>(logits, s.n_keys, 1, lse);
@@ -150,6 +169,15 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
         default:
             return EA_ERR_UNSUPPORTED;
     }
-    ea_count_launches(ctx, 2);
+    ea_count_launches(ctx, lse_ready ? 1 : 2);
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+
+ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const float* lse_part, int n_chunks,
+                                float* lse, cudaStream_t st) {
+    const int rows = s.n_units * s.n_q_heads;
+    lse_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(lse_part, rows, n_chunks, lse);
+    ea_count_launches(ctx, 1);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

@@ -57,9 +57,10 @@ struct Geo {
     static constexpr int LIN_CTA = ROWS_CTA * 32;
     static constexpr int IMG_FULL = IMG_MAIN + LIN_FULL; // bytes of a whole image (global)
     static constexpr int PART = 2 * HPC * kTileKeys * (int)sizeof(float);   // partial sums of the two column halves
+    static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
     static constexpr int NBAR = 2 * NSLOT + 6;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + ONES + LIN_CTA + VEC + PART + CTRL + 1024;
+    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + ONES + LIN_CTA + VEC + PART + RED + CTRL + 1024;
     // warps that must release a chunk slot before it is refilled
     static constexpr int SLOT_RELEASERS = D == 64 ? kEpiWarps : kEpiWarps / 2;
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
@@ -70,6 +71,7 @@ struct MmaParams {
     const float* vec;        // fp32 [U*Hq][D]: diag(Sigma_bar)/(2d)
     const uint8_t* image;    // bf16 images, IMG_FULL bytes per (unit, kv head, head subset)
     float* logits;           // fp32 [U, Hq, n]
+    float* lse_part;         // fp32 [U*Hq][n_chunks (x2 for CTA pairs)][2]: (max, sum of exp) per work unit and CTA
     int* status;             // device-visible status word
     int Hq, Hkv, n;
     int n_subsets;           // head subsets per KV head
@@ -193,8 +195,9 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     const uint32_t s_vec = base + kOffVec;
     const float* vec_gen = reinterpret_cast<const float*>(gen_base + kOffVec);
     float* part_gen = reinterpret_cast<float*>(gen_base + kOffVec + G::VEC);
-    const uint32_t s_bar = base + kOffVec + G::VEC + G::PART;
-    uint8_t* bar_gen = gen_base + kOffVec + G::VEC + G::PART;
+    float* red_gen = reinterpret_cast<float*>(gen_base + kOffVec + G::VEC + G::PART);
+    const uint32_t s_bar = base + kOffVec + G::VEC + G::PART + G::RED;
+    uint8_t* bar_gen = gen_base + kOffVec + G::VEC + G::PART + G::RED;
     auto full_k = [&](int slot) { return s_bar + 8u * slot; };
     auto empty_k = [&](int slot) { return s_bar + 8u * (G::NSLOT + slot); };
     auto tmem_full = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + a); };
@@ -413,6 +416,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             }
             const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
             const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
+            // running (max, sum of exp) of this thread's keys, for the heads this half finishes
+            float m_run[G::HPC], l_run[G::HPC];
+#pragma unroll
+            for (int j = 0; j < G::HPC; ++j) { m_run[j] = -INFINITY; l_run[j] = 0.f; }
             for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
                 const int stage = (int)(tile_no % G::STAGES);
                 const int a = (int)(tile_no & 1);
@@ -506,10 +513,50 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 if (key < p.n) {
 #pragma unroll
                     for (int j = 0; j < G::HPC; ++j)
-                        if ((j & 1) == half && j < it.hpc)
-                            p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] =
-                                s_out[j] + part[j * kTileKeys + row];
+                        if ((j & 1) == half && j < it.hpc) {
+                            const float sv = s_out[j] + part[j * kTileKeys + row];
+                            p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] = sv;
+                            const float m_new = fmaxf(m_run[j], sv);
+                            l_run[j] = l_run[j] * __expf(m_run[j] - m_new) + __expf(sv - m_new);
+                            m_run[j] = m_new;
+                        }
                 }
+            }
+            if (!ok) break;
+            // log-sum-exp partial of the work unit: lanes, then the four warps of the finishing half
+#pragma unroll
+            for (int j = 0; j < G::HPC; ++j)
+                if ((j & 1) == half) {
+                    float m = m_run[j], l = l_run[j];
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) {
+                        const float mo = __shfl_xor_sync(0xffffffffu, m, off);
+                        const float lo = __shfl_xor_sync(0xffffffffu, l, off);
+                        const float mn = fmaxf(m, mo);
+                        l = mn == -INFINITY ? 0.f : l * __expf(m - mn) + lo * __expf(mo - mn);
+                        m = mn;
+                    }
+                    if (lane == 0) {
+                        red_gen[(j * 4 + quarter) * 2 + 0] = m;
+                        red_gen[(j * 4 + quarter) * 2 + 1] = l;
+                    }
+                }
+            if (!epi_all(true)) { ok = false; break; }
+            if (threadIdx.x - 64 < G::HPC && (int)(threadIdx.x - 64) < it.hpc) {
+                const int j = threadIdx.x - 64;
+                float m = -INFINITY, l = 0.f;
+                for (int w = 0; w < 4; ++w) {          // fixed order: bitwise reproducible
+                    const float mo = red_gen[(j * 4 + w) * 2], lo = red_gen[(j * 4 + w) * 2 + 1];
+                    const float mn = fmaxf(m, mo);
+                    l = mn == -INFINITY ? 0.f : l * __expf(m - mn) + lo * __expf(mo - mn);
+                    m = mn;
+                }
+                // one slot per work unit and CTA of the pair
+                constexpr int R = PAIR ? 2 : 1;
+                const int slot = (int)(item % p.n_chunks) * R + (int)rank;
+                float* dst = p.lse_part + (((size_t)u * p.Hq + h0 + j) * (p.n_chunks * R) + slot) * 2;
+                dst[0] = m;
+                dst[1] = l;
             }
         }
     }
@@ -564,7 +611,8 @@ bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, long lon
 
 template <int D, bool PAIR>
 ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k, const float* mu_bar,
-                     const float* sigma_bar, uint8_t* image, float* vec, float* logits, cudaStream_t st) {
+                     const float* sigma_bar, uint8_t* image, float* vec, float* logits, float* lse_part,
+                     int* n_chunks_out, cudaStream_t st) {
     using G = Geo<D, PAIR>;
     const int Gq = s.n_q_heads / s.n_kv_heads;
     constexpr int keys_per_step = PAIR ? 2 * kTileKeys : kTileKeys;
@@ -573,6 +621,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     p.vec = vec;
     p.image = image;
     p.logits = logits;
+    p.lse_part = lse_part;
     p.status = ctx->status_dev;
     p.Hq = s.n_q_heads;
     p.Hkv = s.n_kv_heads;
@@ -590,6 +639,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     p.chunk_tiles = chunk;
     p.n_chunks = (p.n_tiles + chunk - 1) / chunk;
     p.n_work = heads * p.n_chunks;
+    *n_chunks_out = p.n_chunks * (PAIR ? 2 : 1);
 
     CUtensorMap k_map;
     if (!make_k_map(&k_map, k, D, s.n_keys, (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
@@ -638,17 +688,22 @@ size_t ea_mma_vec_bytes(const ea_shape& s) {
     return (size_t)s.n_units * s.n_q_heads * s.head_dim * sizeof(float);
 }
 
+size_t ea_mma_lse_part_bytes(const ea_shape& s) {
+    // at most one work unit per 128-key tile
+    return (size_t)s.n_units * s.n_q_heads * (size_t)((s.n_keys + kTileKeys - 1) / kTileKeys) * 2 * sizeof(float);
+}
+
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                const float* mu_bar, const float* sigma_bar, void* image, float* vec,
-                               float* logits, cudaStream_t st) {
+                               float* logits, float* lse_part, int* n_chunks, cudaStream_t st) {
     uint8_t* img = static_cast<uint8_t*>(image);
     switch (s.head_dim) {
         case 64:
-            return launch_mma<64, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, st);
+            return launch_mma<64, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, lse_part, n_chunks, st);
         case 128:
-            return launch_mma<128, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, st);
+            return launch_mma<128, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, lse_part, n_chunks, st);
         case 256:
-            return launch_mma<256, true>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, st);
+            return launch_mma<256, true>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, lse_part, n_chunks, st);
         default:
             return EA_ERR_UNSUPPORTED;
     }

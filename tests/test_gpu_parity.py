@@ -99,6 +99,17 @@ def test_whole_path_head_dim_256(ea, oracle, n, scale, eps):
         assert rep["score_unstable"] == 0
 
 
+@pytest.mark.parametrize("cfg_id,layer", [(2, 3), (3, 0), (4, 1)])
+def test_whole_path_full_size_layer(ea, oracle, cfg_id, layer):
+    """One layer of the benchmark workloads at their full sizes (32k keys at head_dim 128, 128k keys
+    at head_dim 256, the decode batch with seven query heads per KV head), same shapes and launch
+    configuration per layer as the benchmark, every output element checked against the oracle."""
+    import dataclasses
+    cfg = dataclasses.replace(inputs.CONFIGS[cfg_id], n_layers=1)
+    rep = _run_whole_path(ea, oracle, cfg, layer=layer)
+    print(rep)
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 def test_group_modes(ea, oracle, mode):
     print(_run_whole_path(ea, oracle, inputs.CONFIGS[0].tempered(2.0), group_mode=mode))

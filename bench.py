@@ -31,6 +31,11 @@ import torch  # noqa: E402
 
 from paper_2510_00636_b200 import inputs  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the log-score kernel divided by the
+# key-slots of that launch (ncu --set full, profiles/logits_mma_kernel_*); None = not captured for
+# the current kernel
+NCU_DRAM_BYTES_PER_KEY_SLOT = {256: 1.1018e9 / 2097152, 128: None, 64: None}
+
 METRIC = "kv_keys_scored_and_compacted_per_second"
 UNIT = "Gkeys/s"
 
@@ -195,28 +200,33 @@ def barrier(world):
 
 # ------------------------------------------------------------------------------------- CPU oracle legs
 def oracle_sample(cfg: inputs.EAConfig, target_seconds=15.0):
-    """A bounded sample of the workload for the fp64 oracle: layer 0, every head, the first
-    `n_sample` keys, sized for roughly `target_seconds` of CPU work (about 2 GFLOP/s/core)."""
+    """Keys per head in one oracle sample: the first `n_sample` keys of every head of a layer, sized
+    for roughly `target_seconds` of CPU work (about 3 GFLOP/s/core in fp64), at most the whole layer."""
     cores = len(os.sched_getaffinity(0))
     per_key = 2.0 * cfg.head_dim ** 2 * cfg.n_q_heads * cfg.batch          # fp64 FLOPs per key index
-    n_sample = int(target_seconds * 2.0e9 * min(cores, cfg.n_q_heads * cfg.batch) / per_key)
+    n_sample = int(target_seconds * 3.0e9 * min(cores, cfg.n_q_heads * cfg.batch) / per_key)
     n_sample = max(256, min(cfg.n_keys, n_sample // 256 * 256))
     return n_sample
 
 
-def time_oracle(cfg, n_sample, repeats=1):
+def time_oracle(cfg, n_sample, min_seconds=10.0, max_layers=4):
+    """Times the oracle, as it stands, on whole-path passes over successive layers (the first
+    `n_sample` keys of every head) until `min_seconds` of CPU work are done.  -> (key-slots, seconds,
+    threads, layers used)."""
     from oracle import ea_oracle
-    q, k, v, pos = inputs.generate_layer(cfg, layer=0, device="cpu", n_keys=n_sample)
-    qb, kb, vb = inputs.bits(q), inputs.bits(k), inputs.bits(v)
-    n_kept = max(1, int(round(n_sample * cfg.n_kept / cfg.n_keys)))
-    best = None
-    for _ in range(repeats):
+    slots, total, layers = 0, 0.0, 0
+    for layer in range(min(cfg.n_layers, max_layers)):
+        q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device="cpu", n_keys=n_sample)
+        qb, kb, vb = inputs.bits(q), inputs.bits(k), inputs.bits(v)
+        n_kept = max(1, int(round(n_sample * cfg.n_kept / cfg.n_keys)))
         t0 = time.perf_counter()
         ea_oracle.compress(qb, kb, vb, pos.numpy(), cfg.n_future, cfg.rope_base, cfg.eps, n_kept)
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    slots = cfg.batch * cfg.n_kv_heads * n_sample
-    return slots, best, ea_oracle.num_threads()
+        total += time.perf_counter() - t0
+        slots += cfg.batch * cfg.n_kv_heads * n_sample
+        layers += 1
+        if total >= min_seconds:
+            break
+    return slots, total, ea_oracle.num_threads(), layers
 
 
 def run_reference(args, cfg):
@@ -328,7 +338,11 @@ def main():
         achieved = bytes_per_launch / (avg_score_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"]}
-    roofline.update({"traffic": None, "kernel": "log-score kernel (k.mu/sqrt(d) + k'Sigma k/2d)",
+    # DRAM bytes per launch from the ncu capture of this kernel (profiles/): measured on a 2-layer
+    # case of the same shapes and scaled by the key-slots of a launch (traffic is proportional to them)
+    traffic_per_slot = NCU_DRAM_BYTES_PER_KEY_SLOT.get(cfg.head_dim)
+    traffic = None if traffic_per_slot is None else traffic_per_slot * slots / n_calls
+    roofline.update({"traffic": traffic, "kernel": "log-score kernel (k.mu/sqrt(d) + k'Sigma k/2d)",
                      "kernel_ms": avg_score_ms, "launches_timed": score_launches,
                      "peak_source": peaks["source"] + " (sustained bf16 matmul)"})
     # whole-path roofline: the slower of the K.Sigma FLOPs at tensor peak and the K/V bytes at HBM bandwidth
@@ -358,11 +372,11 @@ def main():
 
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
         n_sample = oracle_sample(cfg)
-        o_slots, o_s, cores = time_oracle(cfg, n_sample)
+        o_slots, o_s, cores, o_layers = time_oracle(cfg, n_sample)
         result["cpu_baseline"] = {
             "value": o_slots / o_s / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"layer 0, all {cfg.n_kv_heads} KV heads, first {n_sample} of {cfg.n_keys} keys "
-                      f"({o_slots} key-slots, {o_s:.1f} s)"}
+            "sample": f"first {o_layers} layer(s), all {cfg.n_kv_heads} KV heads, first {n_sample} of "
+                      f"{cfg.n_keys} keys ({o_slots} key-slots, {o_s:.1f} s)"}
     if rank == 0:
         print(json.dumps(result))
     if world > 1:

@@ -34,7 +34,6 @@ ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     p.rope_coef = off;  off = ea_align_up(off + U * (d / 2) * 2 * sizeof(float), 256);
     p.logits = off;     off = ea_align_up(off + U * Hq * n * sizeof(float), 256);
     p.lse = off;        off = ea_align_up(off + U * Hq * sizeof(float), 256);
-    p.sel_state = off;  off = ea_align_up(off + U * Hkv * 4 * sizeof(uint32_t), 256);
     const bool mma = ea_mma_path_supported(s);
     p.image = off;      off = ea_align_up(off + (mma ? ea_mma_image_bytes(s) : 0), 1024);
     p.vec = off;        off = ea_align_up(off + (mma ? ea_mma_vec_bytes(s) : 0), 256);

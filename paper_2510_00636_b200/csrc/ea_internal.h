@@ -44,7 +44,6 @@ struct ea_ws_plan {
     size_t rope_coef;    // fp32 [U, d/2, 2]             (ea_query_stats)
     size_t logits;       // fp32 [U, Hq, n]              (ea_score, when logits_opt == NULL)
     size_t lse;          // fp32 [U, Hq]                 (ea_score)
-    size_t sel_state;    // uint32 [U*Hkv, 4]            (ea_select_compact)
     size_t image;        // bf16 covariance images of the tensor-core log-score kernel (ea_score)
     size_t vec;          // fp32 [U*Hq, d] epilogue vectors of that kernel               (ea_score)
     size_t lse_part;     // fp32 [U*Hq, chunks, 2] log-sum-exp partials of that kernel    (ea_score)

@@ -195,6 +195,34 @@ def test_score_ragged_sizes(ea, oracle, n):
     np.testing.assert_allclose(sc.cpu().numpy(), sc_r, rtol=1e-2)
 
 
+def test_decode_events_below_the_budget_keep_every_key(ea, oracle):
+    """Streaming decode: while the cache is within its budget (the first events of the schedule) scores
+    are still computed but compaction is the identity; the first event above the budget evicts."""
+    import dataclasses
+    base = inputs.CONFIGS[4]
+    events = inputs.decode_schedule()
+    for pos, n, kept in (events[0], events[3], events[4]):
+        cfg = dataclasses.replace(base, n_layers=1, batch=2, n_keys=n, n_kept=kept)
+        q, k, v, _ = inputs.generate_layer(cfg, layer=2, device="cuda", q_phase=0.3)
+        pos_next = torch.full((cfg.batch,), pos, dtype=torch.int64)
+        shape = _shape(ea, cfg, n_units=cfg.batch)
+        ctx = ea.Context.for_shape(shape)
+        out = ea.compress(ctx, shape, q, k, v, pos_next.cuda(), cfg.n_future, cfg.rope_base, cfg.eps, kept)
+        ctx.sync_status()
+        if kept == n:
+            want = torch.arange(n, dtype=torch.int32, device="cuda").expand(cfg.batch, cfg.n_kv_heads, n)
+            assert torch.equal(out.kept_idx, want)
+            assert torch.equal(out.k_out.view(torch.int16), k.view(torch.int16))
+            assert torch.equal(out.v_out.view(torch.int16), v.view(torch.int16))
+        else:
+            ref = oracle.compress(inputs.bits(q), inputs.bits(k), inputs.bits(v), pos_next.numpy(), cfg.n_future,
+                                  cfg.rope_base, cfg.eps, kept)
+            own = oracle.select(out.scores.cpu().numpy().astype(np.float64), kept)
+            assert np.array_equal(out.kept_idx.cpu().numpy(), own)
+            agree = (out.kept_idx.cpu().numpy() == ref["kept_idx"]).mean()
+            assert agree > 0.99
+
+
 def test_run_to_run_bitwise_determinism(ea):
     cfg = inputs.CONFIGS[1]
     q, k, v, pos = inputs.generate_layer(cfg, device="cuda")

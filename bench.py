@@ -161,6 +161,72 @@ class Workload:
                                  self.idx[u0:u1], self.k_out[u0:u1], self.v_out[u0:u1])
 
 
+class DecodeWorkload:
+    """The streaming-decode config: one step replays the 28 compression events of a generation that
+    grows every sequence's cache from 2048 to 16384 keys in steps of 512 with a 4096-key budget
+    (inputs.decode_schedule).  Every distinct cache length has its own resident synthetic cache (all
+    28 layers x batch 8 folded into the units of one call); the window queries rotate through
+    `n_phases` slowly turning query means."""
+
+    def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4):
+        import dataclasses
+        self.cfg, self.device, self.ea = cfg, device, ea
+        self.events = inputs.decode_schedule()
+        L, B = cfg.n_layers, cfg.batch
+        U, Hq, Hkv, d, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
+        bf, f32 = torch.bfloat16, torch.float32
+        self.n_units = U
+        self.caches, self.windows = {}, []
+        for n in sorted({n for _, n, _ in self.events}):
+            k = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
+            v = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
+            for layer in range(L):
+                _, kk, vv, _ = inputs.generate_layer(dataclasses.replace(cfg, window=1), layer=layer, device=device,
+                                                     n_keys=n)
+                k[layer * B:(layer + 1) * B], v[layer * B:(layer + 1) * B] = kk, vv
+            kept = min(n, cfg.n_kept)
+            self.caches[n] = dict(
+                k=k, v=v, scores=torch.empty((U, Hkv, n), dtype=f32, device=device),
+                idx=torch.empty((U, Hkv, kept), dtype=torch.int32, device=device),
+                k_out=torch.empty((U, Hkv, kept, d), dtype=bf, device=device),
+                v_out=torch.empty((U, Hkv, kept, d), dtype=bf, device=device))
+        for ph in range(n_phases):
+            q = torch.empty((U, Hq, W, d), dtype=bf, device=device)
+            for layer in range(L):
+                qq, _, _, _ = inputs.generate_layer(cfg, layer=layer, device=device, n_keys=1,
+                                                    q_phase=2 * 3.141592653589793 / 64 * ph)
+                q[layer * B:(layer + 1) * B] = qq
+            self.windows.append(q)
+        self.pos = [torch.full((U,), pos, dtype=torch.int64, device=device) for pos, _, _ in self.events]
+        self.mu = torch.empty((U, Hq, d), dtype=f32, device=device)
+        self.sigma = torch.empty((U, Hq, d, d), dtype=f32, device=device)
+        # for the caller: the largest shape decides the workspace
+        self.k = self.caches[max(self.caches)]["k"]
+
+    def make_ctx(self, units_per_call):
+        cfg = self.cfg
+        shape = self.ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, max(self.caches),
+                                   cfg.window)
+        return self.ea.Context.for_shape(shape, self.device.index)
+
+    def step(self, ctx, units_per_call):
+        ea, cfg = self.ea, self.cfg
+        for e, (pos, n, kept) in enumerate(self.events):
+            c = self.caches[n]
+            shape = ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, n, cfg.window)
+            ea.ea_query_stats(ctx, shape, self.windows[e % len(self.windows)], self.pos[e], cfg.n_future,
+                              cfg.rope_base, self.mu, self.sigma)
+            ea.ea_score(ctx, shape, c["k"], c["v"], self.mu, self.sigma, cfg.eps, c["scores"])
+            ea.ea_select_compact(ctx, shape, c["scores"], kept, c["k"], c["v"], c["idx"], c["k_out"], c["v_out"])
+
+    def work(self):
+        cfg = self.cfg
+        per_head = self.n_units * cfg.n_kv_heads
+        slots = sum(per_head * n for _, n, _ in self.events)
+        bytes_ = slots * 4 * cfg.head_dim + sum(per_head * kept for _, _, kept in self.events) * 4 * cfg.head_dim
+        return slots, bytes_, slots * 2 * cfg.head_dim ** 2 * cfg.group
+
+
 def algorithmic_work(cfg: inputs.EAConfig):
     """Per step: key-slots, algorithmic HBM bytes (read K, read V, write kept K and V) and the
     FLOPs of the quadratic form k^T Sigma k for each query head (2 d^2 G per key-slot)."""
@@ -267,7 +333,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4])
     ap.add_argument("--units-per-call", type=int, default=0, help="layers per library call (0 = all)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: only the first N layers of the stack")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -293,10 +359,13 @@ def main():
     from paper_2510_00636_b200 import binding as ea
     ea.lib()
 
-    wl = Workload(cfg, device, ea)
-    upc = args.units_per_call or wl.n_units
+    decode = cfg.cfg_id == 4
+    wl = DecodeWorkload(cfg, device, ea) if decode else Workload(cfg, device, ea)
+    upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
-    slots, alg_bytes, alg_flops = algorithmic_work(cfg)
+    slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg)
+    if decode:
+        args.skip_e2e = True           # the host-buffer leg is defined for the prefill configs
     peaks = measured_peaks()
 
     sampler = ClockSampler(local)
@@ -324,7 +393,7 @@ def main():
     ctx.sync_status()
 
     # roofline of the dominant kernel (the log-score kernel, Eq. 7)
-    n_calls = (wl.n_units + upc - 1) // upc
+    n_calls = len(wl.events) if decode else (wl.n_units + upc - 1) // upc
     avg_score_ms = score_ms / max(1, score_launches)
     flops_per_launch = alg_flops / n_calls
     bytes_per_launch = slots * 2 * cfg.head_dim / n_calls            # the K rows this kernel must read

@@ -5,9 +5,9 @@
 // cos/sin(p * theta_m) over p = pos_next .. pos_next + T - 1, evaluated in fp64
 // with the closed form of the geometric series
 //   (1/T) sum_j e^{i theta (p+j)} = e^{i theta (p + (T-1)/2)} sin(T theta/2) / (T sin(theta/2)).
-// Kernel 2 (stats_kernel): per query head, mu_bar = R_bar mu and
+// Kernel 2 (stats_mma_kernel): per query head, mu_bar = R_bar mu and
 //   Sigma_bar = (1/N) sum_w x_w x_w^T,  x_w = R_bar (u_w - mu),
-// which equals R_bar Sigma R_bar^T.  fp32 accumulation of bf16 inputs.
+// which equals R_bar Sigma R_bar^T.  Tensor cores on a bf16 (hi, lo) pair of x, fp32 accumulation.
 #include "ea_internal.h"
 
 namespace {
@@ -29,94 +29,151 @@ __global__ void rope_coef_kernel(const int64_t* __restrict__ pos_next, int n_uni
     coef[2 * (size_t)t + 1] = (float)(sc * ratio);
 }
 
-constexpr int kStatsThreads = 256;
-constexpr int kRowBlock = 64;    // rows of Sigma_bar per CTA
-constexpr int kWChunk = 32;      // window rows staged per step
+// ---------------------------------------------------------------------------------------------
+// Sigma_bar = (1/N) X^T X with X[w] = R_bar (u_w - mu) is a
+// symmetric rank-W update; each CTA computes one BM x BM block of the upper triangle with
+// mma.sync.m16n8k16 (bf16 x bf16 -> fp32).  X is kept as a bf16 pair (hi, lo) and three products
+// (hi.hi + hi.lo + lo.hi) are accumulated, so every product carries 16 significant bits of each
+// factor; the lower triangle is a copy of the upper one, which makes the result bitwise symmetric.
+constexpr int kKC = 32;            // window rows per shared-memory chunk
+constexpr int kXtPitch = 40;       // bf16 per row of the transposed chunk: 80 bytes, conflict-free for ldmatrix
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
 template <int D>
-__global__ void __launch_bounds__(kStatsThreads)
-stats_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
-             int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar) {
+__global__ void __launch_bounds__(256)
+stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
+                 int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar) {
     constexpr int HALF = D / 2;
-    constexpr int CT = D / 32;                     // columns per thread
+    constexpr int BM = D < 128 ? D : 128;          // block edge
+    constexpr int NB1 = D / BM;                    // blocks per edge (1 or 2)
+    constexpr int WM = BM / 2, WN = BM / 4;        // warp tile: 2 x 4 warps
+    constexpr int TM = WM / 16, TN = WN / 8;       // mma tiles per warp
     __shared__ float mu_s[D];
     __shared__ float c_s[HALF], s_s[HALF];
-    __shared__ __align__(16) float x_s[kWChunk][D];
+    // [hi / lo][row: BM channels of the block's rows, then BM channels of its columns][w in chunk]
+    __shared__ __align__(16) __nv_bfloat16 xt[2][2 * BM][kXtPitch];
 
     const int uh = blockIdx.x;
     const int u = uh / Hq;
-    const int rb = blockIdx.y;
-    const int tid = threadIdx.x;
+    // blockIdx.y -> (bi <= bj)
+    const int bi = NB1 == 1 ? 0 : (blockIdx.y == 2 ? 1 : 0);
+    const int bj = NB1 == 1 ? 0 : (blockIdx.y == 0 ? 0 : 1);
+    const bool diag = bi == bj;
+    const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
     const __nv_bfloat16* q = q_win + (size_t)uh * W * D;
 
-    for (int m = tid; m < HALF; m += kStatsThreads) {
+    for (int m = tid; m < HALF; m += 256) {
         c_s[m] = coef[2 * ((size_t)u * HALF + m)];
         s_s[m] = coef[2 * ((size_t)u * HALF + m) + 1];
     }
-    for (int c = tid; c < D; c += kStatsThreads) {
+    for (int c = tid; c < D; c += 256) {
         float acc = 0.f;
         for (int w = 0; w < W; ++w) acc += __bfloat162float(q[(size_t)w * D + c]);
         mu_s[c] = acc / (float)W;
     }
     __syncthreads();
-
-    if (rb == 0) {
-        for (int m = tid; m < HALF; m += kStatsThreads) {
-            int a = layout == EA_ROPE_INTERLEAVED ? 2 * m : m;
-            int b = layout == EA_ROPE_INTERLEAVED ? 2 * m + 1 : m + HALF;
-            float ma = mu_s[a], mb = mu_s[b];
+    if (blockIdx.y == 0) {
+        for (int m = tid; m < HALF; m += 256) {
+            const int a = layout == EA_ROPE_INTERLEAVED ? 2 * m : m;
+            const int b = layout == EA_ROPE_INTERLEAVED ? 2 * m + 1 : m + HALF;
+            const float ma = mu_s[a], mb = mu_s[b];
             mu_bar[(size_t)uh * D + a] = c_s[m] * ma - s_s[m] * mb;
             mu_bar[(size_t)uh * D + b] = s_s[m] * ma + c_s[m] * mb;
         }
     }
 
-    const int ty = tid / 32, tx = tid % 32;
-    const int row0 = rb * kRowBlock + ty * 8;
-    float acc[8][CT];
+    float acc[TM][TN][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < CT; ++j) acc[i][j] = 0.f;
+        for (int j = 0; j < TN; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
 
-    for (int w0 = 0; w0 < W; w0 += kWChunk) {
-        const int rows = min(kWChunk, W - w0);
+    const int wm = warp / 4, wn = warp % 4;        // warp position in the block
+    const int n_rows = diag ? BM : 2 * BM;         // channel rows staged per chunk
+    const uint32_t xt_hi = static_cast<uint32_t>(__cvta_generic_to_shared(&xt[0][0][0]));
+    const uint32_t xt_lo = static_cast<uint32_t>(__cvta_generic_to_shared(&xt[1][0][0]));
+
+    for (int w0 = 0; w0 < W; w0 += kKC) {
         __syncthreads();
-        // stage x_w = R_bar (u_w - mu) for this chunk of window rows
-        for (int e = tid; e < kWChunk * HALF; e += kStatsThreads) {
-            int w = e / HALF, m = e % HALF;
-            int a = layout == EA_ROPE_INTERLEAVED ? 2 * m : m;
-            int b = layout == EA_ROPE_INTERLEAVED ? 2 * m + 1 : m + HALF;
-            float xa = 0.f, xb = 0.f;
-            if (w < rows) {
-                xa = __bfloat162float(q[(size_t)(w0 + w) * D + a]) - mu_s[a];
-                xb = __bfloat162float(q[(size_t)(w0 + w) * D + b]) - mu_s[b];
+        // stage x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
+        for (int e = tid; e < n_rows * kKC; e += 256) {
+            const int w = e / n_rows, r = e % n_rows;              // consecutive threads: consecutive channels
+            const int ch = (r < BM ? bi * BM : bj * BM - BM) + r;
+            float x = 0.f;
+            if (w0 + w < W) {
+                int m, partner;
+                bool first;                                         // ch is the first channel of its rotation pair
+                if (layout == EA_ROPE_INTERLEAVED) { m = ch >> 1; first = (ch & 1) == 0; partner = ch ^ 1; }
+                else { m = ch < HALF ? ch : ch - HALF; first = ch < HALF; partner = first ? ch + HALF : ch - HALF; }
+                const float xa = __bfloat162float(q[(size_t)(w0 + w) * D + ch]) - mu_s[ch];
+                const float xb = __bfloat162float(q[(size_t)(w0 + w) * D + partner]) - mu_s[partner];
+                x = first ? c_s[m] * xa - s_s[m] * xb : s_s[m] * xb + c_s[m] * xa;
             }
-            x_s[w][a] = c_s[m] * xa - s_s[m] * xb;
-            x_s[w][b] = s_s[m] * xa + c_s[m] * xb;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+            xt[0][r][w] = hi;
+            xt[1][r][w] = __float2bfloat16_rn(x - __bfloat162float(hi));
         }
         __syncthreads();
-#pragma unroll 4
-        for (int w = 0; w < kWChunk; ++w) {
-            float r[8], c[CT];
-            const float4 r0 = *reinterpret_cast<const float4*>(&x_s[w][row0]);
-            const float4 r1 = *reinterpret_cast<const float4*>(&x_s[w][row0 + 4]);
-            r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
-            r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
 #pragma unroll
-            for (int j = 0; j < CT; ++j) c[j] = x_s[w][tx + 32 * j];
+        for (int k0 = 0; k0 < kKC; k0 += 16) {
+            uint32_t a_hi[TM][4], a_lo[TM][4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < TM; ++i) {
+                const int row = wm * WM + i * 16 + (lane % 8) + 8 * ((lane / 8) % 2);
+                const uint32_t off = (uint32_t)((row * kXtPitch + k0 + 8 * (lane / 16)) * 2);
+                ldmatrix_x4(xt_hi + off, a_hi[i]);
+                ldmatrix_x4(xt_lo + off, a_lo[i]);
+            }
 #pragma unroll
-                for (int j = 0; j < CT; ++j) acc[i][j] = fmaf(r[i], c[j], acc[i][j]);
+            for (int j2 = 0; j2 < TN; j2 += 2) {
+                // two 8-channel column tiles per ldmatrix.x4
+                uint32_t b_hi[4], b_lo[4];
+                const int row = (diag ? 0 : BM) + wn * WN + j2 * 8 + (lane % 8) + 8 * (lane / 16);
+                const uint32_t off = (uint32_t)((row * kXtPitch + k0 + 8 * ((lane / 8) % 2)) * 2);
+                ldmatrix_x4(xt_hi + off, b_hi);
+                ldmatrix_x4(xt_lo + off, b_lo);
+#pragma unroll
+                for (int i = 0; i < TM; ++i)
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        mma_bf16_16816(acc[i][j2 + jj], a_hi[i], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                        mma_bf16_16816(acc[i][j2 + jj], a_hi[i], b_lo[2 * jj], b_lo[2 * jj + 1]);
+                        mma_bf16_16816(acc[i][j2 + jj], a_lo[i], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                    }
+            }
         }
     }
 
+    // upper triangle from the accumulators, lower triangle as its mirror
     float* out = sigma_bar + (size_t)uh * D * D;
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < CT; ++j)
-            out[(size_t)(row0 + i) * D + tx + 32 * j] = acc[i][j] * inv_norm;
+        for (int j = 0; j < TN; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int a = bi * BM + wm * WM + i * 16 + lane / 4 + 8 * (e / 2);
+                const int c = bj * BM + wn * WN + j * 8 + 2 * (lane % 4) + (e % 2);
+                if (a <= c) {
+                    const float v = acc[i][j][e] * inv_norm;
+                    out[(size_t)a * D + c] = v;
+                    out[(size_t)c * D + a] = v;
+                }
+            }
 }
 
 }  // namespace
@@ -130,19 +187,19 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
                                                            rope_base, rope_coef);
     const float inv_norm =
         1.0f / (float)(s.cov_norm == EA_COV_SAMPLE ? s.window - 1 : s.window);
-    dim3 grid((unsigned)(s.n_units * s.n_q_heads), (unsigned)(d / kRowBlock));
+    const unsigned heads = (unsigned)(s.n_units * s.n_q_heads);
     switch (d) {
         case 64:
-            stats_kernel<64><<<grid, kStatsThreads, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
-                                                            s.rope_layout, inv_norm, mu_bar, sigma_bar);
+            stats_mma_kernel<64><<<dim3(heads, 1), 256, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
+                                                                s.rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 128:
-            stats_kernel<128><<<grid, kStatsThreads, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
-                                                             s.rope_layout, inv_norm, mu_bar, sigma_bar);
+            stats_mma_kernel<128><<<dim3(heads, 1), 256, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
+                                                                 s.rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 256:
-            stats_kernel<256><<<grid, kStatsThreads, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
-                                                             s.rope_layout, inv_norm, mu_bar, sigma_bar);
+            stats_mma_kernel<256><<<dim3(heads, 3), 256, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
+                                                                 s.rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         default:
             return EA_ERR_UNSUPPORTED;
@@ -216,19 +273,19 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
     rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, stream>>>(pos_next, s->n_units, half, d, n_future,
                                                                rope_base, coef);
     const float inv_norm = 1.0f / (float)(s->cov_norm == EA_COV_SAMPLE ? s->window - 1 : s->window);
-    dim3 grid((unsigned)(s->n_units * s->n_q_heads), (unsigned)(d / kRowBlock));
+    const unsigned heads = (unsigned)(s->n_units * s->n_q_heads);
     switch (d) {
         case 64:
-            stats_kernel<64><<<grid, kStatsThreads, 0, stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                 s->rope_layout, inv_norm, mu_bar, sigma_bar);
+            stats_mma_kernel<64><<<dim3(heads, 1), 256, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+                                                                    s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 128:
-            stats_kernel<128><<<grid, kStatsThreads, 0, stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                  s->rope_layout, inv_norm, mu_bar, sigma_bar);
+            stats_mma_kernel<128><<<dim3(heads, 1), 256, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         default:
-            stats_kernel<256><<<grid, kStatsThreads, 0, stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                  s->rope_layout, inv_norm, mu_bar, sigma_bar);
+            stats_mma_kernel<256><<<dim3(heads, 3), 256, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
     }
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;

@@ -52,6 +52,12 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
 }
 
 template <int D>
+constexpr int stats_smem_bytes() {
+    constexpr int BM = D < 128 ? D : 128;
+    return 2 * 2 * BM * kXtPitch * 2 + kKC * D * 2 + (D + D) * 4 + (256 / (D / 2)) * D * 4;
+}
+
+template <int D>
 __global__ void __launch_bounds__(256)
 stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
                  int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar) {
@@ -60,10 +66,17 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
     constexpr int NB1 = D / BM;                    // blocks per edge (1 or 2)
     constexpr int WM = BM / 2, WN = BM / 4;        // warp tile: 2 x 4 warps
     constexpr int TM = WM / 16, TN = WN / 8;       // mma tiles per warp
-    __shared__ float mu_s[D];
-    __shared__ float c_s[HALF], s_s[HALF];
+    // dynamic shared memory: the transposed (hi, lo) chunk, the raw window chunk, the mean, R_bar
+    extern __shared__ __align__(16) unsigned char stats_smem[];
     // [hi / lo][row: BM channels of the block's rows, then BM channels of its columns][w in chunk]
-    __shared__ __align__(16) __nv_bfloat16 xt[2][2 * BM][kXtPitch];
+    typedef __nv_bfloat16 (*xt_t)[2 * BM][kXtPitch];
+    xt_t xt = reinterpret_cast<xt_t>(stats_smem);
+    constexpr int kXtBytes = 2 * 2 * BM * kXtPitch * 2;
+    __nv_bfloat16* raw = reinterpret_cast<__nv_bfloat16*>(stats_smem + kXtBytes);          // [kKC][D]
+    float* mu_s = reinterpret_cast<float*>(stats_smem + kXtBytes + kKC * D * 2);           // [D]
+    float* c_s = mu_s + D;                                                                  // [HALF]
+    float* s_s = c_s + HALF;                                                                // [HALF]
+    float* red = s_s + HALF;                                                                // [256 / (D/2)][D]
 
     const int uh = blockIdx.x;
     const int u = uh / Hq;
@@ -78,10 +91,26 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
         c_s[m] = coef[2 * ((size_t)u * HALF + m)];
         s_s[m] = coef[2 * ((size_t)u * HALF + m) + 1];
     }
-    for (int c = tid; c < D; c += 256) {
-        float acc = 0.f;
-        for (int w = 0; w < W; ++w) acc += __bfloat162float(q[(size_t)w * D + c]);
-        mu_s[c] = acc / (float)W;
+    {   // mean: thread = (group of window rows, channel pair); groups meet in shared memory
+        constexpr int NG = 256 / HALF;
+        const int cp = tid % HALF, g = tid / HALF;
+        float a0 = 0.f, a1 = 0.f;
+        const uint32_t* q2 = reinterpret_cast<const uint32_t*>(q);
+#pragma unroll 4
+        for (int w = g; w < W; w += NG) {
+            const uint32_t x = __ldg(q2 + (size_t)w * HALF + cp);
+            a0 += __uint_as_float(x << 16);
+            a1 += __uint_as_float(x & 0xffff0000u);
+        }
+        red[g * D + 2 * cp] = a0;
+        red[g * D + 2 * cp + 1] = a1;
+        __syncthreads();
+        for (int c = tid; c < D; c += 256) {
+            float acc = 0.f;
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) acc += red[gg * D + c];      // fixed order
+            mu_s[c] = acc / (float)W;
+        }
     }
     __syncthreads();
     if (blockIdx.y == 0) {
@@ -106,10 +135,18 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
     const int n_rows = diag ? BM : 2 * BM;         // channel rows staged per chunk
     const uint32_t xt_hi = static_cast<uint32_t>(__cvta_generic_to_shared(&xt[0][0][0]));
     const uint32_t xt_lo = static_cast<uint32_t>(__cvta_generic_to_shared(&xt[1][0][0]));
+    const uint4* q4 = reinterpret_cast<const uint4*>(q);
+    uint4* raw4 = reinterpret_cast<uint4*>(raw);
 
     for (int w0 = 0; w0 < W; w0 += kKC) {
         __syncthreads();
-        // stage x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
+        // the raw chunk with 128-bit loads (rows past the window read as zero) ...
+        for (int e = tid; e < kKC * D / 8; e += 256) {
+            const int w = e / (D / 8);
+            raw4[e] = w0 + w < W ? __ldg(q4 + (size_t)w0 * (D / 8) + e) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncthreads();
+        // ... then x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
         for (int e = tid; e < n_rows * kKC; e += 256) {
             const int w = e / n_rows, r = e % n_rows;              // consecutive threads: consecutive channels
             const int ch = (r < BM ? bi * BM : bj * BM - BM) + r;
@@ -119,8 +156,8 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
                 bool first;                                         // ch is the first channel of its rotation pair
                 if (layout == EA_ROPE_INTERLEAVED) { m = ch >> 1; first = (ch & 1) == 0; partner = ch ^ 1; }
                 else { m = ch < HALF ? ch : ch - HALF; first = ch < HALF; partner = first ? ch + HALF : ch - HALF; }
-                const float xa = __bfloat162float(q[(size_t)(w0 + w) * D + ch]) - mu_s[ch];
-                const float xb = __bfloat162float(q[(size_t)(w0 + w) * D + partner]) - mu_s[partner];
+                const float xa = __bfloat162float(raw[w * D + ch]) - mu_s[ch];
+                const float xb = __bfloat162float(raw[w * D + partner]) - mu_s[partner];
                 x = first ? c_s[m] * xa - s_s[m] * xb : s_s[m] * xb + c_s[m] * xa;
             }
             const __nv_bfloat16 hi = __float2bfloat16_rn(x);
@@ -190,15 +227,21 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
     const unsigned heads = (unsigned)(s.n_units * s.n_q_heads);
     switch (d) {
         case 64:
-            stats_mma_kernel<64><<<dim3(heads, 1), 256, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
+            stats_mma_kernel<64><<<dim3(heads, 1), 256, stats_smem_bytes<64>(), st>>>(q_win, rope_coef, s.n_q_heads, s.window,
                                                                 s.rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 128:
-            stats_mma_kernel<128><<<dim3(heads, 1), 256, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
+            if (cudaFuncSetAttribute(stats_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     stats_smem_bytes<128>()) != cudaSuccess)
+                return EA_ERR_CUDA;
+            stats_mma_kernel<128><<<dim3(heads, 1), 256, stats_smem_bytes<128>(), st>>>(q_win, rope_coef, s.n_q_heads, s.window,
                                                                  s.rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 256:
-            stats_mma_kernel<256><<<dim3(heads, 3), 256, 0, st>>>(q_win, rope_coef, s.n_q_heads, s.window,
+            if (cudaFuncSetAttribute(stats_mma_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     stats_smem_bytes<256>()) != cudaSuccess)
+                return EA_ERR_CUDA;
+            stats_mma_kernel<256><<<dim3(heads, 3), 256, stats_smem_bytes<256>(), st>>>(q_win, rope_coef, s.n_q_heads, s.window,
                                                                  s.rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         default:
@@ -276,15 +319,21 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
     const unsigned heads = (unsigned)(s->n_units * s->n_q_heads);
     switch (d) {
         case 64:
-            stats_mma_kernel<64><<<dim3(heads, 1), 256, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+            stats_mma_kernel<64><<<dim3(heads, 1), 256, stats_smem_bytes<64>(), stream>>>(q, coef, s->n_q_heads, s->window,
                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 128:
-            stats_mma_kernel<128><<<dim3(heads, 1), 256, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+            if (cudaFuncSetAttribute(stats_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     stats_smem_bytes<128>()) != cudaSuccess)
+                return EA_ERR_CUDA;
+            stats_mma_kernel<128><<<dim3(heads, 1), 256, stats_smem_bytes<128>(), stream>>>(q, coef, s->n_q_heads, s->window,
                                                                      s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         default:
-            stats_mma_kernel<256><<<dim3(heads, 3), 256, 0, stream>>>(q, coef, s->n_q_heads, s->window,
+            if (cudaFuncSetAttribute(stats_mma_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     stats_smem_bytes<256>()) != cudaSuccess)
+                return EA_ERR_CUDA;
+            stats_mma_kernel<256><<<dim3(heads, 3), 256, stats_smem_bytes<256>(), stream>>>(q, coef, s->n_q_heads, s->window,
                                                                      s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
     }

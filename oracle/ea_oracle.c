@@ -293,6 +293,96 @@ void eao_gather(const uint16_t *rows, const int32_t *idx, int64_t n_heads, int64
                 out[(h * n_kept + j) * d + c] = rows[(h * n + idx[h * n_kept + j]) * d + c];
 }
 
+/*
+ * Head-adaptive eviction (the head-adaptive paragraph of Sec. 2.2, which adopts the
+ * per-layer budget allocation of Ada-KV; the paper prints no formula, so the rule is
+ * the published one: a safeguard share per head, the rest of the layer's budget to the
+ * best remaining pairs of the layer whichever head they belong to).
+ *
+ * One unit = one layer of one sequence with Hkv heads of n keys.  Its budget is
+ * Hkv * n_kept pairs.
+ *   1. Safeguard: every head keeps its n_floor best keys
+ *      (order: score descending, index ascending).
+ *   2. The other Hkv * (n_kept - n_floor) places go to the best pairs not kept in
+ *      step 1, over all heads of the unit
+ *      (order: score descending, head ascending, index ascending).
+ *   3. The kept indices of a head are reported ascending; heads are concatenated in
+ *      head order: idx[u][offsets[u][g] .. offsets[u][g+1]) belongs to head g.
+ * score: [n_units, Hkv, n]; idx: [n_units, Hkv * n_kept]; offsets: [n_units, Hkv + 1].
+ * Needs 0 <= n_floor <= n_kept <= n.
+ */
+typedef struct { double score; int32_t head; int32_t idx; } eao_pair;
+
+static int pair_cmp(const void *pa, const void *pb) {
+    const eao_pair *a = (const eao_pair *)pa, *b = (const eao_pair *)pb;
+    if (a->score > b->score) return -1;
+    if (a->score < b->score) return 1;
+    if (a->head != b->head) return (a->head > b->head) - (a->head < b->head);
+    return (a->idx > b->idx) - (a->idx < b->idx);
+}
+
+void eao_select_adaptive(const double *score, int64_t n_units, int64_t Hkv, int64_t n, int64_t n_kept,
+                         int64_t n_floor, int32_t *idx, int32_t *offsets) {
+    const int64_t budget = Hkv * n_kept;
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t u = 0; u < n_units; ++u) {
+        const double *sc = score + u * Hkv * n;
+        char *kept = (char *)calloc((size_t)(Hkv * n > 0 ? Hkv * n : 1), 1);
+        eao_item *items = (eao_item *)malloc((size_t)(n > 0 ? n : 1) * sizeof(eao_item));
+        eao_pair *rest = (eao_pair *)malloc((size_t)(Hkv * n > 0 ? Hkv * n : 1) * sizeof(eao_pair));
+        /* step 1: the safeguard share of every head */
+        for (int64_t g = 0; g < Hkv; ++g) {
+            for (int64_t i = 0; i < n; ++i) { items[i].score = sc[g * n + i]; items[i].idx = (int32_t)i; }
+            qsort(items, (size_t)n, sizeof(eao_item), item_cmp);
+            for (int64_t j = 0; j < n_floor; ++j) kept[g * n + items[j].idx] = 1;
+        }
+        /* step 2: the rest of the budget over the whole unit */
+        int64_t n_rest = 0;
+        for (int64_t g = 0; g < Hkv; ++g)
+            for (int64_t i = 0; i < n; ++i)
+                if (!kept[g * n + i]) {
+                    rest[n_rest].score = sc[g * n + i];
+                    rest[n_rest].head = (int32_t)g;
+                    rest[n_rest].idx = (int32_t)i;
+                    ++n_rest;
+                }
+        qsort(rest, (size_t)n_rest, sizeof(eao_pair), pair_cmp);
+        const int64_t places = budget - Hkv * n_floor;
+        for (int64_t j = 0; j < places; ++j) kept[(int64_t)rest[j].head * n + rest[j].idx] = 1;
+        /* step 3: ascending indices per head, heads in order */
+        int32_t *out = idx + u * budget, *off = offsets + u * (Hkv + 1);
+        int64_t pos = 0;
+        for (int64_t g = 0; g < Hkv; ++g) {
+            off[g] = (int32_t)pos;
+            for (int64_t i = 0; i < n; ++i)
+                if (kept[g * n + i]) out[pos++] = (int32_t)i;
+        }
+        off[Hkv] = (int32_t)pos;
+        free(rest);
+        free(items);
+        free(kept);
+    }
+}
+
+/* Ragged compaction: out[u][j][:] = rows[u][g][idx[u][j]][:] with g the head whose range holds j. */
+void eao_gather_adaptive(const uint16_t *rows, const int32_t *idx, const int32_t *offsets, int64_t n_units,
+                         int64_t Hkv, int64_t n, int64_t budget, int d, uint16_t *out) {
+    for (int64_t u = 0; u < n_units; ++u)
+        for (int64_t g = 0; g < Hkv; ++g)
+            for (int64_t j = offsets[u * (Hkv + 1) + g]; j < offsets[u * (Hkv + 1) + g + 1]; ++j)
+                for (int c = 0; c < d; ++c)
+                    out[(u * budget + j) * d + c] = rows[((u * Hkv + g) * n + idx[u * budget + j]) * d + c];
+}
+
+/* Safeguard share floor(alpha * n_kept), evaluated in double. */
+int64_t eao_n_floor(int64_t n_kept, double alpha) {
+    double x = (double)n_kept * alpha;
+    int64_t k = (int64_t)x;
+    if (k < 0) k = 0;
+    if (k > n_kept) k = n_kept;
+    return k;
+}
+
 /* int(n * (1 - r)) evaluated in double, as the listing computes n_kept. */
 int64_t eao_n_kept(int64_t n, double compression_ratio) {
     double x = (double)n * (1.0 - compression_ratio);

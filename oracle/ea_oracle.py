@@ -58,9 +58,13 @@ def _load():
         lib.eao_gather.argtypes = [vp, vp, i64, i64, i64, i32, vp]
         lib.eao_n_kept.argtypes = [i64, f64]
         lib.eao_n_kept.restype = i64
+        lib.eao_select_adaptive.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp]
+        lib.eao_gather_adaptive.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp]
+        lib.eao_n_floor.argtypes = [i64, f64]
+        lib.eao_n_floor.restype = i64
         for name in ("eao_set_num_threads", "eao_mean_cov", "eao_rope_average",
                      "eao_apply_rope_average", "eao_logits", "eao_scores", "eao_select",
-                     "eao_gather"):
+                     "eao_gather", "eao_select_adaptive", "eao_gather_adaptive"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -175,6 +179,38 @@ def gather(rows_bits, idx):
     out = np.empty((nh, nk, d), np.uint16)
     _load().eao_gather(_p(rows), _p(idx), nh, n, nk, d, _p(out))
     return out.reshape(*lead, nk, d)
+
+
+def n_floor(n_kept_: int, alpha: float) -> int:
+    return int(_load().eao_n_floor(int(n_kept_), float(alpha)))
+
+
+def select_adaptive(score, n_kept_, n_floor_):
+    """score [U, Hkv, n] -> (idx int32 [U, Hkv * n_kept], offsets int32 [U, Hkv + 1]).
+
+    Head-adaptive eviction: each head keeps its n_floor best keys, the rest of the unit's budget of
+    Hkv * n_kept goes to the best remaining pairs of the unit.
+    """
+    sc = _c(score, np.float64)
+    U, Hkv, n = sc.shape
+    if not 0 <= int(n_floor_) <= int(n_kept_) <= n:
+        raise ValueError("need 0 <= n_floor <= n_kept <= n")
+    idx = np.empty((U, Hkv * int(n_kept_)), np.int32)
+    off = np.empty((U, Hkv + 1), np.int32)
+    _load().eao_select_adaptive(_p(sc), U, Hkv, n, int(n_kept_), int(n_floor_), _p(idx), _p(off))
+    return idx, off
+
+
+def gather_adaptive(rows_bits, idx, offsets):
+    """rows_bits uint16 [U, Hkv, n, d]; idx [U, B]; offsets [U, Hkv + 1] -> uint16 [U, B, d]."""
+    rows = _c(rows_bits, np.uint16)
+    idx = _c(idx, np.int32)
+    off = _c(offsets, np.int32)
+    U, Hkv, n, d = rows.shape
+    B = idx.shape[1]
+    out = np.empty((U, B, d), np.uint16)
+    _load().eao_gather_adaptive(_p(rows), _p(idx), _p(off), U, Hkv, n, B, d, _p(out))
+    return out
 
 
 def compress(q_win_bits, k_bits, v_bits, pos_next, n_future, rope_base, eps, n_kept_,

@@ -278,6 +278,113 @@ def test_gather(oracle):
     assert np.array_equal(out, np.take_along_axis(rows, idx[..., None].astype(np.int64), axis=2))
 
 
+# ---------------------------------------------------------------- head-adaptive selection
+def _per_head(idx, off, u):
+    return [list(idx[u, off[u, g]:off[u, g + 1]]) for g in range(off.shape[1] - 1)]
+
+
+def test_adaptive_select_brute_force(oracle):
+    """The kept set maximises the total score over all sets of the unit's budget that hold at least
+    n_floor keys of every head (distinct scores: the maximiser is unique)."""
+    rng = np.random.default_rng(21)
+    for Hkv, n, kept, floor in [(2, 5, 2, 1), (2, 5, 3, 0), (3, 4, 2, 1), (2, 6, 3, 3), (3, 4, 1, 0), (2, 6, 4, 2)]:
+        sc = rng.random(size=(2, Hkv, n))
+        idx, off = oracle.select_adaptive(sc, kept, floor)
+        B = Hkv * kept
+        assert idx.shape == (2, B) and off.shape == (2, Hkv + 1)
+        for u in range(2):
+            flat = sc[u].reshape(-1)
+            best, best_sum = None, -1.0
+            for c in itertools.combinations(range(Hkv * n), B):
+                per_head = np.bincount(np.asarray(c) // n, minlength=Hkv)
+                if per_head.min() < floor:
+                    continue
+                tot = flat[list(c)].sum()
+                if tot > best_sum:
+                    best, best_sum = c, tot
+            got = [g * n + i for g, lst in enumerate(_per_head(idx, off, u)) for i in lst]
+            assert got == sorted(best)
+            assert off[u, 0] == 0 and off[u, -1] == B
+
+
+def test_adaptive_select_limits_reduce_to_library_routines(oracle):
+    rng = np.random.default_rng(22)
+    U, Hkv, n, kept = 3, 4, 50, 13
+    sc = rng.random(size=(U, Hkv, n))
+    # safeguard = whole budget: plain per-head selection
+    idx, off = oracle.select_adaptive(sc, kept, kept)
+    assert np.array_equal(off, np.tile(np.arange(Hkv + 1) * kept, (U, 1)))
+    assert np.array_equal(idx.reshape(U, Hkv, kept), oracle.select(sc, kept))
+    # no safeguard: the Hkv * kept largest of the flattened unit (numpy's sort as the library routine)
+    idx, off = oracle.select_adaptive(sc, kept, 0)
+    for u in range(U):
+        top = np.sort(np.argsort(-sc[u].reshape(-1), kind="stable")[: Hkv * kept])
+        got = [g * n + i for g, lst in enumerate(_per_head(idx, off, u)) for i in lst]
+        assert got == list(top)
+
+
+def test_adaptive_select_ties_go_to_the_lower_head_then_index(oracle):
+    # all scores equal: the safeguard takes the first n_floor keys of every head, the other places go
+    # to head 0 until it is full, then head 1, ...
+    Hkv, n, kept, floor = 3, 6, 3, 1
+    idx, off = oracle.select_adaptive(np.ones((1, Hkv, n)), kept, floor)
+    assert _per_head(idx, off, 0) == [[0, 1, 2, 3, 4, 5], [0, 1], [0]]
+    # one tie across heads at the threshold
+    sc = np.array([[[5.0, 1.0, 3.0, 0.0], [4.0, 3.0, 0.5, 3.0]]])
+    idx, off = oracle.select_adaptive(sc, 2, 1)           # budget 4: 5, 4 (safeguards), then 3 (head 0), 3 (head 1, idx 1)
+    assert _per_head(idx, off, 0) == [[0, 2], [0, 1]]
+    idx, off = oracle.select_adaptive(sc, 2, 0)           # no safeguard: 5, 4, 3 (head 0), 3 (head 1, idx 1)
+    assert _per_head(idx, off, 0) == [[0, 2], [0, 1]]
+
+
+def test_adaptive_select_invariants(oracle):
+    rng = np.random.default_rng(23)
+    U, Hkv, n, kept, floor = 2, 4, 200, 30, 10
+    plain = rng.random(size=(U, Hkv, n))
+    skewed = plain.copy()
+    skewed[:, 1] *= 10.0                                 # one head matters far more than the others
+    for sc in (plain, skewed):
+        idx, off = oracle.select_adaptive(sc, kept, floor)
+        for u in range(U):
+            heads = _per_head(idx, off, u)
+            sizes = [len(h) for h in heads]
+            assert sum(sizes) == Hkv * kept and min(sizes) >= floor
+            if sc is skewed:
+                # about 170 keys of the strong head beat every key of the others: it takes every free place
+                assert sizes == [floor, floor + Hkv * (kept - floor), floor, floor]
+            else:
+                assert max(sizes) > kept > min(sizes)     # the budget really moves between heads
+            beyond_floor_min, dropped_max = np.inf, -np.inf
+            for g, lst in enumerate(heads):
+                assert lst == sorted(set(lst))
+                # within a head the kept keys are its best ones
+                assert lst == list(oracle.select(sc[u, g][None], len(lst))[0])
+                order = np.sort(sc[u, g])[::-1]
+                if len(lst) > floor:
+                    beyond_floor_min = min(beyond_floor_min, order[len(lst) - 1])
+                if len(lst) < n:
+                    dropped_max = max(dropped_max, order[max(len(lst), floor)])
+            # one threshold for the whole unit separates what was kept beyond the safeguard from what was dropped
+            assert beyond_floor_min >= dropped_max
+        # scaling every score of the unit by a positive constant changes nothing
+        idx2, off2 = oracle.select_adaptive(sc * 3.0, kept, floor)
+        assert np.array_equal(idx, idx2) and np.array_equal(off, off2)
+
+
+def test_adaptive_gather_and_floor(oracle):
+    rng = np.random.default_rng(24)
+    U, Hkv, n, d, kept, floor = 2, 3, 9, 4, 4, 1
+    rows = rng.integers(0, 65535, size=(U, Hkv, n, d), dtype=np.uint16)
+    sc = rng.random(size=(U, Hkv, n))
+    idx, off = oracle.select_adaptive(sc, kept, floor)
+    out = oracle.gather_adaptive(rows, idx, off)
+    for u in range(U):
+        want = np.concatenate([rows[u, g][lst] for g, lst in enumerate(_per_head(idx, off, u))])
+        assert np.array_equal(out[u], want)
+    assert oracle.n_floor(4096, 0.2) == 819 and oracle.n_floor(256, 0.2) == 51
+    assert oracle.n_floor(10, 0.0) == 0 and oracle.n_floor(10, 1.0) == 10
+
+
 def test_n_kept_is_truncated_product(oracle):
     assert oracle.n_kept(512, 0.5) == 256
     assert oracle.n_kept(8192, 0.5) == 4096

@@ -119,8 +119,9 @@ class ClockSampler:
 class Workload:
     """All layers of one config resident in HBM, plus preallocated outputs."""
 
-    def __init__(self, cfg: inputs.EAConfig, device, ea):
+    def __init__(self, cfg: inputs.EAConfig, device, ea, safeguard=None):
         self.cfg, self.device, self.ea = cfg, device, ea
+        self.safeguard = safeguard          # None: n_kept per head; else head-adaptive with this safeguard share
         L, B = cfg.n_layers, cfg.batch
         U, Hq, Hkv, d, n, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window
         bf, f32 = torch.bfloat16, torch.float32
@@ -139,6 +140,7 @@ class Workload:
         self.idx = torch.empty((U, Hkv, cfg.n_kept), dtype=torch.int32, device=device)
         self.k_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
         self.v_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
+        self.head_off = torch.empty((U, Hkv + 1), dtype=torch.int32, device=device)
         self.n_units = U
 
     def make_ctx(self, units_per_call):
@@ -157,8 +159,15 @@ class Workload:
                               self.mu[u0:u1], self.sigma[u0:u1])
             ea.ea_score(ctx, shape, self.k[u0:u1], self.v[u0:u1], self.mu[u0:u1], self.sigma[u0:u1], cfg.eps,
                         self.scores[u0:u1])
-            ea.ea_select_compact(ctx, shape, self.scores[u0:u1], cfg.n_kept, self.k[u0:u1], self.v[u0:u1],
-                                 self.idx[u0:u1], self.k_out[u0:u1], self.v_out[u0:u1])
+            if self.safeguard is None:
+                ea.ea_select_compact(ctx, shape, self.scores[u0:u1], cfg.n_kept, self.k[u0:u1], self.v[u0:u1],
+                                     self.idx[u0:u1], self.k_out[u0:u1], self.v_out[u0:u1])
+            else:
+                # same output bytes, ragged over the heads of a layer
+                ea.ea_select_compact_adaptive(ctx, shape, self.scores[u0:u1], cfg.n_kept,
+                                              ea.ea_n_floor(cfg.n_kept, self.safeguard), self.k[u0:u1],
+                                              self.v[u0:u1], self.idx[u0:u1], self.head_off[u0:u1],
+                                              self.k_out[u0:u1], self.v_out[u0:u1])
 
 
 class DecodeWorkload:
@@ -336,6 +345,9 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4])
     ap.add_argument("--units-per-call", type=int, default=0, help="layers per library call (0 = all)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: only the first N layers of the stack")
+    ap.add_argument("--head-adaptive", type=float, default=None, metavar="SAFEGUARD",
+                    help="prefill configs: head-adaptive eviction with this safeguard share (e.g. 0.2) in place of "
+                         "n_kept per head; the device-resident line only")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -360,10 +372,14 @@ def main():
     ea.lib()
 
     decode = cfg.cfg_id == 4
-    wl = DecodeWorkload(cfg, device, ea) if decode else Workload(cfg, device, ea)
+    if args.head_adaptive is not None and decode:
+        raise SystemExit("--head-adaptive applies to the prefill configs")
+    wl = DecodeWorkload(cfg, device, ea) if decode else Workload(cfg, device, ea, args.head_adaptive)
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
     slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg)
+    if args.head_adaptive is not None:
+        args.skip_e2e = True           # the host-buffer entry point evicts n_kept per head
     if decode:
         args.skip_e2e = True           # the host-buffer leg is defined for the prefill configs
     peaks = measured_peaks()
@@ -425,6 +441,8 @@ def main():
         "config": {"workload": cfg.name, "layers": cfg.n_layers, "batch": cfg.batch,
                    "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                    "n_keys": cfg.n_keys, "window": cfg.window, "n_kept": cfg.n_kept,
+                   "eviction": "n_kept per head" if args.head_adaptive is None else
+                               "head-adaptive, safeguard share %g" % args.head_adaptive,
                    "key_slots_per_step": slots, "units_per_call": upc, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (K+V %.1f GB per step)" % (slots * 4 * cfg.head_dim / 1e9)},
         "ms_per_128k_compression": ms if cfg.cfg_id == 3 else None,

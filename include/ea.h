@@ -203,6 +203,45 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
                             void* k_out, void* v_out, void* cuda_stream);
 
 /*
+ * Head-adaptive eviction and compaction (the "Head-Adaptive Compression"
+ * paragraph of Sec. 2.2: the per-layer budget allocation of Ada-KV, so that
+ * heads whose pairs matter more retain more of them).  The paper prints no
+ * formula; the rule is the published one with its safeguard:
+ *
+ *   A unit (one layer of one sequence) has a budget of Hkv * n_kept pairs.
+ *   1. Every head keeps its n_floor best pairs (score descending, index
+ *      ascending).
+ *   2. The other Hkv * (n_kept - n_floor) places go to the best pairs not yet
+ *      kept, over all heads of the unit (score descending, then head
+ *      ascending, then index ascending).
+ *   3. The kept indices of a head are emitted ascending, heads one after the
+ *      other: kept_idx[u][head_offsets[u][g] .. head_offsets[u][g+1]) belongs
+ *      to head g, and K/V rows are gathered in that order.
+ *
+ * n_floor == n_kept gives the result of ea_select_compact; n_floor == 0 is
+ * one top-(Hkv * n_kept) over the unit.  ea_n_floor gives the safeguard share
+ * floor(safeguard * n_kept) (the published default safeguard is 0.2).
+ *
+ * scores       fp32 [n_units, Hkv, n] (any finite values; -0 is treated as +0)
+ * n_kept       0 <= n_kept <= n_keys; n_floor: 0 <= n_floor <= n_kept;
+ *              Hkv * n_kept < 2^31 (EA_ERR_INVALID_ARG otherwise)
+ * k, v         bf16 [n_units, Hkv, n, d], 16-byte aligned
+ * kept_idx     int32 [n_units, Hkv * n_kept]       (output; key index within its head)
+ * head_offsets int32 [n_units, Hkv + 1]            (output; first is 0, last is Hkv * n_kept)
+ * k_out,v_out  bf16 [n_units, Hkv * n_kept, d]     (output; must not overlap k, v)
+ *              k_out/v_out may both be NULL to skip the gather.
+ * Uses the context's workspace (EA_ERR_WORKSPACE if smaller than
+ * ea_workspace_bytes(shape)).
+ */
+ea_status ea_select_compact_adaptive(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                                     int32_t n_kept, int32_t n_floor, const void* k, const void* v,
+                                     int32_t* kept_idx, int32_t* head_offsets, void* k_out,
+                                     void* v_out, void* cuda_stream);
+
+/* floor(safeguard * n_kept) evaluated in double, clamped to [0, n_kept]. */
+int64_t ea_n_floor(int64_t n_kept, double safeguard);
+
+/*
  * Synchronises cuda_stream and returns the device-side status recorded since
  * the last call of this function (EA_OK, EA_ERR_DEVICE_TIMEOUT, or
  * EA_ERR_CUDA if the stream reports an error), then clears it.

@@ -24,6 +24,7 @@ EXPORTS = (
     "ea_version", "ea_status_string", "ea_workspace_bytes", "ea_n_kept", "ea_create", "ea_destroy",
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
+    "ea_select_compact_adaptive", "ea_n_floor",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -68,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.ea_query_stats_static.restype = ctypes.c_int
         L.ea_score.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
         L.ea_select_compact.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp]
+        L.ea_select_compact_adaptive.argtypes = [vp, sp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.ea_n_floor.argtypes = [i64, f64]
+        L.ea_n_floor.restype = i64
         L.ea_sync_status.argtypes = [vp, vp]
         L.ea_host_workspace_bytes.argtypes = [sp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         L.ea_compress_host.argtypes = [vp, sp, vp, vp, vp, vp, i32, f64, f32, i32, i32, vp, vp, vp, vp, vp]
@@ -75,7 +79,7 @@ def lib() -> ctypes.CDLL:
         L.ea_profile_end.argtypes = [vp, vp, ctypes.POINTER(f64), ctypes.POINTER(i64), ctypes.POINTER(i64)]
         for name in ("ea_workspace_bytes", "ea_create", "ea_destroy", "ea_query_stats", "ea_score",
                      "ea_select_compact", "ea_sync_status", "ea_profile_begin", "ea_profile_end",
-                     "ea_host_workspace_bytes", "ea_compress_host"):
+                     "ea_host_workspace_bytes", "ea_compress_host", "ea_select_compact_adaptive"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -88,6 +92,10 @@ def _check(status: int, where: str):
 
 def ea_n_kept(n_keys: int, compression_ratio: float) -> int:
     return int(lib().ea_n_kept(int(n_keys), float(compression_ratio)))
+
+
+def ea_n_floor(n_kept: int, safeguard: float) -> int:
+    return int(lib().ea_n_floor(int(n_kept), float(safeguard)))
 
 
 def ea_workspace_bytes(shape: Shape) -> int:
@@ -226,6 +234,30 @@ def ea_select_compact(ctx: Context, shape: Shape, scores, n_kept: int, k=None, v
                                    _ptr(v), _ptr(kept_idx), _ptr(k_out), _ptr(v_out),
                                    _stream(ctx.device)), "ea_select_compact")
     return kept_idx, k_out, v_out
+
+
+def ea_select_compact_adaptive(ctx: Context, shape: Shape, scores, n_kept: int, n_floor: int, k=None, v=None,
+                               kept_idx=None, head_offsets=None, k_out=None, v_out=None, gather: bool = True):
+    """scores fp32 [U,Hkv,n] -> (kept_idx int32 [U,Hkv*n_kept], head_offsets int32 [U,Hkv+1],
+    k_out, v_out bf16 [U,Hkv*n_kept,d]); head g of unit u owns kept_idx[u, off[u,g]:off[u,g+1]]."""
+    _dev_tensor(scores, torch.float32, "scores")
+    U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
+    B = Hkv * max(n_kept, 0)
+    if kept_idx is None:
+        kept_idx = torch.empty((U, B), dtype=torch.int32, device=scores.device)
+    if head_offsets is None:
+        head_offsets = torch.empty((U, Hkv + 1), dtype=torch.int32, device=scores.device)
+    if gather:
+        _dev_tensor(k, torch.bfloat16, "k")
+        _dev_tensor(v, torch.bfloat16, "v")
+        if k_out is None:
+            k_out = torch.empty((U, B, d), dtype=torch.bfloat16, device=scores.device)
+        if v_out is None:
+            v_out = torch.empty((U, B, d), dtype=torch.bfloat16, device=scores.device)
+    _check(lib().ea_select_compact_adaptive(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), int(n_floor),
+                                            _ptr(k), _ptr(v), _ptr(kept_idx), _ptr(head_offsets), _ptr(k_out),
+                                            _ptr(v_out), _stream(ctx.device)), "ea_select_compact_adaptive")
+    return kept_idx, head_offsets, k_out, v_out
 
 
 @dataclass

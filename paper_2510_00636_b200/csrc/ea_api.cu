@@ -38,6 +38,7 @@ ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     p.image = off;      off = ea_align_up(off + (mma ? ea_mma_image_bytes(s) : 0), 1024);
     p.vec = off;        off = ea_align_up(off + (mma ? ea_mma_vec_bytes(s) : 0), 256);
     p.lse_part = off;   off = ea_align_up(off + (mma ? ea_mma_lse_part_bytes(s) : 0), 256);
+    p.adaptive = off;   off = ea_align_up(off + ea_adaptive_ws_bytes(s), 256);
     p.total = off;
     return p;
 }
@@ -257,6 +258,57 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
                               static_cast<__nv_bfloat16*>(v_out), stream);
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
+}
+
+ea_status ea_select_compact_adaptive(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                                     int32_t n_kept, int32_t n_floor, const void* k, const void* v,
+                                     int32_t* kept_idx, int32_t* head_offsets, void* k_out, void* v_out,
+                                     void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (n_kept < 0 || n_kept > shape->n_keys || n_floor < 0 || n_floor > n_kept) return EA_ERR_INVALID_ARG;
+    if ((long long)shape->n_kv_heads * n_kept > 0x7fffffffLL) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0) return EA_OK;
+    if (!head_offsets) return EA_ERR_INVALID_ARG;
+    if (n_kept > 0 && (!scores || !kept_idx)) return EA_ERR_INVALID_ARG;
+    const bool do_gather = n_kept > 0 && (k_out != nullptr || v_out != nullptr);
+    if (do_gather && (!k || !v || !k_out || !v_out)) return EA_ERR_INVALID_ARG;
+    if (!aligned16(scores) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+        return EA_ERR_INVALID_ARG;
+    if (do_gather) {
+        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys *
+                                shape->head_dim * sizeof(__nv_bfloat16);
+        const size_t out_bytes = (size_t)shape->n_units * shape->n_kv_heads * n_kept *
+                                 shape->head_dim * sizeof(__nv_bfloat16);
+        const char* ins[2] = {static_cast<const char*>(k), static_cast<const char*>(v)};
+        const char* outs[2] = {static_cast<const char*>(k_out), static_cast<const char*>(v_out)};
+        for (const char* o : outs)
+            for (const char* i : ins)
+                if (o < i + in_bytes && i < o + out_bytes) return EA_ERR_INVALID_ARG;
+    }
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    if (ctx->workspace_bytes < plan.total) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = ea_launch_select_adaptive(ctx, *shape, scores, n_kept, n_floor,
+                                   static_cast<char*>(ctx->workspace) + plan.adaptive, kept_idx, head_offsets, stream);
+    if (st == EA_OK && do_gather)
+        st = ea_launch_gather_adaptive(ctx, *shape, n_kept, kept_idx, head_offsets,
+                                       static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
+                                       static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+int64_t ea_n_floor(int64_t n_kept, double safeguard) {
+    const double x = (double)n_kept * safeguard;
+    int64_t f = (int64_t)x;
+    if (f < 0) f = 0;
+    if (f > n_kept) f = n_kept;
+    return f;
 }
 
 ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream) {

@@ -47,6 +47,7 @@ struct ea_ws_plan {
     size_t image;        // bf16 covariance images of the tensor-core log-score kernel (ea_score)
     size_t vec;          // fp32 [U*Hq, d] epilogue vectors of that kernel               (ea_score)
     size_t lse_part;     // fp32 [U*Hq, chunks, 2] log-sum-exp partials of that kernel    (ea_score)
+    size_t adaptive;     // radix histograms, search state and per-head counts (ea_select_compact_adaptive)
     size_t total;
 };
 
@@ -87,6 +88,16 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
 
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
                            int32_t* kept_idx, cudaStream_t st);
+
+// Head-adaptive eviction: per-head counts and offsets from one radix search over the unit's scores,
+// then the per-head selection with those counts and a gather through the offsets.
+size_t ea_adaptive_ws_bytes(const ea_shape& s);
+ea_status ea_launch_select_adaptive(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
+                                    int n_floor, void* ws, int32_t* kept_idx, int32_t* head_offsets,
+                                    cudaStream_t st);
+ea_status ea_launch_gather_adaptive(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
+                                    const int32_t* head_offsets, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                    __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t st);
 
 ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
                            const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* k_out,

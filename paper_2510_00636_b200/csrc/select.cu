@@ -15,6 +15,16 @@
 // reproducible.
 // gather_kernel: lanes copy 16 bytes each; a warp moves 512 contiguous output
 // bytes per step.
+//
+// Head-adaptive eviction (the head-adaptive paragraph of Sec. 2.2): every head keeps its n_floor
+// best pairs and the rest of the unit's budget goes to the best remaining pairs of the unit.  The
+// kept set of a head is then a prefix of that head's own order, so all that is new is the count
+// m_g per head.  With c_g(x) the number of keys of head g at or above x, the pairs at or above x
+// that are not safeguarded number f(x) = sum_g max(0, c_g(x) - n_floor), and the threshold T is the
+// largest x with f(x) >= places.  adaptive_hist_kernel / adaptive_decide_kernel find T with the same
+// MSB-first radix search, one 256-bin histogram per head and pass; the last decide step hands the
+// pairs equal to T to the heads in head order and writes m_g and the offsets.  The per-head
+// selection kernels then run with those counts.
 #include <cooperative_groups.h>
 
 #include "ea_internal.h"
@@ -31,15 +41,32 @@ __device__ __forceinline__ uint32_t order_key(float x) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// Where a head's kept indices go and how many there are: n_kept each, one head after the other, or
+// (head-adaptive) a count per head and an offset per head inside the unit's range of the output.
+struct HeadPlan {
+    const int32_t* head_kept;     // [units * Hkv] or nullptr
+    const int32_t* head_off;      // [units, Hkv + 1]
+    int Hkv;
+    int unit_stride;              // kept indices per unit
+};
+
+__device__ __forceinline__ int32_t* head_output(const HeadPlan& plan, int head, int32_t* kept_idx, int& n_kept) {
+    if (!plan.head_kept) return kept_idx + (size_t)head * n_kept;
+    const int u = head / plan.Hkv, g = head % plan.Hkv;
+    n_kept = plan.head_kept[head];
+    return kept_idx + (size_t)u * plan.unit_stride + plan.head_off[(size_t)u * (plan.Hkv + 1) + g];
+}
+
 __global__ void __launch_bounds__(kSelThreads)
-select_kernel(const float* __restrict__ scores, int n, int n_kept, int32_t* __restrict__ kept_idx) {
+select_kernel(const float* __restrict__ scores, int n, int n_kept, const HeadPlan plan,
+              int32_t* __restrict__ kept_idx) {
     __shared__ unsigned hist[256];
     __shared__ unsigned sh_prefix, sh_need;
     __shared__ unsigned warp_tot[32];
     __shared__ unsigned chunk_tot;
 
     const float* s = scores + (size_t)blockIdx.x * n;
-    int32_t* out = kept_idx + (size_t)blockIdx.x * n_kept;
+    int32_t* out = head_output(plan, (int)blockIdx.x, kept_idx, n_kept);
     const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
     if (n_kept <= 0) return;
 
@@ -142,7 +169,7 @@ constexpr int kClMaxSlice = 49152;      // keys of one CTA's slice: 192 KiB of s
 
 // Cluster of C CTAs per head; CTA `rank` owns keys [rank * slice, min(n, (rank + 1) * slice)).
 __global__ void __launch_bounds__(kClThreads)
-select_cluster_kernel(const float* __restrict__ scores, int n, int n_kept, int slice,
+select_cluster_kernel(const float* __restrict__ scores, int n, int n_kept, int slice, const HeadPlan plan,
                       int32_t* __restrict__ kept_idx) {
     extern __shared__ uint32_t keys[];                 // [slice] order keys of this CTA's slice
     __shared__ unsigned hist[256];                     // local histogram; in rank 0 also the cluster's sum
@@ -160,7 +187,8 @@ select_cluster_kernel(const float* __restrict__ scores, int n, int n_kept, int s
     const int begin = (int)rank * slice;
     const int count = max(0, min(n, begin + slice) - begin);
     const float* s = scores + (size_t)head * n + begin;
-    int32_t* out = kept_idx + (size_t)head * n_kept;
+    int32_t* out = head_output(plan, head, kept_idx, n_kept);
+    if (n_kept <= 0) return;                           // the same for every CTA of the cluster
     unsigned* ghist0 = cluster.map_shared_rank(&ghist[0][0], 0);
     unsigned* cnt0 = cluster.map_shared_rank(&slice_cnt[0][0], 0);
 
@@ -329,10 +357,161 @@ __global__ void gather_kernel(const int32_t* __restrict__ kept_idx, long long n_
     }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Head-adaptive counts.
+constexpr int kAdSpan = 16384;        // keys per CTA of the histogram kernel
+
+struct AdaptiveWs {
+    unsigned* ghist;      // [4][heads][256]
+    unsigned* prefix;     // [units]  digits of the threshold found so far
+    unsigned* above;      // [heads]  keys of the head above every key that shares the prefix
+    int32_t* head_kept;   // [heads]  m_g
+};
+
+__host__ __device__ inline AdaptiveWs adaptive_ws(void* ws, size_t units, size_t heads) {
+    AdaptiveWs a;
+    a.ghist = static_cast<unsigned*>(ws);
+    a.prefix = a.ghist + 4 * heads * 256;
+    a.above = a.prefix + units;
+    a.head_kept = reinterpret_cast<int32_t*>(a.above + heads);
+    return a;
+}
+
+// Histogram of digit `pass` (MSB first) over the keys of a head that share the unit's prefix.
+__global__ void __launch_bounds__(kSelThreads)
+adaptive_hist_kernel(const float* __restrict__ scores, int n, int Hkv, int pass,
+                     const unsigned* __restrict__ prefix_u, unsigned* __restrict__ ghist_pass) {
+    __shared__ unsigned hist[256];
+    const int head = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid % 32;
+    const int shift = 24 - 8 * pass;
+    const unsigned mask = pass == 0 ? 0u : 0xffffffffu << (32 - 8 * pass);
+    const unsigned prefix = pass == 0 ? 0u : prefix_u[head / Hkv];
+    const float* s = scores + (size_t)head * n;
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const int begin = blockIdx.y * kAdSpan, end = min(n, begin + kAdSpan);
+    for (int i0 = begin; i0 < end; i0 += kSelThreads) {
+        const int i = i0 + tid;
+        const bool live = i < end;
+        const uint32_t key = live ? order_key(s[i]) : 0u;
+        const bool cand = live && ((key & mask) == prefix);
+        const unsigned digit = (key >> shift) & 255u;
+        const unsigned voters = __ballot_sync(0xffffffffu, cand);
+        if (cand) {
+            const unsigned peers = __match_any_sync(voters, digit);
+            if (lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+        }
+    }
+    __syncthreads();
+    if (tid < 256 && hist[tid]) atomicAdd(&ghist_pass[(size_t)head * 256 + tid], hist[tid]);   // integer sums: order-free
+}
+
+// Inclusive suffix sum over the 256 threads of a block (thread b gets the sum over threads >= b).
+__device__ __forceinline__ unsigned block_suffix_sum(unsigned v, unsigned* warp_tot) {
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned o = __shfl_down_sync(0xffffffffu, v, off);
+        if (lane + off < 32) v += o;
+    }
+    __syncthreads();                       // warp_tot may still be read from the previous call
+    if (lane == 0) warp_tot[warp] = v;
+    __syncthreads();
+    for (int w = warp + 1; w < 8; ++w) v += warp_tot[w];
+    return v;
+}
+
+// One CTA of 256 threads (one per bin) per unit: the digit of the threshold at this pass; after the
+// last pass also the count of every head and the offsets.
+__global__ void __launch_bounds__(256)
+adaptive_decide_kernel(int Hkv, int n_floor, unsigned long long places, int pass,
+                       const unsigned* __restrict__ ghist_pass, unsigned* __restrict__ prefix_u,
+                       unsigned* __restrict__ above, int32_t* __restrict__ head_kept,
+                       int32_t* __restrict__ head_off) {
+    __shared__ unsigned warp_tot[8];
+    __shared__ int sh_digit;
+    const int u = blockIdx.x, b = threadIdx.x;
+    const int shift = 24 - 8 * pass;
+    // f(b): pairs of the unit, outside the safeguard shares, whose key is at or above bin b of the prefix
+    unsigned long long f = 0ull;
+    for (int g = 0; g < Hkv; ++g) {
+        const size_t head = (size_t)u * Hkv + g;
+        const unsigned at_or_above = above[head] + block_suffix_sum(ghist_pass[head * 256 + b], warp_tot);
+        f += at_or_above > (unsigned)n_floor ? at_or_above - (unsigned)n_floor : 0u;
+    }
+    if (b == 0) sh_digit = 0;
+    __syncthreads();
+    if (f >= places) atomicMax(&sh_digit, b);          // f falls as b rises: the largest bin that still reaches `places`
+    __syncthreads();
+    const int digit = sh_digit;
+    // keys above the chosen bin are above the threshold for good
+    for (int g = 0; g < Hkv; ++g) {
+        const size_t head = (size_t)u * Hkv + g;
+        const unsigned h = ghist_pass[head * 256 + b];
+        const unsigned higher = block_suffix_sum(b > digit ? h : 0u, warp_tot);
+        if (b == 0) above[head] += higher;
+    }
+    if (b == 0) prefix_u[u] |= (unsigned)digit << shift;
+    if (pass < 3) return;
+    __syncthreads();
+    if (b == 0) {
+        // threshold T = prefix: every pair above T outside the safeguard shares is kept, the pairs equal
+        // to T fill what is left, heads in order (inside a head: lowest index first)
+        unsigned long long taken_above = 0ull;
+        for (int g = 0; g < Hkv; ++g) {
+            const unsigned gt = above[(size_t)u * Hkv + g];
+            taken_above += gt > (unsigned)n_floor ? gt - (unsigned)n_floor : 0u;
+        }
+        unsigned long long left = places - taken_above;
+        int32_t off = 0;
+        for (int g = 0; g < Hkv; ++g) {
+            const size_t head = (size_t)u * Hkv + g;
+            const unsigned gt = above[head], eq = ghist_pass[head * 256 + digit];
+            const unsigned base = gt > (unsigned)n_floor ? gt : (unsigned)n_floor;
+            const unsigned free_eq = gt + eq > base ? gt + eq - base : 0u;
+            const unsigned take = (unsigned long long)free_eq < left ? free_eq : (unsigned)left;
+            left -= take;
+            head_kept[head] = (int32_t)(base + take);
+            head_off[(size_t)u * (Hkv + 1) + g] = off;
+            off += (int32_t)(base + take);
+        }
+        head_off[(size_t)u * (Hkv + 1) + Hkv] = off;
+    }
+}
+
+template <int D>
+__global__ void gather_adaptive_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ head_off,
+                                       long long n_rows_out, int n, int Hkv, int unit_stride,
+                                       const uint4* __restrict__ k, const uint4* __restrict__ v,
+                                       uint4* __restrict__ k_out, uint4* __restrict__ v_out) {
+    constexpr int LPR = D / 8;                 // 16-byte pieces per row
+    const long long total = n_rows_out * LPR;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
+        const long long row = t / LPR;
+        const int piece = (int)(t % LPR);
+        const long long u = row / unit_stride;
+        const int j = (int)(row % unit_stride);
+        // the head whose range holds j: the last g with head_off[g] <= j
+        const int32_t* off = head_off + u * (Hkv + 1);
+        int lo = 0, hi = Hkv - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) / 2;
+            if (off[mid] <= j) lo = mid;
+            else hi = mid - 1;
+        }
+        const long long src = (u * Hkv + lo) * n + kept_idx[row];
+        k_out[t] = __ldg(k + src * LPR + piece);
+        v_out[t] = __ldg(v + src * LPR + piece);
+    }
+}
+
 }  // namespace
 
-ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
-                           int32_t* kept_idx, cudaStream_t st) {
+static ea_status launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
+                               const HeadPlan& plan, int32_t* kept_idx, cudaStream_t st) {
     if (n_kept <= 0) return EA_OK;
     ea_count_launches(ctx, 1);
     const int heads = s.n_units * s.n_kv_heads;
@@ -357,10 +536,80 @@ ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* sc
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, select_cluster_kernel, scores, s.n_keys, n_kept, slice, kept_idx) != cudaSuccess)
+        if (cudaLaunchKernelEx(&cfg, select_cluster_kernel, scores, s.n_keys, n_kept, slice, plan, kept_idx) !=
+            cudaSuccess)
             return EA_ERR_CUDA;
     } else {
-        select_kernel<<<heads, kSelThreads, 0, st>>>(scores, s.n_keys, n_kept, kept_idx);
+        select_kernel<<<heads, kSelThreads, 0, st>>>(scores, s.n_keys, n_kept, plan, kept_idx);
+    }
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
+                           int32_t* kept_idx, cudaStream_t st) {
+    const HeadPlan plan = {nullptr, nullptr, s.n_kv_heads, 0};
+    return launch_select(ctx, s, scores, n_kept, plan, kept_idx, st);
+}
+
+size_t ea_adaptive_ws_bytes(const ea_shape& s) {
+    const size_t units = (size_t)s.n_units, heads = units * (size_t)s.n_kv_heads;
+    return (4 * heads * 256 + units + 2 * heads) * sizeof(unsigned);
+}
+
+ea_status ea_launch_select_adaptive(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
+                                    int n_floor, void* ws, int32_t* kept_idx, int32_t* head_offsets,
+                                    cudaStream_t st) {
+    const size_t units = (size_t)s.n_units, heads = units * (size_t)s.n_kv_heads;
+    const AdaptiveWs a = adaptive_ws(ws, units, heads);
+    if (cudaMemsetAsync(ws, 0, ea_adaptive_ws_bytes(s), st) != cudaSuccess) return EA_ERR_CUDA;
+    const unsigned long long places = (unsigned long long)s.n_kv_heads * (unsigned long long)(n_kept - n_floor);
+    const dim3 hist_grid((unsigned)heads, (unsigned)((s.n_keys + kAdSpan - 1) / kAdSpan));
+    if (hist_grid.y > 65535u) return EA_ERR_UNSUPPORTED;
+    for (int pass = 0; pass < 4; ++pass) {
+        unsigned* gh = a.ghist + (size_t)pass * heads * 256;
+        if (s.n_keys > 0)
+            adaptive_hist_kernel<<<hist_grid, kSelThreads, 0, st>>>(scores, s.n_keys, s.n_kv_heads, pass, a.prefix, gh);
+        adaptive_decide_kernel<<<(unsigned)units, 256, 0, st>>>(s.n_kv_heads, n_floor, places, pass, gh, a.prefix,
+                                                                a.above, a.head_kept, head_offsets);
+        ea_count_launches(ctx, s.n_keys > 0 ? 2 : 1);
+    }
+    if (cudaGetLastError() != cudaSuccess) return EA_ERR_CUDA;
+    const HeadPlan plan = {a.head_kept, head_offsets, s.n_kv_heads, s.n_kv_heads * n_kept};
+    // n_kept here only says "some head may keep something"; every head reads its own count
+    return launch_select(ctx, s, scores, n_kept, plan, kept_idx, st);
+}
+
+ea_status ea_launch_gather_adaptive(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
+                                    const int32_t* head_offsets, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                    __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t st) {
+    if (n_kept <= 0) return EA_OK;
+    ea_count_launches(ctx, 1);
+    const int unit_stride = s.n_kv_heads * n_kept;
+    const long long rows = (long long)s.n_units * unit_stride;
+    const int threads = 256;
+    const long long pieces = rows * (s.head_dim / 8);
+    long long want = (pieces + threads - 1) / threads;
+    const long long cap = (long long)ctx->sm_count * 16;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    const uint4* k4 = reinterpret_cast<const uint4*>(k);
+    const uint4* v4 = reinterpret_cast<const uint4*>(v);
+    uint4* ko = reinterpret_cast<uint4*>(k_out);
+    uint4* vo = reinterpret_cast<uint4*>(v_out);
+    switch (s.head_dim) {
+        case 64:
+            gather_adaptive_kernel<64><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, s.n_keys, s.n_kv_heads,
+                                                                 unit_stride, k4, v4, ko, vo);
+            break;
+        case 128:
+            gather_adaptive_kernel<128><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, s.n_keys, s.n_kv_heads,
+                                                                  unit_stride, k4, v4, ko, vo);
+            break;
+        case 256:
+            gather_adaptive_kernel<256><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, s.n_keys, s.n_kv_heads,
+                                                                  unit_stride, k4, v4, ko, vo);
+            break;
+        default:
+            return EA_ERR_UNSUPPORTED;
     }
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

@@ -92,6 +92,69 @@ void eao_mean_cov(const uint16_t *q_win, int64_t n_heads, int W, int d, int cov_
 }
 
 /*
+ * Query statistics from hidden states (Eq. 5 as the paper writes it): the hidden
+ * states of a unit, h_w (W rows of d_model), have mean mu_h and covariance
+ * Sigma_h; the queries of head j are q = W_Q^j h (pre-RoPE), so
+ *   mu_j = W_Q^j mu_h,     Sigma_j = W_Q^j Sigma_h W_Q^j^T.
+ * hidden: bf16 [n_units, W, dm]; w_q: bf16 [n_sets, Hq * d, dm], unit u uses set
+ * u % n_sets (row j * d + c of a set is row c of W_Q^j).  Sigma_h is built in
+ * full (dm x dm) and the two products are plain triple loops.
+ */
+void eao_hidden_mean_cov(const uint16_t *hidden, const uint16_t *w_q, int n_units, int n_sets, int Hq,
+                         int W, int d, int dm, int cov_norm, double *mu, double *sigma) {
+    double denom = (cov_norm == EAO_COV_SAMPLE) ? (double)(W - 1) : (double)W;
+    for (int u = 0; u < n_units; ++u) {
+        const uint16_t *H = hidden + (int64_t)u * W * dm;
+        const uint16_t *WQ = w_q + (int64_t)(u % n_sets) * Hq * d * dm;
+        double *mh = (double *)calloc((size_t)dm, sizeof(double));
+        double *Sh = (double *)calloc((size_t)dm * dm, sizeof(double));
+        for (int a = 0; a < dm; ++a) {
+            double acc = 0.0;
+            for (int w = 0; w < W; ++w) acc += bf16_to_f64(H[(int64_t)w * dm + a]);
+            mh[a] = acc / (double)W;
+        }
+#pragma omp parallel for schedule(static)
+        for (int a = 0; a < dm; ++a)
+            for (int b = 0; b < dm; ++b) {
+                double acc = 0.0;
+                for (int w = 0; w < W; ++w)
+                    acc += (bf16_to_f64(H[(int64_t)w * dm + a]) - mh[a]) *
+                           (bf16_to_f64(H[(int64_t)w * dm + b]) - mh[b]);
+                Sh[(int64_t)a * dm + b] = acc / denom;
+            }
+#pragma omp parallel for schedule(dynamic)
+        for (int j = 0; j < Hq; ++j) {
+            const uint16_t *Wj = WQ + (int64_t)j * d * dm;
+            double *m = mu + ((int64_t)u * Hq + j) * d;
+            double *S = sigma + ((int64_t)u * Hq + j) * d * d;
+            double *tmp = (double *)calloc((size_t)d * dm, sizeof(double));      /* W_Q Sigma_h */
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int a = 0; a < dm; ++a) acc += bf16_to_f64(Wj[(int64_t)c * dm + a]) * mh[a];
+                m[c] = acc;
+            }
+            for (int c = 0; c < d; ++c)
+                for (int b = 0; b < dm; ++b) {
+                    double acc = 0.0;
+                    for (int a = 0; a < dm; ++a)
+                        acc += bf16_to_f64(Wj[(int64_t)c * dm + a]) * Sh[(int64_t)a * dm + b];
+                    tmp[(int64_t)c * dm + b] = acc;
+                }
+            for (int c = 0; c < d; ++c)
+                for (int e = 0; e < d; ++e) {
+                    double acc = 0.0;
+                    for (int b = 0; b < dm; ++b)
+                        acc += tmp[(int64_t)c * dm + b] * bf16_to_f64(Wj[(int64_t)e * dm + b]);
+                    S[(int64_t)c * d + e] = acc;
+                }
+            free(tmp);
+        }
+        free(Sh);
+        free(mh);
+    }
+}
+
+/*
  * Averaged RoPE rotation (Eq. 6): R_bar = (1/T) sum_j R_p over the T future
  * positions p = pos_next .. pos_next + T - 1 (0-based positions; the paper's
  * t+1 .. t+T with 1-based keys 1..t).  R_p is block diagonal with one 2x2
@@ -248,6 +311,48 @@ void eao_scores(const double *s, const uint16_t *v, int n_units, int Hq, int Hkv
             if (a_out) a_out[ug * n + i] = a[i];
         }
         free(a);
+    }
+}
+
+/*
+ * Contribution score with the output projection (Eq. 9 as written, ||W_o v||).
+ * The output projection W_o is [dm, Hq * d]; query head h multiplies the value it
+ * reads by its own slice W_o^h = W_o[:, h*d : (h+1)*d], so the pair (g, i) leaves
+ * the head-h branch with magnitude ||W_o^h v_{g,i}||.  Per query head
+ *   c_{h,i} = (a_hat_{h,i} + eps) * ||W_o^h v_{g,i}||_2,    a_hat from Eq. 8,
+ * and the heads of a group are reduced as the attention is:
+ *   MEAN_PROB: score_{g,i} = (1/G) sum_{h in g} c_{h,i};   SUM_PROB: the plain sum.
+ * w_o: bf16 [n_sets, dm, Hq * d], unit u uses set u % n_sets.  The product W_o^h v
+ * is formed explicitly (dm entries) and its norm taken.
+ */
+void eao_scores_wo(const double *s, const uint16_t *v, const uint16_t *w_o, int n_units, int n_sets,
+                   int Hq, int Hkv, int64_t n, int d, int dm, double eps, int group_mode,
+                   double *score) {
+    int G = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t ug = 0; ug < (int64_t)n_units * Hkv; ++ug) {
+        int u = (int)(ug / Hkv), g = (int)(ug % Hkv);
+        const uint16_t *Wo = w_o + (int64_t)(u % n_sets) * dm * Hq * d;
+        const uint16_t *vv = v + ug * n * d;
+        for (int64_t i = 0; i < n; ++i) score[ug * n + i] = 0.0;
+        for (int j = 0; j < G; ++j) {
+            int h = g * G + j;
+            const double *sh = s + ((int64_t)u * Hq + h) * n;
+            double lse = n > 0 ? log_sum_exp(sh, n) : 0.0;
+            for (int64_t i = 0; i < n; ++i) {
+                double ss = 0.0;
+                for (int a = 0; a < dm; ++a) {
+                    double y = 0.0;
+                    for (int c = 0; c < d; ++c)
+                        y += bf16_to_f64(Wo[(int64_t)a * Hq * d + (int64_t)h * d + c]) *
+                             bf16_to_f64(vv[i * d + c]);
+                    ss += y * y;
+                }
+                score[ug * n + i] += (exp(sh[i] - lse) + eps) * sqrt(ss);
+            }
+        }
+        if (group_mode == EAO_GROUP_MEAN_PROB)
+            for (int64_t i = 0; i < n; ++i) score[ug * n + i] /= (double)G;
     }
 }
 

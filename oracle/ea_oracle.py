@@ -58,6 +58,10 @@ def _load():
         lib.eao_gather.argtypes = [vp, vp, i64, i64, i64, i32, vp]
         lib.eao_n_kept.argtypes = [i64, f64]
         lib.eao_n_kept.restype = i64
+        lib.eao_hidden_mean_cov.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
+        lib.eao_hidden_mean_cov.restype = None
+        lib.eao_scores_wo.argtypes = [vp, vp, vp, i32, i32, i32, i32, i64, i32, i32, f64, i32, vp]
+        lib.eao_scores_wo.restype = None
         lib.eao_select_adaptive.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp]
         lib.eao_gather_adaptive.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp]
         lib.eao_n_floor.argtypes = [i64, f64]
@@ -134,6 +138,29 @@ def query_stats(q_win_bits, pos_next, n_future, rope_base, layout=ROPE_HALF_SPLI
     return apply_rope_average(mu, sigma, cbar, sbar, layout)
 
 
+def hidden_mean_cov(hidden_bits, w_q_bits, n_q_heads, cov_norm=COV_POPULATION):
+    """hidden_bits uint16 [U, W, dm]; w_q_bits uint16 [sets, Hq*d, dm] (unit u uses set u % sets)
+    -> (mu [U,Hq,d], sigma [U,Hq,d,d]) of the pre-RoPE queries q = W_Q h."""
+    H = _c(hidden_bits, np.uint16)
+    Wq = _c(w_q_bits, np.uint16)
+    U, W, dm = H.shape
+    sets, rows, dm2 = Wq.shape
+    assert dm2 == dm and rows % n_q_heads == 0
+    d = rows // n_q_heads
+    mu = np.empty((U, n_q_heads, d), np.float64)
+    sigma = np.empty((U, n_q_heads, d, d), np.float64)
+    _load().eao_hidden_mean_cov(_p(H), _p(Wq), U, sets, n_q_heads, W, d, dm, cov_norm, _p(mu), _p(sigma))
+    return mu, sigma
+
+
+def query_stats_hidden(hidden_bits, w_q_bits, n_q_heads, pos_next, n_future, rope_base,
+                       layout=ROPE_HALF_SPLIT, cov_norm=COV_POPULATION):
+    """Hidden states and query projections -> (mu_bar, sigma_bar) as query_stats gives them."""
+    mu, sigma = hidden_mean_cov(hidden_bits, w_q_bits, n_q_heads, cov_norm)
+    cbar, sbar = rope_average(pos_next, n_future, rope_base, mu.shape[-1])
+    return apply_rope_average(mu, sigma, cbar, sbar, layout)
+
+
 def logits(k_bits, mu_bar, sigma_bar):
     """k_bits uint16 [U,Hkv,n,d]; mu_bar [U,Hq,d]; sigma_bar [U,Hq,d,d] -> s [U,Hq,n]."""
     k = _c(k_bits, np.uint16)
@@ -157,6 +184,23 @@ def scores(s, v_bits, eps, group_mode=GROUP_MEAN_PROB, return_attention=False):
     _load().eao_scores(_p(s), _p(v), U, Hq, Hkv, n, d, float(eps), group_mode, _p(score),
                        _p(a) if a is not None else None)
     return (score, a) if return_attention else score
+
+
+def scores_wo(s, v_bits, w_o_bits, eps, group_mode=GROUP_MEAN_PROB):
+    """s [U,Hq,n]; v_bits uint16 [U,Hkv,n,d]; w_o_bits uint16 [sets, dm, Hq*d] -> score [U,Hkv,n]
+    with ||W_o^h v|| in place of ||v|| (Eq. 9 as written); MEAN_PROB or SUM_PROB."""
+    if group_mode == GROUP_MEAN_LOGIT:
+        raise ValueError("the output-projection weighting is defined per query head")
+    s = _c(s, np.float64)
+    v = _c(v_bits, np.uint16)
+    wo = _c(w_o_bits, np.uint16)
+    U, Hkv, n, d = v.shape
+    Hq = s.shape[1]
+    sets, dm, cols = wo.shape
+    assert cols == Hq * d
+    score = np.empty((U, Hkv, n), np.float64)
+    _load().eao_scores_wo(_p(s), _p(v), _p(wo), U, sets, Hq, Hkv, n, d, dm, float(eps), group_mode, _p(score))
+    return score
 
 
 def select(score, n_kept_):

@@ -59,6 +59,48 @@ def test_mean_cov_matches_numpy(oracle, norm):
     assert (ev > 1e-10).sum() <= 4
 
 
+# ---------------------------------------------------------------- statistics from hidden states
+@pytest.mark.parametrize("norm", [0, 1])
+def test_hidden_statistics_equal_statistics_of_projected_samples(oracle, norm):
+    """W_Q mu_h and W_Q Sigma_h W_Q^T against numpy's mean / cov of the explicitly projected rows."""
+    rng = np.random.default_rng(31)
+    U, W, dm, Hq, d = 3, 11, 24, 2, 8
+    hb, h = bf16_bits(rng.normal(size=(U, W, dm)) + rng.normal(size=(U, 1, dm)))
+    wb, wq = bf16_bits(rng.normal(size=(2, Hq * d, dm)) / np.sqrt(dm))
+    mu, sigma = oracle.hidden_mean_cov(hb, wb, Hq, cov_norm=norm)
+    for u in range(U):
+        q = h[u] @ wq[u % 2].T                                     # [W, Hq*d]
+        for j in range(Hq):
+            qj = q[:, j * d:(j + 1) * d]
+            np.testing.assert_allclose(mu[u, j], qj.mean(0), rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(sigma[u, j], np.cov(qj.T, bias=(norm == 0)), rtol=1e-10, atol=1e-13)
+
+
+def test_hidden_statistics_with_selector_projection_are_window_statistics(oracle):
+    """W_Q that picks d hidden channels per head: the result is mean_cov of those channels."""
+    rng = np.random.default_rng(32)
+    U, W, Hq, d = 2, 9, 3, 4
+    dm = Hq * d
+    hb, _ = bf16_bits(rng.normal(size=(U, W, dm)))
+    wb, _ = bf16_bits(np.eye(dm)[None])
+    mu, sigma = oracle.hidden_mean_cov(hb, wb, Hq)
+    q_win = hb.reshape(U, W, Hq, d).transpose(0, 2, 1, 3)           # [U, Hq, W, d]
+    mu2, sigma2 = oracle.mean_cov(q_win)
+    np.testing.assert_allclose(mu, mu2, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(sigma, sigma2, rtol=1e-12, atol=1e-15)
+    # scaling the projection by c scales the mean by c and the covariance by c^2
+    wb2, _ = bf16_bits(2.0 * np.eye(dm)[None])
+    mu3, sigma3 = oracle.hidden_mean_cov(hb, wb2, Hq)
+    np.testing.assert_allclose(mu3, 2.0 * mu, rtol=1e-13)
+    np.testing.assert_allclose(sigma3, 4.0 * sigma, rtol=1e-13)
+    # and the whole statistics step agrees with the window form
+    pos = np.array([7, 100], np.int64)
+    a = oracle.query_stats_hidden(hb, wb, Hq, pos, 5, 1e4)
+    b = oracle.query_stats(q_win, pos, 5, 1e4)
+    np.testing.assert_allclose(a[0], b[0], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(a[1], b[1], rtol=1e-12, atol=1e-15)
+
+
 # ---------------------------------------------------------------- O2 averaged rotation
 @pytest.mark.parametrize("pos,T,base,d", [(512, 512, 1e4, 64), (8192, 512, 5e5, 128),
                                           (131072, 1024, 1e6, 256), (0, 1, 1e4, 8), (7, 3, 10.0, 4)])
@@ -233,6 +275,46 @@ def test_group_modes_coincide_without_grouping(oracle):
     base = oracle.scores(s, v_bits, 0.02, oracle.GROUP_MEAN_PROB)
     for mode in (oracle.GROUP_SUM_PROB, oracle.GROUP_MEAN_LOGIT):
         np.testing.assert_allclose(oracle.scores(s, v_bits, 0.02, mode), base, rtol=1e-13)
+
+
+# ---------------------------------------------------------------- Eq. 9 with the output projection
+def test_scores_with_output_projection(oracle):
+    rng = np.random.default_rng(41)
+    U, Hq, Hkv, n, d, dm = 2, 4, 2, 13, 8, 12
+    G = Hq // Hkv
+    s = rng.normal(size=(U, Hq, n)) * 3
+    vb, v = bf16_bits(rng.normal(size=(U, Hkv, n, d)))
+    wb, wo = bf16_bits(rng.normal(size=(2, dm, Hq * d)))
+    for mode in (0, 1):
+        got = oracle.scores_wo(s, vb, wb, 0.02, group_mode=mode)
+        # numpy restatement through the softmax library form and explicit matrix-vector products
+        a_hat = np.exp(s - s.max(-1, keepdims=True))
+        a_hat /= a_hat.sum(-1, keepdims=True)
+        want = np.zeros((U, Hkv, n))
+        for u in range(U):
+            for h in range(Hq):
+                g = h // G
+                y = v[u, g] @ wo[u % 2][:, h * d:(h + 1) * d].T          # [n, dm]
+                want[u, g] += (a_hat[u, h] + 0.02) * np.linalg.norm(y, axis=-1)
+        if mode == 0:
+            want /= G
+        np.testing.assert_allclose(got, want, rtol=1e-12)
+    # an output projection with orthonormal columns per head leaves the norm of v unchanged:
+    # the score falls back to the ||v|| form
+    q, _ = np.linalg.qr(rng.normal(size=(dm, d)))                          # [dm, d], orthonormal columns
+    wo_iso = np.concatenate([q] * Hq, axis=1)[None]
+    wb_iso, wo_iso_r = bf16_bits(wo_iso)
+    got = oracle.scores_wo(s, vb, wb_iso, 0.02)
+    plain = oracle.scores(s, vb, 0.02)
+    np.testing.assert_allclose(got, plain, rtol=2e-2)                      # bf16 rounding of the projection
+    # exactly so for a selector matrix (representable in bf16)
+    sel = np.zeros((dm, d)); sel[:d, :d] = np.eye(d)
+    wb_sel, _ = bf16_bits(np.concatenate([sel] * Hq, axis=1)[None])
+    np.testing.assert_allclose(oracle.scores_wo(s, vb, wb_sel, 0.02), plain, rtol=1e-12)
+    np.testing.assert_allclose(oracle.scores_wo(s, vb, wb_sel, 0.0, group_mode=1),
+                               oracle.scores(s, vb, 0.0, group_mode=1), rtol=1e-12)
+    with pytest.raises(ValueError):
+        oracle.scores_wo(s, vb, wb_sel, 0.02, group_mode=2)
 
 
 # ---------------------------------------------------------------- O8-O9 selection and compaction

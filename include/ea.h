@@ -166,6 +166,35 @@ ea_status ea_query_stats_static(const ea_shape* shape, const void* q_win, const 
                                 void* cuda_stream);
 
 /*
+ * The same statistics from buffered hidden states (Eq. 5 as the paper writes
+ * it: h ~ N(mu_h, Sigma_h), q = W_Q h, so mu = W_Q mu_h and
+ * Sigma = W_Q Sigma_h W_Q^T per query head; the decoding set-up keeps a
+ * buffer of the last hidden states for this).  The library projects the W
+ * buffered rows (Q = H W_Q^T on the tensor cores, fp32) and takes the mean and
+ * covariance of the projected rows, which are those two expressions exactly;
+ * the d_model x d_model covariance is never formed.  Then Eq. 6 as in
+ * ea_query_stats.
+ *
+ * hidden     bf16 [n_units, W, d_model]  the inputs of the query projection
+ *            (i.e. after the layer's input norm), W = shape->window <= 512
+ * w_q        bf16 [n_weight_sets, Hq * d, d_model]  query projections; row
+ *            j * d + c of a set is row c of W_Q of head j.  Units are taken
+ *            set-major: unit u uses set u / (n_units / n_weight_sets)
+ *            (n_units = layers * batch with one set per layer).
+ * d_model    a multiple of 8
+ * q_scratch  fp32 [n_units, Hq, W, d]  caller-owned scratch; holds the
+ *            projected window queries on return
+ * the other arguments as for ea_query_stats.
+ * EA_ERR_UNSUPPORTED for W > 512; EA_ERR_INVALID_ARG for a bad d_model or
+ * n_weight_sets that does not divide n_units.
+ */
+ea_status ea_query_stats_hidden(ea_ctx* ctx, const ea_shape* shape, const void* hidden,
+                                const void* w_q, int32_t d_model, int32_t n_weight_sets,
+                                float* q_scratch, const int64_t* pos_next, int32_t n_future,
+                                double rope_base, float* mu_bar, float* sigma_bar,
+                                void* cuda_stream);
+
+/*
  * Contribution score of every cached pair (Eq. 7, 8, 9 with ||v|| in place of
  * ||W_o v||, as the paper's implementation note states):
  *   s_{h,i}   = mu_bar_h . k_i / sqrt(d) + k_i^T sigma_bar_h k_i / (2d)

@@ -96,8 +96,8 @@ void eao_mean_cov(const uint16_t *q_win, int64_t n_heads, int W, int d, int cov_
  * states of a unit, h_w (W rows of d_model), have mean mu_h and covariance
  * Sigma_h; the queries of head j are q = W_Q^j h (pre-RoPE), so
  *   mu_j = W_Q^j mu_h,     Sigma_j = W_Q^j Sigma_h W_Q^j^T.
- * hidden: bf16 [n_units, W, dm]; w_q: bf16 [n_sets, Hq * d, dm], unit u uses set
- * u % n_sets (row j * d + c of a set is row c of W_Q^j).  Sigma_h is built in
+ * hidden: bf16 [n_units, W, dm]; w_q: bf16 [n_sets, Hq * d, dm], units are set-major: unit u uses
+ * set u / (n_units / n_sets) (row j * d + c of a set is row c of W_Q^j).  Sigma_h is built in
  * full (dm x dm) and the two products are plain triple loops.
  */
 void eao_hidden_mean_cov(const uint16_t *hidden, const uint16_t *w_q, int n_units, int n_sets, int Hq,
@@ -105,7 +105,7 @@ void eao_hidden_mean_cov(const uint16_t *hidden, const uint16_t *w_q, int n_unit
     double denom = (cov_norm == EAO_COV_SAMPLE) ? (double)(W - 1) : (double)W;
     for (int u = 0; u < n_units; ++u) {
         const uint16_t *H = hidden + (int64_t)u * W * dm;
-        const uint16_t *WQ = w_q + (int64_t)(u % n_sets) * Hq * d * dm;
+        const uint16_t *WQ = w_q + (int64_t)(u / (n_units / n_sets)) * Hq * d * dm;
         double *mh = (double *)calloc((size_t)dm, sizeof(double));
         double *Sh = (double *)calloc((size_t)dm * dm, sizeof(double));
         for (int a = 0; a < dm; ++a) {
@@ -322,7 +322,7 @@ void eao_scores(const double *s, const uint16_t *v, int n_units, int Hq, int Hkv
  *   c_{h,i} = (a_hat_{h,i} + eps) * ||W_o^h v_{g,i}||_2,    a_hat from Eq. 8,
  * and the heads of a group are reduced as the attention is:
  *   MEAN_PROB: score_{g,i} = (1/G) sum_{h in g} c_{h,i};   SUM_PROB: the plain sum.
- * w_o: bf16 [n_sets, dm, Hq * d], unit u uses set u % n_sets.  The product W_o^h v
+ * w_o: bf16 [n_sets, dm, Hq * d], unit u uses set u / (n_units / n_sets).  The product W_o^h v
  * is formed explicitly (dm entries) and its norm taken.
  */
 void eao_scores_wo(const double *s, const uint16_t *v, const uint16_t *w_o, int n_units, int n_sets,
@@ -332,7 +332,7 @@ void eao_scores_wo(const double *s, const uint16_t *v, const uint16_t *w_o, int 
 #pragma omp parallel for schedule(dynamic)
     for (int64_t ug = 0; ug < (int64_t)n_units * Hkv; ++ug) {
         int u = (int)(ug / Hkv), g = (int)(ug % Hkv);
-        const uint16_t *Wo = w_o + (int64_t)(u % n_sets) * dm * Hq * d;
+        const uint16_t *Wo = w_o + (int64_t)(u / (n_units / n_sets)) * dm * Hq * d;
         const uint16_t *vv = v + ug * n * d;
         for (int64_t i = 0; i < n; ++i) score[ug * n + i] = 0.0;
         for (int j = 0; j < G; ++j) {

@@ -139,7 +139,7 @@ def query_stats(q_win_bits, pos_next, n_future, rope_base, layout=ROPE_HALF_SPLI
 
 
 def hidden_mean_cov(hidden_bits, w_q_bits, n_q_heads, cov_norm=COV_POPULATION):
-    """hidden_bits uint16 [U, W, dm]; w_q_bits uint16 [sets, Hq*d, dm] (unit u uses set u % sets)
+    """hidden_bits uint16 [U, W, dm]; w_q_bits uint16 [sets, Hq*d, dm] (unit u uses set u // (U // sets))
     -> (mu [U,Hq,d], sigma [U,Hq,d,d]) of the pre-RoPE queries q = W_Q h."""
     H = _c(hidden_bits, np.uint16)
     Wq = _c(w_q_bits, np.uint16)

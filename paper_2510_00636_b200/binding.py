@@ -24,7 +24,7 @@ EXPORTS = (
     "ea_version", "ea_status_string", "ea_workspace_bytes", "ea_n_kept", "ea_create", "ea_destroy",
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
-    "ea_select_compact_adaptive", "ea_n_floor",
+    "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.ea_query_stats.argtypes = [vp, sp, vp, vp, i32, f64, vp, vp, vp]
         L.ea_query_stats_static.argtypes = [sp, vp, vp, i32, f64, vp, vp, vp]
         L.ea_query_stats_static.restype = ctypes.c_int
+        L.ea_query_stats_hidden.argtypes = [vp, sp, vp, vp, i32, i32, vp, vp, i32, f64, vp, vp, vp]
+        L.ea_query_stats_hidden.restype = ctypes.c_int
         L.ea_score.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
         L.ea_select_compact.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.ea_select_compact_adaptive.argtypes = [vp, sp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
@@ -178,6 +180,28 @@ def ea_query_stats(ctx: Context, shape: Shape, q_win, pos_next, n_future: int, r
                                 float(rope_base), _ptr(mu_bar), _ptr(sigma_bar), _stream(ctx.device)),
            "ea_query_stats")
     return mu_bar, sigma_bar
+
+
+def ea_query_stats_hidden(ctx: Context, shape: Shape, hidden, w_q, pos_next, n_future: int, rope_base: float,
+                          q_scratch=None, mu_bar=None, sigma_bar=None):
+    """hidden bf16 [U,W,d_model], w_q bf16 [sets, Hq*d, d_model] -> (mu_bar, sigma_bar, q_scratch fp32 [U,Hq,W,d])."""
+    _dev_tensor(hidden, torch.bfloat16, "hidden")
+    _dev_tensor(w_q, torch.bfloat16, "w_q")
+    _dev_tensor(pos_next, torch.int64, "pos_next")
+    U, Hq, d, W = shape.n_units, shape.n_q_heads, shape.head_dim, shape.window
+    d_model, n_sets = hidden.shape[-1], w_q.shape[0]
+    dev = hidden.device
+    if q_scratch is None:
+        q_scratch = torch.empty((U, Hq, W, d), dtype=torch.float32, device=dev)
+    if mu_bar is None:
+        mu_bar = torch.empty((U, Hq, d), dtype=torch.float32, device=dev)
+    if sigma_bar is None:
+        sigma_bar = torch.empty((U, Hq, d, d), dtype=torch.float32, device=dev)
+    _check(lib().ea_query_stats_hidden(ctx._h, ctypes.byref(shape), _ptr(hidden), _ptr(w_q), int(d_model),
+                                       int(n_sets), _ptr(q_scratch), _ptr(pos_next), int(n_future),
+                                       float(rope_base), _ptr(mu_bar), _ptr(sigma_bar), _stream(ctx.device)),
+           "ea_query_stats_hidden")
+    return mu_bar, sigma_bar, q_scratch
 
 
 def ea_query_stats_static(shape: Shape, q_win, pos_next, n_future: int, rope_base: float, mu_bar, sigma_bar):

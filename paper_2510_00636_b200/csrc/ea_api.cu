@@ -177,6 +177,40 @@ ea_status ea_query_stats(ea_ctx* ctx, const ea_shape* shape, const void* q_win,
     return st;
 }
 
+ea_status ea_query_stats_hidden(ea_ctx* ctx, const ea_shape* shape, const void* hidden, const void* w_q,
+                                int32_t d_model, int32_t n_weight_sets, float* q_scratch,
+                                const int64_t* pos_next, int32_t n_future, double rope_base, float* mu_bar,
+                                float* sigma_bar, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (shape->n_units == 0) return EA_OK;
+    if (!hidden || !w_q || !q_scratch || !pos_next || !mu_bar || !sigma_bar) return EA_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(w_q) || !aligned16(q_scratch) || !aligned16(mu_bar) ||
+        !aligned16(sigma_bar))
+        return EA_ERR_INVALID_ARG;
+    if (n_future < 1 || !(rope_base > 0.0)) return EA_ERR_INVALID_ARG;
+    if (shape->window < 1 || (shape->cov_norm == EA_COV_SAMPLE && shape->window < 2))
+        return EA_ERR_INVALID_ARG;
+    if (d_model < 8 || d_model % 8 != 0) return EA_ERR_INVALID_ARG;
+    if (n_weight_sets < 1 || shape->n_units % n_weight_sets != 0) return EA_ERR_INVALID_ARG;
+    if (!ea_project_supported(*shape, d_model)) return EA_ERR_UNSUPPORTED;
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    if (ctx->workspace_bytes < plan.logits /* rope_coef region only */) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    float* coef = reinterpret_cast<float*>(static_cast<char*>(ctx->workspace) + plan.rope_coef);
+    st = ea_launch_project(ctx, *shape, static_cast<const __nv_bfloat16*>(hidden),
+                           static_cast<const __nv_bfloat16*>(w_q), d_model, n_weight_sets, q_scratch, stream);
+    if (st == EA_OK)
+        st = ea_launch_stats_f32(ctx, *shape, q_scratch, pos_next, n_future, rope_base, coef, mu_bar, sigma_bar,
+                                 stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
 ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
                    const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
                    float* logits_opt, void* cuda_stream) {

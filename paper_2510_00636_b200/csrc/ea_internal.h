@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libea.so.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
@@ -69,6 +70,19 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
 ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                 const float* mu_bar, const float* sigma_bar, float* logits,
                                 cudaStream_t st);
+
+// bf16 rank-3 TMA tensor map, box (box0 x box1 x 1), 128-byte swizzle, zero fill outside.
+bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint64_t n1, uint64_t n2,
+                           uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1);
+
+// Window queries from hidden states, Q[u,h,w,:] = W_Q^h H[u,w,:] in fp32 (tcgen05 GEMM).
+bool ea_project_supported(const ea_shape& s, int d_model);
+ea_status ea_launch_project(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* hidden,
+                            const __nv_bfloat16* w_q, int d_model, int n_sets, float* q_win, cudaStream_t st);
+// The statistics kernels on fp32 window queries.
+ea_status ea_launch_stats_f32(const ea_ctx* ctx, const ea_shape& s, const float* q_win, const int64_t* pos_next,
+                              int n_future, double rope_base, float* rope_coef, float* mu_bar, float* sigma_bar,
+                              cudaStream_t st);
 
 // Tensor-core log-score kernel (tcgen05): available for some shapes only.
 bool ea_mma_path_supported(const ea_shape& s);

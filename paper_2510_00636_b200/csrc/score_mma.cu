@@ -574,39 +574,11 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 }
 
 // ------------------------------------------------------------------------------------------
-typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                    CUtensorMapFloatOOBfill);
-
-encode_tiled_fn get_encode_tiled() {
-    static encode_tiled_fn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult res;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) == cudaSuccess &&
-            res == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<encode_tiled_fn>(ptr);
-        else
-            cudaGetLastError();
-    }
-    return fn;
-}
-
 // K as a rank-3 tensor (d, n, unit*kv_head); one box is 64 channels x 128 keys, 128-byte swizzle.
 // Rows past n read as zero.
 bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, long long heads) {
-    encode_tiled_fn enc = get_encode_tiled();
-    if (!enc) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)n, (cuuint64_t)heads};
-    const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)n * d * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kTileKeys, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(k), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return ea_tensor_map_bf16_3d(map, k, (uint64_t)d, (uint64_t)n, (uint64_t)heads, (uint64_t)d * 2,
+                                 (uint64_t)n * d * 2, 64, kTileKeys);
 }
 
 template <int D, bool PAIR>
@@ -671,6 +643,36 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
 }
 
 }  // namespace
+
+// bf16 rank-3 tensor map (innermost extent first) with a (box0 x box1 x 1) box, 128-byte swizzle,
+// zero fill outside the tensor.  Strides in bytes, multiples of 16; base 16-byte aligned.
+bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint64_t n1, uint64_t n2,
+                           uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1) {
+    typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                        const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                        CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                        CUtensorMapFloatOOBfill);
+    static encode_tiled_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) == cudaSuccess &&
+            res == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(ptr);
+        else
+            cudaGetLastError();
+    }
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {n0, n1, n2};
+    const cuuint64_t strides[2] = {stride1, stride2};
+    const cuuint32_t box[3] = {box0, box1, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 bool ea_mma_path_supported(const ea_shape& s) {
     if (s.head_dim == 256) return s.n_keys >= 2 * kTileKeys;

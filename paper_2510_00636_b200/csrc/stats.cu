@@ -51,15 +51,19 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int D>
+template <int D, typename QT>
 constexpr int stats_smem_bytes() {
     constexpr int BM = D < 128 ? D : 128;
-    return 2 * 2 * BM * kXtPitch * 2 + kKC * D * 2 + (D + D) * 4 + (256 / (D / 2)) * D * 4;
+    return 2 * 2 * BM * kXtPitch * 2 + kKC * D * (int)sizeof(QT) + (D + D) * 4 + (256 / (D / 2)) * D * 4;
 }
 
-template <int D>
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ float to_f32(float x) { return x; }
+
+// QT: the window queries as bf16 (what a model's query projection emits) or fp32 (from project_kernel).
+template <int D, typename QT>
 __global__ void __launch_bounds__(256)
-stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
+stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
                  int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar) {
     constexpr int HALF = D / 2;
     constexpr int BM = D < 128 ? D : 128;          // block edge
@@ -72,8 +76,8 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
     typedef __nv_bfloat16 (*xt_t)[2 * BM][kXtPitch];
     xt_t xt = reinterpret_cast<xt_t>(stats_smem);
     constexpr int kXtBytes = 2 * 2 * BM * kXtPitch * 2;
-    __nv_bfloat16* raw = reinterpret_cast<__nv_bfloat16*>(stats_smem + kXtBytes);          // [kKC][D]
-    float* mu_s = reinterpret_cast<float*>(stats_smem + kXtBytes + kKC * D * 2);           // [D]
+    QT* raw = reinterpret_cast<QT*>(stats_smem + kXtBytes);                                // [kKC][D]
+    float* mu_s = reinterpret_cast<float*>(stats_smem + kXtBytes + kKC * D * sizeof(QT));  // [D]
     float* c_s = mu_s + D;                                                                  // [HALF]
     float* s_s = c_s + HALF;                                                                // [HALF]
     float* red = s_s + HALF;                                                                // [256 / (D/2)][D]
@@ -85,7 +89,7 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
     const int bj = NB1 == 1 ? 0 : (blockIdx.y == 0 ? 0 : 1);
     const bool diag = bi == bj;
     const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
-    const __nv_bfloat16* q = q_win + (size_t)uh * W * D;
+    const QT* q = q_win + (size_t)uh * W * D;
 
     for (int m = tid; m < HALF; m += 256) {
         c_s[m] = coef[2 * ((size_t)u * HALF + m)];
@@ -95,12 +99,22 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
         constexpr int NG = 256 / HALF;
         const int cp = tid % HALF, g = tid / HALF;
         float a0 = 0.f, a1 = 0.f;
-        const uint32_t* q2 = reinterpret_cast<const uint32_t*>(q);
+        if constexpr (sizeof(QT) == 2) {
+            const uint32_t* q2 = reinterpret_cast<const uint32_t*>(q);
 #pragma unroll 4
-        for (int w = g; w < W; w += NG) {
-            const uint32_t x = __ldg(q2 + (size_t)w * HALF + cp);
-            a0 += __uint_as_float(x << 16);
-            a1 += __uint_as_float(x & 0xffff0000u);
+            for (int w = g; w < W; w += NG) {
+                const uint32_t x = __ldg(q2 + (size_t)w * HALF + cp);
+                a0 += __uint_as_float(x << 16);
+                a1 += __uint_as_float(x & 0xffff0000u);
+            }
+        } else {
+            const float2* q2 = reinterpret_cast<const float2*>(q);
+#pragma unroll 4
+            for (int w = g; w < W; w += NG) {
+                const float2 x = __ldg(q2 + (size_t)w * HALF + cp);
+                a0 += x.x;
+                a1 += x.y;
+            }
         }
         red[g * D + 2 * cp] = a0;
         red[g * D + 2 * cp + 1] = a1;
@@ -141,9 +155,10 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
     for (int w0 = 0; w0 < W; w0 += kKC) {
         __syncthreads();
         // the raw chunk with 128-bit loads (rows past the window read as zero) ...
-        for (int e = tid; e < kKC * D / 8; e += 256) {
-            const int w = e / (D / 8);
-            raw4[e] = w0 + w < W ? __ldg(q4 + (size_t)w0 * (D / 8) + e) : make_uint4(0u, 0u, 0u, 0u);
+        constexpr int kRowPieces = D * (int)sizeof(QT) / 16;      // 16-byte pieces per window row
+        for (int e = tid; e < kKC * kRowPieces; e += 256) {
+            const int w = e / kRowPieces;
+            raw4[e] = w0 + w < W ? __ldg(q4 + (size_t)w0 * kRowPieces + e) : make_uint4(0u, 0u, 0u, 0u);
         }
         __syncthreads();
         // ... then x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
@@ -156,8 +171,8 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
                 bool first;                                         // ch is the first channel of its rotation pair
                 if (layout == EA_ROPE_INTERLEAVED) { m = ch >> 1; first = (ch & 1) == 0; partner = ch ^ 1; }
                 else { m = ch < HALF ? ch : ch - HALF; first = ch < HALF; partner = first ? ch + HALF : ch - HALF; }
-                const float xa = __bfloat162float(raw[w * D + ch]) - mu_s[ch];
-                const float xb = __bfloat162float(raw[w * D + partner]) - mu_s[partner];
+                const float xa = to_f32(raw[w * D + ch]) - mu_s[ch];
+                const float xb = to_f32(raw[w * D + partner]) - mu_s[partner];
                 x = first ? c_s[m] * xa - s_s[m] * xb : s_s[m] * xb + c_s[m] * xa;
             }
             const __nv_bfloat16 hi = __float2bfloat16_rn(x);
@@ -215,9 +230,10 @@ stats_mma_kernel(const __nv_bfloat16* __restrict__ q_win, const float* __restric
 
 }  // namespace
 
-ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
-                          const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
-                          float* mu_bar, float* sigma_bar, cudaStream_t st) {
+template <typename QT>
+static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_win, const int64_t* pos_next,
+                              int n_future, double rope_base, float* rope_coef, float* mu_bar, float* sigma_bar,
+                              cudaStream_t st) {
     const int d = s.head_dim, half = d / 2;
     const int n_coef = s.n_units * half;
     rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, st>>>(pos_next, s.n_units, half, d, n_future,
@@ -225,30 +241,36 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
     const float inv_norm =
         1.0f / (float)(s.cov_norm == EA_COV_SAMPLE ? s.window - 1 : s.window);
     const unsigned heads = (unsigned)(s.n_units * s.n_q_heads);
+    auto launch = [&](auto kern, int smem, unsigned blocks_y) {
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+            return false;
+        kern<<<dim3(heads, blocks_y), 256, smem, st>>>(q_win, rope_coef, s.n_q_heads, s.window, s.rope_layout,
+                                                       inv_norm, mu_bar, sigma_bar);
+        return true;
+    };
+    bool ok;
     switch (d) {
-        case 64:
-            stats_mma_kernel<64><<<dim3(heads, 1), 256, stats_smem_bytes<64>(), st>>>(q_win, rope_coef, s.n_q_heads, s.window,
-                                                                s.rope_layout, inv_norm, mu_bar, sigma_bar);
-            break;
-        case 128:
-            if (cudaFuncSetAttribute(stats_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     stats_smem_bytes<128>()) != cudaSuccess)
-                return EA_ERR_CUDA;
-            stats_mma_kernel<128><<<dim3(heads, 1), 256, stats_smem_bytes<128>(), st>>>(q_win, rope_coef, s.n_q_heads, s.window,
-                                                                 s.rope_layout, inv_norm, mu_bar, sigma_bar);
-            break;
-        case 256:
-            if (cudaFuncSetAttribute(stats_mma_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     stats_smem_bytes<256>()) != cudaSuccess)
-                return EA_ERR_CUDA;
-            stats_mma_kernel<256><<<dim3(heads, 3), 256, stats_smem_bytes<256>(), st>>>(q_win, rope_coef, s.n_q_heads, s.window,
-                                                                 s.rope_layout, inv_norm, mu_bar, sigma_bar);
-            break;
-        default:
-            return EA_ERR_UNSUPPORTED;
+        case 64: ok = launch(stats_mma_kernel<64, QT>, stats_smem_bytes<64, QT>(), 1); break;
+        case 128: ok = launch(stats_mma_kernel<128, QT>, stats_smem_bytes<128, QT>(), 1); break;
+        case 256: ok = launch(stats_mma_kernel<256, QT>, stats_smem_bytes<256, QT>(), 3); break;
+        default: return EA_ERR_UNSUPPORTED;
     }
+    if (!ok) return EA_ERR_CUDA;
     ea_count_launches(ctx, 2);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
+                          const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
+                          float* mu_bar, float* sigma_bar, cudaStream_t st) {
+    return launch_stats(ctx, s, q_win, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st);
+}
+
+ea_status ea_launch_stats_f32(const ea_ctx* ctx, const ea_shape& s, const float* q_win, const int64_t* pos_next,
+                              int n_future, double rope_base, float* rope_coef, float* mu_bar, float* sigma_bar,
+                              cudaStream_t st) {
+    return launch_stats(ctx, s, q_win, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -319,21 +341,21 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
     const unsigned heads = (unsigned)(s->n_units * s->n_q_heads);
     switch (d) {
         case 64:
-            stats_mma_kernel<64><<<dim3(heads, 1), 256, stats_smem_bytes<64>(), stream>>>(q, coef, s->n_q_heads, s->window,
+            stats_mma_kernel<64, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<64, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         case 128:
-            if (cudaFuncSetAttribute(stats_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     stats_smem_bytes<128>()) != cudaSuccess)
+            if (cudaFuncSetAttribute(stats_mma_kernel<128, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     stats_smem_bytes<128, __nv_bfloat16>()) != cudaSuccess)
                 return EA_ERR_CUDA;
-            stats_mma_kernel<128><<<dim3(heads, 1), 256, stats_smem_bytes<128>(), stream>>>(q, coef, s->n_q_heads, s->window,
+            stats_mma_kernel<128, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<128, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
                                                                      s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
         default:
-            if (cudaFuncSetAttribute(stats_mma_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     stats_smem_bytes<256>()) != cudaSuccess)
+            if (cudaFuncSetAttribute(stats_mma_kernel<256, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     stats_smem_bytes<256, __nv_bfloat16>()) != cudaSuccess)
                 return EA_ERR_CUDA;
-            stats_mma_kernel<256><<<dim3(heads, 3), 256, stats_smem_bytes<256>(), stream>>>(q, coef, s->n_q_heads, s->window,
+            stats_mma_kernel<256, __nv_bfloat16><<<dim3(heads, 3), 256, stats_smem_bytes<256, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
                                                                      s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
     }

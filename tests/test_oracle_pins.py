@@ -64,12 +64,12 @@ def test_mean_cov_matches_numpy(oracle, norm):
 def test_hidden_statistics_equal_statistics_of_projected_samples(oracle, norm):
     """W_Q mu_h and W_Q Sigma_h W_Q^T against numpy's mean / cov of the explicitly projected rows."""
     rng = np.random.default_rng(31)
-    U, W, dm, Hq, d = 3, 11, 24, 2, 8
+    U, W, dm, Hq, d = 4, 11, 24, 2, 8          # two weight sets, units set-major: 0, 0, 1, 1
     hb, h = bf16_bits(rng.normal(size=(U, W, dm)) + rng.normal(size=(U, 1, dm)))
     wb, wq = bf16_bits(rng.normal(size=(2, Hq * d, dm)) / np.sqrt(dm))
     mu, sigma = oracle.hidden_mean_cov(hb, wb, Hq, cov_norm=norm)
     for u in range(U):
-        q = h[u] @ wq[u % 2].T                                     # [W, Hq*d]
+        q = h[u] @ wq[u // 2].T                                    # [W, Hq*d]
         for j in range(Hq):
             qj = q[:, j * d:(j + 1) * d]
             np.testing.assert_allclose(mu[u, j], qj.mean(0), rtol=1e-12, atol=1e-13)
@@ -294,7 +294,7 @@ def test_scores_with_output_projection(oracle):
         for u in range(U):
             for h in range(Hq):
                 g = h // G
-                y = v[u, g] @ wo[u % 2][:, h * d:(h + 1) * d].T          # [n, dm]
+                y = v[u, g] @ wo[u][:, h * d:(h + 1) * d].T              # [n, dm]; one set per unit
                 want[u, g] += (a_hat[u, h] + 0.02) * np.linalg.norm(y, axis=-1)
         if mode == 0:
             want /= G

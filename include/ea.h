@@ -215,6 +215,36 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
                    float* logits_opt, void* cuda_stream);
 
 /*
+ * Contribution scores with the output projection (Eq. 9 as written:
+ * (a_hat + epsilon) * ||W_o v||; the paper's experiments drop W_o, see
+ * ea_score).  Query head h multiplies the value it reads by its own slice
+ * W_o^h = W_o[:, h*d : (h+1)*d], so per query head
+ *   c_{h,i} = (a_hat_{h,i} + epsilon) * ||W_o^h v_{g,i}||_2,
+ * reduced over the G heads of KV head g like the attention itself (mean for
+ * EA_GROUP_MEAN_PROB, sum for EA_GROUP_SUM_PROB; EA_GROUP_MEAN_LOGIT has no
+ * per-head attention: EA_ERR_UNSUPPORTED).  ||W_o^h v||^2 = v^T M_h v with the
+ * Gram matrix M_h = W_o^h^T W_o^h, which ea_wo_gram computes once per model;
+ * the quadratic form runs on the same tensor-core kernel as Eq. 7, with the
+ * value rows in place of the keys.
+ *
+ * ea_wo_gram
+ *   w_o      bf16 [n_weight_sets, d_model, Hq * d]  output projections (row =
+ *            output channel), 16-byte aligned
+ *   wo_gram  fp32 [n_weight_sets, Hq, d, d]  (output)
+ * ea_score_wo: the arguments of ea_score, plus
+ *   wo_gram, n_weight_sets   as above; units are set-major: unit u uses set
+ *            u / (n_units / n_weight_sets); n_weight_sets must divide n_units
+ *   wo_scratch fp32 [n_units, Hq, n]  caller-owned scratch; holds
+ *            ||W_o^h v_i||^2 on return
+ */
+ea_status ea_wo_gram(ea_ctx* ctx, const void* w_o, int32_t d_model, int32_t n_weight_sets,
+                     int32_t n_q_heads, int32_t head_dim, float* wo_gram, void* cuda_stream);
+ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
+                      const float* mu_bar, const float* sigma_bar, const float* wo_gram,
+                      int32_t n_weight_sets, float epsilon, float* wo_scratch, float* scores,
+                      float* logits_opt, void* cuda_stream);
+
+/*
  * Eviction and compaction: per (unit, KV head) keep the n_kept pairs with the
  * highest score; among equal scores the lowest index wins; kept indices are
  * emitted in ascending order (the cache keeps its temporal order) and the

@@ -24,7 +24,7 @@ EXPORTS = (
     "ea_version", "ea_status_string", "ea_workspace_bytes", "ea_n_kept", "ea_create", "ea_destroy",
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
-    "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden",
+    "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.ea_query_stats_hidden.argtypes = [vp, sp, vp, vp, i32, i32, vp, vp, i32, f64, vp, vp, vp]
         L.ea_query_stats_hidden.restype = ctypes.c_int
         L.ea_score.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
+        L.ea_wo_gram.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp]
+        L.ea_wo_gram.restype = ctypes.c_int
+        L.ea_score_wo.argtypes = [vp, sp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
+        L.ea_score_wo.restype = ctypes.c_int
         L.ea_select_compact.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.ea_select_compact_adaptive.argtypes = [vp, sp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.ea_n_floor.argtypes = [i64, f64]
@@ -238,6 +242,40 @@ def ea_score(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, epsilon: float
     _check(lib().ea_score(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(mu_bar), _ptr(sigma_bar),
                           float(epsilon), _ptr(scores), _ptr(logits), _stream(ctx.device)), "ea_score")
     return (scores, logits) if (want_logits or logits is not None) else scores
+
+
+def ea_wo_gram(ctx: Context, w_o, n_q_heads: int, head_dim: int, wo_gram=None):
+    """w_o bf16 [sets, d_model, Hq*d] -> Gram matrices fp32 [sets, Hq, d, d] of the per-head slices."""
+    _dev_tensor(w_o, torch.bfloat16, "w_o")
+    sets, d_model, cols = w_o.shape
+    if cols != n_q_heads * head_dim:
+        raise ValueError("w_o must be [sets, d_model, Hq * d]")
+    if wo_gram is None:
+        wo_gram = torch.empty((sets, n_q_heads, head_dim, head_dim), dtype=torch.float32, device=w_o.device)
+    _check(lib().ea_wo_gram(ctx._h, _ptr(w_o), int(d_model), int(sets), int(n_q_heads), int(head_dim),
+                            _ptr(wo_gram), _stream(ctx.device)), "ea_wo_gram")
+    return wo_gram
+
+
+def ea_score_wo(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, wo_gram, epsilon: float, scores=None,
+                wo_scratch=None, logits=None, want_logits: bool = False):
+    """As ea_score with ||W_o^h v|| per query head in place of ||v||; returns (scores, wo_scratch[, logits])."""
+    _dev_tensor(k, torch.bfloat16, "k")
+    _dev_tensor(v, torch.bfloat16, "v")
+    _dev_tensor(mu_bar, torch.float32, "mu_bar")
+    _dev_tensor(sigma_bar, torch.float32, "sigma_bar")
+    _dev_tensor(wo_gram, torch.float32, "wo_gram")
+    U, Hq, Hkv, n = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys
+    if scores is None:
+        scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=k.device)
+    if wo_scratch is None:
+        wo_scratch = torch.empty((U, Hq, n), dtype=torch.float32, device=k.device)
+    if logits is None and want_logits:
+        logits = torch.empty((U, Hq, n), dtype=torch.float32, device=k.device)
+    _check(lib().ea_score_wo(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(mu_bar), _ptr(sigma_bar),
+                             _ptr(wo_gram), int(wo_gram.shape[0]), float(epsilon), _ptr(wo_scratch), _ptr(scores),
+                             _ptr(logits), _stream(ctx.device)), "ea_score_wo")
+    return (scores, wo_scratch, logits) if want_logits else (scores, wo_scratch)
 
 
 def ea_select_compact(ctx: Context, shape: Shape, scores, n_kept: int, k=None, v=None, kept_idx=None,

@@ -234,25 +234,88 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
     const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
+    const ea_quad_form eq7 = ea_eq7_form(*shape, mu_bar, sigma_bar);
     if (ea_mma_path_supported(*shape) && shape->group_mode != EA_GROUP_MEAN_LOGIT) {
         // tensor-core log-scores with the log-sum-exp partials from their epilogue
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
         int n_chunks = 0;
-        st = ea_launch_logits_mma(ctx, *shape, kb, mu_bar, sigma_bar, ws + plan.image,
+        st = ea_launch_logits_mma(ctx, *shape, kb, eq7, ws + plan.image,
                                   reinterpret_cast<float*>(ws + plan.vec), logits, lse_part, &n_chunks, stream);
         if (st == EA_OK) st = ea_launch_lse_combine(ctx, *shape, lse_part, n_chunks, lse, stream);
         if (st == EA_OK) st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, true, scores, stream);
     } else {
         if (ea_mma_path_supported(*shape)) {
             int n_chunks = 0;
-            st = ea_launch_logits_mma(ctx, *shape, kb, mu_bar, sigma_bar, ws + plan.image,
+            st = ea_launch_logits_mma(ctx, *shape, kb, eq7, ws + plan.image,
                                       reinterpret_cast<float*>(ws + plan.vec), logits,
                                       reinterpret_cast<float*>(ws + plan.lse_part), &n_chunks, stream);
         } else {
-            st = ea_launch_logits_simt(ctx, *shape, kb, mu_bar, sigma_bar, logits, stream);
+            st = ea_launch_logits_simt(ctx, *shape, kb, eq7, logits, stream);
         }
         if (st == EA_OK) st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, false, scores, stream);
     }
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_wo_gram(ea_ctx* ctx, const void* w_o, int32_t d_model, int32_t n_weight_sets, int32_t n_q_heads,
+                     int32_t head_dim, float* wo_gram, void* cuda_stream) {
+    if (!ctx || !w_o || !wo_gram) return EA_ERR_INVALID_ARG;
+    if (d_model < 1 || n_weight_sets < 1 || n_q_heads < 1) return EA_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128 && head_dim != 256) return EA_ERR_INVALID_ARG;
+    if (!aligned16(w_o) || !aligned16(wo_gram)) return EA_ERR_INVALID_ARG;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    const ea_status st = ea_launch_wo_gram(ctx, static_cast<const __nv_bfloat16*>(w_o), d_model, n_weight_sets,
+                                           n_q_heads, head_dim, wo_gram, static_cast<cudaStream_t>(cuda_stream));
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v, const float* mu_bar,
+                      const float* sigma_bar, const float* wo_gram, int32_t n_weight_sets, float epsilon,
+                      float* wo_scratch, float* scores, float* logits_opt, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (shape->group_mode == EA_GROUP_MEAN_LOGIT) return EA_ERR_UNSUPPORTED;   // the weighting is per query head
+    if (shape->n_units == 0 || shape->n_keys == 0) return EA_OK;
+    if (!k || !v || !mu_bar || !sigma_bar || !wo_gram || !wo_scratch || !scores) return EA_ERR_INVALID_ARG;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(mu_bar) || !aligned16(sigma_bar) || !aligned16(wo_gram) ||
+        !aligned16(wo_scratch) || !aligned16(scores) || !aligned16(logits_opt))
+        return EA_ERR_INVALID_ARG;
+    if (!(epsilon >= 0.0f)) return EA_ERR_INVALID_ARG;
+    if (n_weight_sets < 1 || shape->n_units % n_weight_sets != 0) return EA_ERR_INVALID_ARG;
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    if (ctx->workspace_bytes < plan.total) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    char* ws = static_cast<char*>(ctx->workspace);
+    float* logits = logits_opt ? logits_opt : reinterpret_cast<float*>(ws + plan.logits);
+    float* lse = reinterpret_cast<float*>(ws + plan.lse);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+    const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
+    const ea_quad_form eq7 = ea_eq7_form(*shape, mu_bar, sigma_bar);
+    // ||W_o^h v||^2 = v^T (W_o^h^T W_o^h) v: the same kernels, the value rows in place of the keys
+    const ea_quad_form norm2 = {nullptr, wo_gram, shape->n_units / n_weight_sets, 0.0f, 1.0f};
+    if (ea_mma_path_supported(*shape)) {
+        float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
+        float* vec = reinterpret_cast<float*>(ws + plan.vec);
+        int n_chunks = 0;
+        st = ea_launch_logits_mma(ctx, *shape, vb, norm2, ws + plan.image, vec, wo_scratch, lse_part, &n_chunks,
+                                  stream);
+        if (st == EA_OK)
+            st = ea_launch_logits_mma(ctx, *shape, kb, eq7, ws + plan.image, vec, logits, lse_part, &n_chunks, stream);
+        if (st == EA_OK) st = ea_launch_lse_combine(ctx, *shape, lse_part, n_chunks, lse, stream);
+    } else {
+        st = ea_launch_logits_simt(ctx, *shape, vb, norm2, wo_scratch, stream);
+        if (st == EA_OK) st = ea_launch_logits_simt(ctx, *shape, kb, eq7, logits, stream);
+        if (st == EA_OK) st = ea_launch_lse(ctx, *shape, logits, lse, stream);
+    }
+    if (st == EA_OK) st = ea_launch_finalize_wo(ctx, *shape, logits, lse, wo_scratch, epsilon, scores, stream);
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

@@ -4,6 +4,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -67,9 +68,23 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
                           const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
                           float* mu_bar, float* sigma_bar, cudaStream_t st);
 
+// What the log-score kernels evaluate per (query head h, row x of the KV head it reads):
+//   lin_scale * lin_h . x + quad_scale * x^T quad_h x
+// Eq. 7: rows = keys, lin = mu_bar, quad = sigma_bar, scales 1/sqrt(d) and 1/(2d), one matrix per unit;
+// ||W_o^h v||^2: rows = values, no linear term, quad = W_o^h^T W_o^h shared by the units of a weight set.
+struct ea_quad_form {
+    const float* lin;        // fp32 [sets * Hq, d] or nullptr
+    const float* quad;       // fp32 [sets * Hq, d, d]
+    int units_per_set;       // unit u reads set u / units_per_set
+    float lin_scale, quad_scale;
+};
+static inline ea_quad_form ea_eq7_form(const ea_shape& s, const float* mu_bar, const float* sigma_bar) {
+    ea_quad_form f = {mu_bar, sigma_bar, 1, 1.0f / sqrtf((float)s.head_dim), 0.5f / (float)s.head_dim};
+    return f;
+}
+
 ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
-                                const float* mu_bar, const float* sigma_bar, float* logits,
-                                cudaStream_t st);
+                                const ea_quad_form& form, float* logits, cudaStream_t st);
 
 // bf16 rank-3 TMA tensor map, box (box0 x box1 x 1), 128-byte swizzle, zero fill outside.
 bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint64_t n1, uint64_t n2,
@@ -90,7 +105,7 @@ size_t ea_mma_image_bytes(const ea_shape& s);
 size_t ea_mma_vec_bytes(const ea_shape& s);
 size_t ea_mma_lse_part_bytes(const ea_shape& s);
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
-                               const float* mu_bar, const float* sigma_bar, void* image, float* vec,
+                               const ea_quad_form& form, void* image, float* vec,
                                float* logits, float* lse_part, int* n_chunks, cudaStream_t st);
 // log-sum-exp per softmax row from the per-work-unit partials of the tensor-core kernel
 ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const float* lse_part, int n_chunks,
@@ -99,6 +114,14 @@ ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const floa
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
                              const __nv_bfloat16* v, float epsilon, float* lse, bool lse_ready, float* scores,
                              cudaStream_t st);
+
+// Eq. 9 with the output projection: Gram matrices of the per-head slices of W_o, and the
+// weighting (1/G) sum_h (a_hat_h + eps) sqrt(wo_norm2_h).
+ea_status ea_launch_wo_gram(const ea_ctx* ctx, const __nv_bfloat16* w_o, int d_model, int n_sets, int Hq, int d,
+                            float* gram, cudaStream_t st);
+ea_status ea_launch_lse(const ea_ctx* ctx, const ea_shape& s, const float* logits, float* lse, cudaStream_t st);
+ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
+                                const float* wo_norm2, float epsilon, float* scores, cudaStream_t st);
 
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
                            int32_t* kept_idx, cudaStream_t st);

@@ -120,6 +120,50 @@ finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
 }
 
 
+// score = group reduction of (a_hat_h + eps) * sqrt(wo_norm2_h) over the query heads of the KV head
+// (Eq. 9 with ||W_o v||); one thread per key.
+__global__ void __launch_bounds__(256)
+finalize_wo_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
+                   const float* __restrict__ wo_norm2, int Hq, int Hkv, int n, int group_mode, float epsilon,
+                   float* __restrict__ scores) {
+    const int G = Hq / Hkv;
+    const int ug = blockIdx.y;
+    const int u = ug / Hkv, g = ug % Hkv;
+    const int key = blockIdx.x * blockDim.x + threadIdx.x;
+    if (key >= n) return;
+    float acc = 0.f;
+    for (int j = 0; j < G; ++j) {
+        const size_t uh = (size_t)u * Hq + (size_t)g * G + j;
+        const float a = expf(logits[uh * n + key] - lse[uh]);
+        acc += (a + epsilon) * sqrtf(fmaxf(wo_norm2[uh * n + key], 0.f));   // rounding can leave -0 or a tiny negative
+    }
+    if (group_mode == EA_GROUP_MEAN_PROB) acc *= 1.0f / (float)G;
+    scores[(size_t)ug * n + key] = acc;
+}
+
+// Gram matrix of head j's slice of the output projection: M_j[c, e] = sum_a W_o[a, j*d + c] W_o[a, j*d + e].
+// One CTA per (set, head, 16 x 16 block of M_j); done once per model, not on the scoring path.
+__global__ void __launch_bounds__(256)
+wo_gram_kernel(const __nv_bfloat16* __restrict__ w_o, int d_model, int Hq, int d, float* __restrict__ gram) {
+    __shared__ float a_s[16][17], b_s[16][17];
+    const int blocks = d / 16;
+    const int bc = blockIdx.x / blocks, be = blockIdx.x % blocks;
+    const int j = blockIdx.y, set = blockIdx.z;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const __nv_bfloat16* W = w_o + (size_t)set * d_model * Hq * d + (size_t)j * d;
+    float acc = 0.f;
+    for (int a0 = 0; a0 < d_model; a0 += 16) {
+        const int a = a0 + ty;
+        a_s[ty][tx] = a < d_model ? __bfloat162float(W[(size_t)a * Hq * d + bc * 16 + tx]) : 0.f;
+        b_s[ty][tx] = a < d_model ? __bfloat162float(W[(size_t)a * Hq * d + be * 16 + tx]) : 0.f;
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < 16; ++r) acc = fmaf(a_s[r][ty], b_s[r][tx], acc);
+        __syncthreads();
+    }
+    gram[(((size_t)set * Hq + j) * d + bc * 16 + ty) * d + be * 16 + tx] = acc;
+}
+
 // One thread per softmax row: combine the (max, sum of exp) partials of its work units in order.
 __global__ void lse_combine_kernel(const float* __restrict__ lse_part, int n_rows, int n_chunks,
                                    float* __restrict__ lse) {
@@ -178,6 +222,31 @@ ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const floa
                                 float* lse, cudaStream_t st) {
     const int rows = s.n_units * s.n_q_heads;
     lse_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(lse_part, rows, n_chunks, lse);
+    ea_count_launches(ctx, 1);
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+ea_status ea_launch_lse(const ea_ctx* ctx, const ea_shape& s, const float* logits, float* lse, cudaStream_t st) {
+    lse_kernel<<<s.n_units * s.n_q_heads, kLseThreads, 0, st>>>(logits, s.n_keys, 1, lse);
+    ea_count_launches(ctx, 1);
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
+                                const float* wo_norm2, float epsilon, float* scores, cudaStream_t st) {
+    dim3 grid((unsigned)((s.n_keys + 255) / 256), (unsigned)(s.n_units * s.n_kv_heads));
+    finalize_wo_kernel<<<grid, 256, 0, st>>>(logits, lse, wo_norm2, s.n_q_heads, s.n_kv_heads, s.n_keys,
+                                             s.group_mode, epsilon, scores);
+    ea_count_launches(ctx, 1);
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+ea_status ea_launch_wo_gram(const ea_ctx* ctx, const __nv_bfloat16* w_o, int d_model, int n_sets, int Hq, int d,
+                            float* gram, cudaStream_t st) {
+    const int blocks = d / 16;
+    dim3 grid((unsigned)(blocks * blocks), (unsigned)Hq, (unsigned)n_sets);
+    if (grid.y > 65535u || grid.z > 65535u) return EA_ERR_UNSUPPORTED;
+    wo_gram_kernel<<<grid, 256, 0, st>>>(w_o, d_model, Hq, d, gram);
     ea_count_launches(ctx, 1);
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

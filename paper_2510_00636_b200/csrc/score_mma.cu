@@ -86,8 +86,8 @@ struct MmaParams {
 // Covariance image and epilogue vectors.  One CTA per query head.
 template <int D>
 __global__ void __launch_bounds__(256)
-sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ sigma_bar, int Hq, int Hkv,
-                   uint8_t* __restrict__ image, float* __restrict__ vec) {
+sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict__ image,
+                   float* __restrict__ vec) {
     using G = Geo<D, true>;
     const int uh = blockIdx.x;
     const int u = uh / Hq, h = uh % Hq;
@@ -95,9 +95,10 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
     const int g = h / Gq, hg = h % Gq;
     const int n_subsets = (Gq + G::HPC - 1) / G::HPC;
     const int hs = hg / G::HPC, j = hg % G::HPC;
-    const float* S = sigma_bar + (size_t)uh * D * D;
+    const size_t set_head = (size_t)(u / form.units_per_set) * Hq + h;
+    const float* S = form.quad + set_head * D * D;
     uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG_FULL;   // 16-byte aligned
-    const float inv_d = 1.0f / (float)D;       // a power of two: the scaling is exact
+    const float quad_scale = form.quad_scale;  // 1/(2d) for Eq. 7, a power of two: the scaling is exact
 
     // one 16-byte unit (8 consecutive a) of one row c per thread step
     for (int e = threadIdx.x; e < D * (D / 8); e += blockDim.x) {
@@ -113,7 +114,7 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
                 if (a != c) {
                     // Sigma_ac / d (the two mirrored entries together carry 2 Sigma_ac / (2d)),
                     // split into a bf16 and the bf16 rounding of its remainder
-                    const float x = (S[(size_t)c * D + a] + S[(size_t)a * D + c]) * (0.5f * inv_d);
+                    const float x = (S[(size_t)c * D + a] + S[(size_t)a * D + c]) * quad_scale;
                     const float hi = __bfloat162float(__float2bfloat16_rn(x));
                     val = a < c ? hi : x - hi;
                 }
@@ -130,9 +131,8 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
     // linear-term operand: row (j, c) holds mu_bar_c / sqrt(d) as a bf16 and the bf16 of its remainder in
     // K columns 0 and 1, zeros elsewhere; unswizzled core-matrix layout (8 rows x 16 bytes, K columns
     // 8..15 another 128 bytes on, next 8 rows 256 bytes on)
-    const float inv_sqrt_d = rsqrtf((float)D), inv_2d = 0.5f / (float)D;
     for (int c = threadIdx.x; c < D; c += blockDim.x) {
-        const float m = mu_bar[(size_t)uh * D + c] * inv_sqrt_d;
+        const float m = form.lin ? form.lin[set_head * D + c] * form.lin_scale : 0.f;
         const __nv_bfloat16 hi = __float2bfloat16_rn(m);
         const __nv_bfloat16 lo = __float2bfloat16_rn(m - __bfloat162float(hi));
         const int row = j * D + c;
@@ -140,7 +140,7 @@ sigma_image_kernel(const float* __restrict__ mu_bar, const float* __restrict__ s
         *reinterpret_cast<uint4*>(dst) =
             make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
         *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
-        vec[(size_t)uh * D + c] = S[(size_t)c * D + c] * inv_2d;
+        vec[(size_t)uh * D + c] = S[(size_t)c * D + c] * quad_scale;
     }
 }
 
@@ -582,9 +582,9 @@ bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, long lon
 }
 
 template <int D, bool PAIR>
-ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k, const float* mu_bar,
-                     const float* sigma_bar, uint8_t* image, float* vec, float* logits, float* lse_part,
-                     int* n_chunks_out, cudaStream_t st) {
+ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k, const ea_quad_form& form,
+                     uint8_t* image, float* vec, float* logits, float* lse_part, int* n_chunks_out,
+                     cudaStream_t st) {
     using G = Geo<D, PAIR>;
     const int Gq = s.n_q_heads / s.n_kv_heads;
     constexpr int keys_per_step = PAIR ? 2 * kTileKeys : kTileKeys;
@@ -616,8 +616,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     CUtensorMap k_map;
     if (!make_k_map(&k_map, k, D, s.n_keys, (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
 
-    sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(mu_bar, sigma_bar, s.n_q_heads, s.n_kv_heads,
-                                                                 image, vec);
+    sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(form, s.n_q_heads, s.n_kv_heads, image, vec);
     auto kern = logits_mma_kernel<D, PAIR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM) != cudaSuccess)
         return EA_ERR_CUDA;
@@ -696,16 +695,16 @@ size_t ea_mma_lse_part_bytes(const ea_shape& s) {
 }
 
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
-                               const float* mu_bar, const float* sigma_bar, void* image, float* vec,
+                               const ea_quad_form& form, void* image, float* vec,
                                float* logits, float* lse_part, int* n_chunks, cudaStream_t st) {
     uint8_t* img = static_cast<uint8_t*>(image);
     switch (s.head_dim) {
         case 64:
-            return launch_mma<64, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, lse_part, n_chunks, st);
+            return launch_mma<64, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
         case 128:
-            return launch_mma<128, false>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, lse_part, n_chunks, st);
+            return launch_mma<128, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
         case 256:
-            return launch_mma<256, true>(ctx, s, k, mu_bar, sigma_bar, img, vec, logits, lse_part, n_chunks, st);
+            return launch_mma<256, true>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
         default:
             return EA_ERR_UNSUPPORTED;
     }

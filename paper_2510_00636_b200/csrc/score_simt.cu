@@ -13,8 +13,7 @@ constexpr int kKeysPerCta = (kThreads / 32) * kKeysPerWarp;   // 64
 
 template <int D>
 __global__ void __launch_bounds__(kThreads)
-logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const float* __restrict__ mu_bar,
-                   const float* __restrict__ sigma_bar, int Hq, int Hkv, int n,
+logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form, int Hq, int Hkv, int n,
                    float* __restrict__ logits) {
     constexpr int CT = D / 32;
     __shared__ __nv_bfloat16 k_s[kKeysPerCta][D];
@@ -23,8 +22,9 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const float* __restrict_
     const int u = uh / Hq, h = uh % Hq, g = h / (Hq / Hkv);
     const int key0 = blockIdx.x * kKeysPerCta;
     const __nv_bfloat16* kk = k + ((size_t)u * Hkv + g) * (size_t)n * D;
-    const float* S = sigma_bar + (size_t)uh * D * D;
-    const float* mu = mu_bar + (size_t)uh * D;
+    const size_t set_head = (size_t)(u / form.units_per_set) * Hq + h;
+    const float* S = form.quad + set_head * D * D;
+    const float* mu = form.lin ? form.lin + set_head * D : nullptr;
 
     for (int e = threadIdx.x; e < kKeysPerCta * D; e += kThreads) {
         int r = e / D, c = e % D;
@@ -52,11 +52,11 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const float* __restrict_
         }
     }
 
-    const float inv_sqrt_d = 1.0f / sqrtf((float)D);
-    const float inv_2d = 0.5f / (float)D;
+    const float inv_sqrt_d = form.lin_scale;
+    const float inv_2d = form.quad_scale;
     float mu_r[CT];
 #pragma unroll
-    for (int j = 0; j < CT; ++j) mu_r[j] = mu[lane + 32 * j] * inv_sqrt_d;
+    for (int j = 0; j < CT; ++j) mu_r[j] = mu ? mu[lane + 32 * j] * inv_sqrt_d : 0.f;
 #pragma unroll
     for (int i = 0; i < kKeysPerWarp; ++i) {
         float acc = 0.f;
@@ -73,25 +73,23 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const float* __restrict_
 }  // namespace
 
 ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
-                                const float* mu_bar, const float* sigma_bar, float* logits,
-                                cudaStream_t st) {
+                                const ea_quad_form& form, float* logits, cudaStream_t st) {
     ea_count_launches(ctx, 1);
     cudaEvent_t stop = ea_profile_mark_start(ctx, st);
     dim3 grid((unsigned)((s.n_keys + kKeysPerCta - 1) / kKeysPerCta),
               (unsigned)(s.n_units * s.n_q_heads));
     switch (s.head_dim) {
         case 64:
-            logits_simt_kernel<64><<<grid, kThreads, 0, st>>>(k, mu_bar, sigma_bar, s.n_q_heads,
+            logits_simt_kernel<64><<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads,
                                                              s.n_kv_heads, s.n_keys, logits);
             break;
         case 128:
-            logits_simt_kernel<128><<<grid, kThreads, 0, st>>>(k, mu_bar, sigma_bar, s.n_q_heads,
+            logits_simt_kernel<128><<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads,
                                                               s.n_kv_heads, s.n_keys, logits);
             break;
         case 256: {
             auto kern = logits_simt_kernel<256>;
-            kern<<<grid, kThreads, 0, st>>>(k, mu_bar, sigma_bar, s.n_q_heads, s.n_kv_heads, s.n_keys,
-                                            logits);
+            kern<<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads, s.n_kv_heads, s.n_keys, logits);
             break;
         }
         default:

@@ -119,9 +119,11 @@ class ClockSampler:
 class Workload:
     """All layers of one config resident in HBM, plus preallocated outputs."""
 
-    def __init__(self, cfg: inputs.EAConfig, device, ea, safeguard=None):
+    def __init__(self, cfg: inputs.EAConfig, device, ea, safeguard=None, hidden_dm=None, wo_dm=None):
         self.cfg, self.device, self.ea = cfg, device, ea
         self.safeguard = safeguard          # None: n_kept per head; else head-adaptive with this safeguard share
+        self.hidden_dm = hidden_dm          # statistics from hidden states of this width through W_Q
+        self.wo_dm = wo_dm                  # ||W_o v|| weighting with an output projection of this width
         L, B = cfg.n_layers, cfg.batch
         U, Hq, Hkv, d, n, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window
         bf, f32 = torch.bfloat16, torch.float32
@@ -142,6 +144,22 @@ class Workload:
         self.v_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
         self.head_off = torch.empty((U, Hkv + 1), dtype=torch.int32, device=device)
         self.n_units = U
+        gen = torch.Generator(device=device).manual_seed(1234)
+        if hidden_dm:
+            # synthetic stand-ins: Gaussian hidden states with a per-channel offset, Gaussian projections (one per layer)
+            self.hidden = (torch.randn((U, W, hidden_dm), device=device, generator=gen) +
+                           0.5 * torch.randn((U, 1, hidden_dm), device=device, generator=gen)).to(bf)
+            self.w_q = torch.empty((L, Hq * d, hidden_dm), dtype=bf, device=device)
+            for layer in range(L):
+                self.w_q[layer] = (torch.randn((Hq * d, hidden_dm), device=device, generator=gen) /
+                                   hidden_dm ** 0.5).to(bf)
+            self.q_scratch = torch.empty((U, Hq, W, d), dtype=f32, device=device)
+        if wo_dm:
+            self.w_o = torch.empty((L, wo_dm, Hq * d), dtype=bf, device=device)
+            for layer in range(L):
+                self.w_o[layer] = (torch.randn((wo_dm, Hq * d), device=device, generator=gen) / wo_dm ** 0.5).to(bf)
+            self.wo_scratch = torch.empty((U, Hq, n), dtype=f32, device=device)
+            self.wo_gram = None             # computed once (model-load work), outside the timed region
 
     def make_ctx(self, units_per_call):
         cfg = self.cfg
@@ -155,10 +173,23 @@ class Workload:
         for u0 in range(0, self.n_units, units_per_call):
             u1 = min(self.n_units, u0 + units_per_call)
             shape = ea.make_shape(u1 - u0, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window)
-            ea.ea_query_stats(ctx, shape, self.q[u0:u1], self.pos[u0:u1], cfg.n_future, cfg.rope_base,
-                              self.mu[u0:u1], self.sigma[u0:u1])
-            ea.ea_score(ctx, shape, self.k[u0:u1], self.v[u0:u1], self.mu[u0:u1], self.sigma[u0:u1], cfg.eps,
-                        self.scores[u0:u1])
+            B = cfg.batch
+            if self.hidden_dm:
+                ea.ea_query_stats_hidden(ctx, shape, self.hidden[u0:u1], self.w_q[u0 // B:(u1 + B - 1) // B],
+                                         self.pos[u0:u1], cfg.n_future, cfg.rope_base, self.q_scratch[u0:u1],
+                                         self.mu[u0:u1], self.sigma[u0:u1])
+            else:
+                ea.ea_query_stats(ctx, shape, self.q[u0:u1], self.pos[u0:u1], cfg.n_future, cfg.rope_base,
+                                  self.mu[u0:u1], self.sigma[u0:u1])
+            if self.wo_dm:
+                if self.wo_gram is None:
+                    self.wo_gram = ea.ea_wo_gram(ctx, self.w_o, cfg.n_q_heads, cfg.head_dim)
+                ea.ea_score_wo(ctx, shape, self.k[u0:u1], self.v[u0:u1], self.mu[u0:u1], self.sigma[u0:u1],
+                               self.wo_gram[u0 // B:(u1 + B - 1) // B], cfg.eps, self.scores[u0:u1],
+                               self.wo_scratch[u0:u1])
+            else:
+                ea.ea_score(ctx, shape, self.k[u0:u1], self.v[u0:u1], self.mu[u0:u1], self.sigma[u0:u1], cfg.eps,
+                            self.scores[u0:u1])
             if self.safeguard is None:
                 ea.ea_select_compact(ctx, shape, self.scores[u0:u1], cfg.n_kept, self.k[u0:u1], self.v[u0:u1],
                                      self.idx[u0:u1], self.k_out[u0:u1], self.v_out[u0:u1])
@@ -348,6 +379,11 @@ def main():
     ap.add_argument("--head-adaptive", type=float, default=None, metavar="SAFEGUARD",
                     help="prefill configs: head-adaptive eviction with this safeguard share (e.g. 0.2) in place of "
                          "n_kept per head; the device-resident line only")
+    ap.add_argument("--hidden-stats", type=int, default=None, metavar="D_MODEL",
+                    help="prefill configs: statistics from buffered hidden states of this width through W_Q "
+                         "(ea_query_stats_hidden) in place of given window queries")
+    ap.add_argument("--with-wo", type=int, default=None, metavar="D_MODEL",
+                    help="prefill configs: weight by ||W_o v|| (ea_score_wo) with an output projection of this width")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -372,14 +408,18 @@ def main():
     ea.lib()
 
     decode = cfg.cfg_id == 4
-    if args.head_adaptive is not None and decode:
-        raise SystemExit("--head-adaptive applies to the prefill configs")
-    wl = DecodeWorkload(cfg, device, ea) if decode else Workload(cfg, device, ea, args.head_adaptive)
+    variant = args.head_adaptive is not None or args.hidden_stats or args.with_wo
+    if variant and decode:
+        raise SystemExit("--head-adaptive, --hidden-stats and --with-wo apply to the prefill configs")
+    wl = DecodeWorkload(cfg, device, ea) if decode else Workload(cfg, device, ea, args.head_adaptive,
+                                                                 args.hidden_stats, args.with_wo)
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
     slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg)
-    if args.head_adaptive is not None:
-        args.skip_e2e = True           # the host-buffer entry point evicts n_kept per head
+    if variant:
+        args.skip_e2e = True           # the host-buffer entry point runs the three basic calls
+    if args.with_wo:
+        alg_flops *= 2                 # v^T (W_o^T W_o) v per query head is a second quadratic form
     if decode:
         args.skip_e2e = True           # the host-buffer leg is defined for the prefill configs
     peaks = measured_peaks()
@@ -411,7 +451,8 @@ def main():
     # roofline of the dominant kernel (the log-score kernel, Eq. 7)
     n_calls = len(wl.events) if decode else (wl.n_units + upc - 1) // upc
     avg_score_ms = score_ms / max(1, score_launches)
-    flops_per_launch = alg_flops / n_calls
+    # (with --with-wo the kernel runs twice per call, once per quadratic form, each with the FLOPs of Eq. 7)
+    flops_per_launch = alg_flops / (2 if args.with_wo else 1) / n_calls
     bytes_per_launch = slots * 2 * cfg.head_dim / n_calls            # the K rows this kernel must read
     t_tensor = flops_per_launch / (peaks["tflops"] * 1e12)
     t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
@@ -443,6 +484,9 @@ def main():
                    "n_keys": cfg.n_keys, "window": cfg.window, "n_kept": cfg.n_kept,
                    "eviction": "n_kept per head" if args.head_adaptive is None else
                                "head-adaptive, safeguard share %g" % args.head_adaptive,
+                   "statistics": "window queries given" if not args.hidden_stats else
+                                 "hidden states through W_Q, d_model %d" % args.hidden_stats,
+                   "value_weight": "||v||" if not args.with_wo else "||W_o v||, d_model %d" % args.with_wo,
                    "key_slots_per_step": slots, "units_per_call": upc, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (K+V %.1f GB per step)" % (slots * 4 * cfg.head_dim / 1e9)},
         "ms_per_128k_compression": ms if cfg.cfg_id == 3 else None,

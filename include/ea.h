@@ -262,6 +262,27 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
                             void* k_out, void* v_out, void* cuda_stream);
 
 /*
+ * Eviction with compaction inside the cache (for a cache that lives in a
+ * fixed buffer and is compressed periodically while decoding, as in the
+ * paper's decoding set-up): the selection of ea_select_compact, then the kept
+ * rows of every head are moved, in order, to the front of that head's range:
+ *   k[u, g, j, :] <- k[u, g, kept_idx[u, g, j], :]   for j < n_kept, same for v.
+ * Rows n_kept .. n-1 of each head keep whatever they held (the caller's cache
+ * length becomes n_kept; new pairs are appended from there).  kept_idx still
+ * refers to the positions before the call.
+ *
+ * k, v      bf16 [n_units, Hkv, n, d], 16-byte aligned, modified in place;
+ *           two distinct buffers
+ * kept_idx  int32 [n_units, Hkv, n_kept]  (output)
+ * The call records only stream work and no allocation, so a sequence of
+ * ea_query_stats / ea_score / ea_select_compact_inplace can be captured into
+ * a CUDA graph and replayed for every compression event of the same shape.
+ */
+ea_status ea_select_compact_inplace(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                                    int32_t n_kept, void* k, void* v, int32_t* kept_idx,
+                                    void* cuda_stream);
+
+/*
  * Head-adaptive eviction and compaction (the "Head-Adaptive Compression"
  * paragraph of Sec. 2.2: the per-layer budget allocation of Ada-KV, so that
  * heads whose pairs matter more retain more of them).  The paper prints no

@@ -25,6 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
+    "ea_select_compact_inplace",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -78,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.ea_select_compact_adaptive.argtypes = [vp, sp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.ea_n_floor.argtypes = [i64, f64]
         L.ea_n_floor.restype = i64
+        L.ea_select_compact_inplace.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp]
+        L.ea_select_compact_inplace.restype = ctypes.c_int
         L.ea_sync_status.argtypes = [vp, vp]
         L.ea_host_workspace_bytes.argtypes = [sp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         L.ea_compress_host.argtypes = [vp, sp, vp, vp, vp, vp, i32, f64, f32, i32, i32, vp, vp, vp, vp, vp]
@@ -296,6 +299,19 @@ def ea_select_compact(ctx: Context, shape: Shape, scores, n_kept: int, k=None, v
                                    _ptr(v), _ptr(kept_idx), _ptr(k_out), _ptr(v_out),
                                    _stream(ctx.device)), "ea_select_compact")
     return kept_idx, k_out, v_out
+
+
+def ea_select_compact_inplace(ctx: Context, shape: Shape, scores, n_kept: int, k, v, kept_idx=None):
+    """Selection, then the kept rows of every head move to the front of k and v (modified in place)."""
+    _dev_tensor(scores, torch.float32, "scores")
+    _dev_tensor(k, torch.bfloat16, "k")
+    _dev_tensor(v, torch.bfloat16, "v")
+    if kept_idx is None:
+        kept_idx = torch.empty((shape.n_units, shape.n_kv_heads, max(n_kept, 0)), dtype=torch.int32,
+                               device=scores.device)
+    _check(lib().ea_select_compact_inplace(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k), _ptr(v),
+                                           _ptr(kept_idx), _stream(ctx.device)), "ea_select_compact_inplace")
+    return kept_idx
 
 
 def ea_select_compact_adaptive(ctx: Context, shape: Shape, scores, n_kept: int, n_floor: int, k=None, v=None,

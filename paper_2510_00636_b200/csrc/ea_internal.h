@@ -126,6 +126,10 @@ ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const floa
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
                            int32_t* kept_idx, cudaStream_t st);
 
+// Compaction inside the cache buffers: the kept rows of every head move to the front of its range.
+ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
+                                    __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st);
+
 // Head-adaptive eviction: per-head counts and offsets from one radix search over the unit's scores,
 // then the per-head selection with those counts and a gather through the offsets.
 size_t ea_adaptive_ws_bytes(const ea_shape& s);

@@ -508,6 +508,42 @@ __global__ void gather_adaptive_kernel(const int32_t* __restrict__ kept_idx, con
     }
 }
 
+// In-place compaction of one head of one tensor per CTA: row j of the head receives row idx[j].
+// idx is ascending, so idx[j] >= j: rows only move towards the front.  The CTA walks the kept rows
+// in chunks, front to back; all of a chunk's source rows are in registers before any of its
+// destination rows is written (the barrier), and a later chunk only reads rows at or behind its own
+// first destination row, which earlier chunks never write.
+constexpr int kIpThreads = 256;
+constexpr int kIpLoads = 4;            // 16-byte pieces per thread and chunk
+
+template <int D>
+__global__ void __launch_bounds__(kIpThreads)
+compact_inplace_kernel(const int32_t* __restrict__ kept_idx, int n, int n_kept, uint4* k, uint4* v) {
+    constexpr int LPR = D / 8;                                  // 16-byte pieces per row
+    constexpr int kChunkRows = kIpThreads * kIpLoads / LPR;
+    const long long head = blockIdx.x;
+    uint4* rows = (blockIdx.y == 0 ? k : v) + head * (long long)n * LPR;
+    const int32_t* idx = kept_idx + head * (long long)n_kept;
+    for (int j0 = 0; j0 < n_kept; j0 += kChunkRows) {
+        uint4 x[kIpLoads];
+        int src[kIpLoads];
+#pragma unroll
+        for (int i = 0; i < kIpLoads; ++i) {
+            const int t = i * kIpThreads + threadIdx.x;
+            const int j = j0 + t / LPR;
+            src[i] = j < n_kept ? idx[j] : -1;
+            if (src[i] >= 0 && src[i] != j) x[i] = rows[(long long)src[i] * LPR + t % LPR];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kIpLoads; ++i) {
+            const int t = i * kIpThreads + threadIdx.x;
+            const int j = j0 + t / LPR;
+            if (src[i] >= 0 && src[i] != j) rows[(long long)j * LPR + t % LPR] = x[i];
+        }
+    }
+}
+
 }  // namespace
 
 static ea_status launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
@@ -641,6 +677,22 @@ ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, con
             break;
         default:
             return EA_ERR_UNSUPPORTED;
+    }
+    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+}
+
+ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
+                                    __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st) {
+    if (n_kept <= 0) return EA_OK;
+    ea_count_launches(ctx, 1);
+    const dim3 grid((unsigned)(s.n_units * s.n_kv_heads), 2);
+    uint4* k4 = reinterpret_cast<uint4*>(k);
+    uint4* v4 = reinterpret_cast<uint4*>(v);
+    switch (s.head_dim) {
+        case 64: compact_inplace_kernel<64><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
+        case 128: compact_inplace_kernel<128><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
+        case 256: compact_inplace_kernel<256><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
+        default: return EA_ERR_UNSUPPORTED;
     }
     return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
 }

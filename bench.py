@@ -208,9 +208,10 @@ class DecodeWorkload:
     28 layers x batch 8 folded into the units of one call); the window queries rotate through
     `n_phases` slowly turning query means."""
 
-    def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4):
+    def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False):
         import dataclasses
         self.cfg, self.device, self.ea = cfg, device, ea
+        self.use_graph, self.graphs = use_graph, {}
         self.events = inputs.decode_schedule()
         L, B = cfg.n_layers, cfg.batch
         U, Hq, Hkv, d, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
@@ -249,15 +250,34 @@ class DecodeWorkload:
                                    cfg.window)
         return self.ea.Context.for_shape(shape, self.device.index)
 
-    def step(self, ctx, units_per_call):
+    def _event(self, ctx, n, kept, window, pos):
         ea, cfg = self.ea, self.cfg
+        c = self.caches[n]
+        shape = ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, n, cfg.window)
+        ea.ea_query_stats(ctx, shape, window, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
+        ea.ea_score(ctx, shape, c["k"], c["v"], self.mu, self.sigma, cfg.eps, c["scores"])
+        ea.ea_select_compact(ctx, shape, c["scores"], kept, c["k"], c["v"], c["idx"], c["k_out"], c["v_out"])
+
+    def step(self, ctx, units_per_call):
         for e, (pos, n, kept) in enumerate(self.events):
-            c = self.caches[n]
-            shape = ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, n, cfg.window)
-            ea.ea_query_stats(ctx, shape, self.windows[e % len(self.windows)], self.pos[e], cfg.n_future,
-                              cfg.rope_base, self.mu, self.sigma)
-            ea.ea_score(ctx, shape, c["k"], c["v"], self.mu, self.sigma, cfg.eps, c["scores"])
-            ea.ea_select_compact(ctx, shape, c["scores"], kept, c["k"], c["v"], c["idx"], c["k_out"], c["v_out"])
+            window = self.windows[e % len(self.windows)]
+            if not self.use_graph:
+                self._event(ctx, n, kept, window, self.pos[e])
+                continue
+            # one CUDA graph per distinct event (cache length, window buffer); the position is read from a
+            # device buffer that is refreshed before each replay
+            key = (n, e % len(self.windows))
+            if key not in self.graphs:
+                pos_buf = self.pos[e].clone()
+                self._event(ctx, n, kept, window, pos_buf)          # warm-up outside the capture
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    self._event(ctx, n, kept, window, pos_buf)
+                self.graphs[key] = (g, pos_buf)
+            g, pos_buf = self.graphs[key]
+            pos_buf.copy_(self.pos[e], non_blocking=True)
+            g.replay()
 
     def work(self):
         cfg = self.cfg
@@ -384,6 +404,8 @@ def main():
                          "(ea_query_stats_hidden) in place of given window queries")
     ap.add_argument("--with-wo", type=int, default=None, metavar="D_MODEL",
                     help="prefill configs: weight by ||W_o v|| (ea_score_wo) with an output projection of this width")
+    ap.add_argument("--graph", action="store_true",
+                    help="decode config: replay each compression event as a captured CUDA graph")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -411,7 +433,7 @@ def main():
     variant = args.head_adaptive is not None or args.hidden_stats or args.with_wo
     if variant and decode:
         raise SystemExit("--head-adaptive, --hidden-stats and --with-wo apply to the prefill configs")
-    wl = DecodeWorkload(cfg, device, ea) if decode else Workload(cfg, device, ea, args.head_adaptive,
+    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph) if decode else Workload(cfg, device, ea, args.head_adaptive,
                                                                  args.hidden_stats, args.with_wo)
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
@@ -447,6 +469,15 @@ def main():
     ms_local = ev0.elapsed_time(ev1) / args.steps
     ms = max_over_ranks(ms_local, world, device)
     ctx.sync_status()
+    if decode and args.graph:
+        # replays do not pass through the library's launch counter or its kernel events: take both from one
+        # untimed step of the same launches made directly (every timed step replayed exactly these)
+        wl.use_graph = False
+        ctx.profile_begin()
+        wl.step(ctx, upc)
+        score_ms, score_launches, total_launches = ctx.profile_end()
+        total_launches *= args.steps
+        wl.use_graph = True
 
     # roofline of the dominant kernel (the log-score kernel, Eq. 7)
     n_calls = len(wl.events) if decode else (wl.n_units + upc - 1) // upc
@@ -487,7 +518,7 @@ def main():
                    "statistics": "window queries given" if not args.hidden_stats else
                                  "hidden states through W_Q, d_model %d" % args.hidden_stats,
                    "value_weight": "||v||" if not args.with_wo else "||W_o v||, d_model %d" % args.with_wo,
-                   "key_slots_per_step": slots, "units_per_call": upc, "parallelism": f"replicas x{world}",
+                   "cuda_graph": bool(decode and args.graph), "key_slots_per_step": slots, "units_per_call": upc, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (K+V %.1f GB per step)" % (slots * 4 * cfg.head_dim / 1e9)},
         "ms_per_128k_compression": ms if cfg.cfg_id == 3 else None,
         "path_roofline": {"t_roof_ms": t_path * 1e3, "frac": path_frac, "alg_bytes": alg_bytes,

@@ -34,7 +34,8 @@ from paper_2510_00636_b200 import inputs  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the log-score kernel divided by the
 # key-slots of that launch (ncu --set full, profiles/logits_mma_kernel_*); None = not captured for
 # the current kernel
-NCU_DRAM_BYTES_PER_KEY_SLOT = {256: 1.1018e9 / 2097152, 128: None, 64: None}
+# keyed by (head_dim, query heads per KV head): the log-score write and the sharing of key tiles depend on both
+NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.1018e9 / 2097152, (128, 4): 294.7e6 / 1048576}
 
 METRIC = "kv_keys_scored_and_compacted_per_second"
 UNIT = "Gkeys/s"
@@ -497,7 +498,7 @@ def main():
                     "frac": achieved / peaks["hbm_gbs"]}
     # DRAM bytes per launch from the ncu capture of this kernel (profiles/): measured on a 2-layer
     # case of the same shapes and scaled by the key-slots of a launch (traffic is proportional to them)
-    traffic_per_slot = NCU_DRAM_BYTES_PER_KEY_SLOT.get(cfg.head_dim)
+    traffic_per_slot = NCU_DRAM_BYTES_PER_KEY_SLOT.get((cfg.head_dim, cfg.group))
     traffic = None if traffic_per_slot is None else traffic_per_slot * slots / n_calls
     roofline.update({"traffic": traffic, "kernel": "log-score kernel (k.mu/sqrt(d) + k'Sigma k/2d)",
                      "kernel_ms": avg_score_ms, "launches_timed": score_launches,

@@ -433,22 +433,25 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     float2 acc[G::HPC][2];
 #pragma unroll
                     for (int j = 0; j < G::HPC; ++j) acc[j][0] = acc[j][1] = make_float2(0.f, 0.f);
-                    // block b -> (cb, j): heads innermost so the unpacked key values are reused
-                    auto cb_of = [&](int b) { return half * CBH + b / G::HPC; };
+                    // block b -> (columns c0 .. c0 + BW of head j): heads innermost so the unpacked key values
+                    // are reused.  Narrow blocks at d <= 128, where the epilogue is the limit: half the
+                    // registers per block leave the scheduler room to overlap the dependent FMAs.
+                    constexpr int BW = D == 256 ? 32 : 16;
+                    constexpr int NBW = NB * (32 / BW);
+                    auto c0_of = [&](int b) { return half * CBH * 32 + (b / G::HPC) * BW; };
                     auto addr_of = [&](int b) {
-                        return t_lane + (uint32_t)(a * kAccCols + (b % G::HPC) * D + cb_of(b) * 32);
+                        return t_lane + (uint32_t)(a * kAccCols + (b % G::HPC) * D + c0_of(b));
                     };
-                    uint32_t dv[2][32];
-                    tmem_ld_x32(addr_of(0), dv[0]);      // head 0 always exists
-                    float2 kf[16];
+                    uint32_t dv[2][BW];
+                    tmem_ld_cols(addr_of(0), dv[0]);      // head 0 always exists
+                    float2 kf[BW / 2];
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) {
+                    for (int b = 0; b < NBW; ++b) {
                         const int j = b % G::HPC;
-                        const int cb = cb_of(b);
-                        const int c0 = cb * 32;
+                        const int c0 = c0_of(b);
                         if (j == 0) {
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
+                            for (int q = 0; q < BW / 8; ++q) {
                                 const int unit = (c0 % 64) / 8 + q;
                                 const uint4 w = lds128(k_row + (c0 / 64) * kChunkA + ((unit ^ (row & 7)) << 4));
                                 const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
@@ -460,18 +463,18 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         }
                         // the block's diagonal constants, requested before the accumulator wait so that
                         // their latency is not paid inside the arithmetic
-                        uint4 dgv[8];
+                        uint4 dgv[BW / 4];
                         if (j < it.hpc) {
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) dgv[q] = lds128(s_vec + (uint32_t)((j * D + c0 + 4 * q) * 4));
+                            for (int q = 0; q < BW / 4; ++q) dgv[q] = lds128(s_vec + (uint32_t)((j * D + c0 + 4 * q) * 4));
                         }
                         tmem_ld_wait();
-                        if (b + 1 < NB && (b + 1) % G::HPC < it.hpc) tmem_ld_x32(addr_of(b + 1), dv[(b + 1) & 1]);
+                        if (b + 1 < NBW && (b + 1) % G::HPC < it.hpc) tmem_ld_cols(addr_of(b + 1), dv[(b + 1) & 1]);
                         if (j < it.hpc) {
                             // accumulator = K.B^T + mu' (the linear term rode in on the extra MMA step)
                             const uint32_t* dd = dv[b & 1];
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
+                            for (int q = 0; q < BW / 4; ++q) {
                                 const float4 dg = make_float4(__uint_as_float(dgv[q].x), __uint_as_float(dgv[q].y),
                                                               __uint_as_float(dgv[q].z), __uint_as_float(dgv[q].w));
                                 const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
@@ -484,10 +487,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                             }
                         }
                         // hand the 64-channel chunk back to the producer once this warp is done with it
-                        const bool chunk_done = j == G::HPC - 1 && (D == 64 || (cb & 1) == 1);
+                        const bool chunk_done = j == G::HPC - 1 && (D == 64 ? b == NBW - 1 : (c0 + BW) % 64 == 0);
                         if (chunk_done) {
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(empty_k(stage * G::KCH + cb / 2));
+                            if (lane == 0) mbar_arrive(empty_k(stage * G::KCH + c0 / 64));
                         }
                     }
                     // the accumulator stage is free again

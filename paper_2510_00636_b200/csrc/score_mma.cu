@@ -100,33 +100,53 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
     uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG_FULL;   // 16-byte aligned
     const float quad_scale = form.quad_scale;  // 1/(2d) for Eq. 7, a power of two: the scaling is exact
 
-    // one 16-byte unit (8 consecutive a) of one row c per thread step
-    for (int e = threadIdx.x; e < D * (D / 8); e += blockDim.x) {
-        const int c = e / (D / 8), a0 = (e % (D / 8)) * 8;
-        uint32_t w[4];
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            uint32_t half[2];
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int a = a0 + 2 * p + q;
-                float val = 0.f;
-                if (a != c) {
-                    // Sigma_ac / d (the two mirrored entries together carry 2 Sigma_ac / (2d)),
-                    // split into a bf16 and the bf16 rounding of its remainder
-                    const float x = (S[(size_t)c * D + a] + S[(size_t)a * D + c]) * quad_scale;
-                    const float hi = __bfloat162float(__float2bfloat16_rn(x));
-                    val = a < c ? hi : x - hi;
-                }
-                half[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(val));
-            }
-            w[p] = half[0] | (half[1] << 16);
+    // Image rows in blocks of 32: the block needs S[c][:] (its own rows) and S[:][c] (its columns).  The
+    // columns go through shared memory, loaded as 128-byte row segments, so that every global sector
+    // is fetched once; a strided read of the columns kept this kernel bound by the L1 tag rate.
+    // Thread = (lane: row c of the block, warp: 16-byte unit of 8 consecutive a, stepping by 8 units).
+    __shared__ float col_s[D][33];                     // col_s[a][c - c_blk] = S[a][c]
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    for (int c_blk = 0; c_blk < D; c_blk += 32) {
+        __syncthreads();                               // the previous block's readers are done
+        for (int e = threadIdx.x; e < D * 8; e += 256) {
+            const int a = e / 8, piece = e % 8;
+            const float4 x = __ldg(reinterpret_cast<const float4*>(S + (size_t)a * D + c_blk) + piece);
+            col_s[a][4 * piece + 0] = x.x;
+            col_s[a][4 * piece + 1] = x.y;
+            col_s[a][4 * piece + 2] = x.z;
+            col_s[a][4 * piece + 3] = x.w;
         }
+        __syncthreads();
+        const int c = c_blk + lane;
         const int row = j * D + c;
-        const int kc = a0 / 64, unit = (a0 % 64) / 8;
-        uint4* dst = reinterpret_cast<uint4*>(img + (size_t)kc * G::CHUNK_B_FULL + (size_t)row * 128 +
-                                              ((unit ^ (row & 7)) << 4));
-        *dst = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int a0 = warp * 8; a0 < D; a0 += 64) {
+            const float4 r0 = __ldg(reinterpret_cast<const float4*>(S + (size_t)c * D + a0));
+            const float4 r1 = __ldg(reinterpret_cast<const float4*>(S + (size_t)c * D + a0) + 1);
+            const float own[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+            uint32_t w[4];
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                uint32_t half[2];
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int a = a0 + 2 * p + q;
+                    float val = 0.f;
+                    if (a != c) {
+                        // the two mirrored entries together carry (S_ca + S_ac) * quad_scale, split into a
+                        // bf16 and the bf16 rounding of its remainder
+                        const float x = (own[2 * p + q] + col_s[a][lane]) * quad_scale;
+                        const float hi = __bfloat162float(__float2bfloat16_rn(x));
+                        val = a < c ? hi : x - hi;
+                    }
+                    half[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(val));
+                }
+                w[p] = half[0] | (half[1] << 16);
+            }
+            const int kc = a0 / 64, unit = (a0 % 64) / 8;
+            uint4* dst = reinterpret_cast<uint4*>(img + (size_t)kc * G::CHUNK_B_FULL + (size_t)row * 128 +
+                                                  ((unit ^ (row & 7)) << 4));
+            *dst = make_uint4(w[0], w[1], w[2], w[3]);
+        }
     }
     // linear-term operand: row (j, c) holds mu_bar_c / sqrt(d) as a bf16 and the bf16 of its remainder in
     // K columns 0 and 1, zeros elsewhere; unswizzled core-matrix layout (8 rows x 16 bytes, K columns

@@ -75,6 +75,13 @@ def test_score_with_output_projection(ea, oracle, cfg_id, n_keys, dm, sets, mode
     _run(ea, oracle, inputs.CONFIGS[cfg_id].tempered(2.0, 0.02), n_keys, dm, sets, mode)
 
 
+def test_score_with_output_projection_head_dim_256(ea, oracle):
+    """The paired-CTA tensor-core path (head_dim 256) with the value rows as its operand, ragged cache."""
+    import dataclasses
+    cfg = dataclasses.replace(inputs.CONFIGS[3].tempered(2.0, 0.02), n_layers=1, n_keys=3000, n_kept=375)
+    _run(ea, oracle, cfg, 3000, 192, 1)
+
+
 def test_whole_path_with_output_projection_against_oracle(ea, oracle):
     cfg = inputs.CONFIGS[0].tempered(2.0, 0.02)
     scores, _, _, (q, k, v, pos, w_o) = _run(ea, oracle, cfg, cfg.n_keys, 96, 1)

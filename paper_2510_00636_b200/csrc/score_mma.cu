@@ -9,7 +9,12 @@
 // B carries the off-diagonal of Sigma_bar/(2d) at twice bf16 precision for the price of one bf16
 // matrix: the quadratic form only sees B[c,a] + B[a,c], so for a < c the entry B[c,a] holds
 // bf16(Sigma_ac/d) and the mirrored entry B[a,c] holds the bf16 rounding of what that left over.
-// The diagonal stays out of B and enters in fp32 in the epilogue: two FMAs per accumulator element.
+// At head_dim 256, where the tensor pipe is the limit, the diagonal stays out of B and enters in fp32
+// in the epilogue (two FMAs per accumulator element).  At head_dim <= 128, where the epilogue is the
+// limit, the diagonal goes through the tensor cores too, as a bf16 pair: its bf16 part on B's diagonal,
+// the bf16 rounding of the rest by one small MMA (N = 16 heads-per-pass columns, K = 16) per 16
+// channels against a diagonal block; the heads' accumulator columns are interleaved in runs of 16 so
+// that one such step serves every head.  The epilogue is then s = sum_c k_c D[i, c]: one FMA per element.
 //
 // A CTA keeps the image of `hpc` query heads of one KV head resident in shared memory
 // (hpc * d = 256 accumulator columns at most) and streams key tiles through a TMA ring:
@@ -55,12 +60,26 @@ struct Geo {
     static constexpr int ONES = kTileKeys * 32;
     static constexpr int LIN_FULL = IMG_ROWS * 32;       // bytes of the mu' operand of a whole image (global)
     static constexpr int LIN_CTA = ROWS_CTA * 32;
-    static constexpr int IMG_FULL = IMG_MAIN + LIN_FULL; // bytes of a whole image (global)
+    // At d <= 128 the epilogue is the limit, so the diagonal goes to the tensor cores as well: its bf16
+    // part sits on the image's diagonal, and the bf16 rounding of what that leaves is added by one
+    // M128 N16 K16 step per (head, 16 channels) against a 16 x 16 diagonal block (unswizzled core
+    // matrices, 512 bytes).  At d = 256 the tensor pipe is the limit and the diagonal stays in fp32 in
+    // the epilogue.
+    static constexpr bool DIAG_MMA = D <= 128;
+    static constexpr int DIAG_BLOCK = 16 * HPC * 32;                    // bytes: 16 HPC rows x 16 bf16
+    static constexpr int DIAG_FULL = DIAG_MMA ? (D / 16) * DIAG_BLOCK : 0;   // per whole image
+    // Accumulator column (= image row) of channel c of head j.  With the diagonal blocks the heads are
+    // interleaved in runs of 16 channels, so that the 16 channels of one MMA step are 16 HPC adjacent
+    // columns and every head's share of the diagonal is added by one instruction per step.
+    __host__ __device__ static constexpr int col(int j, int c) {
+        return DIAG_MMA ? (c / 16) * (16 * HPC) + j * 16 + c % 16 : j * D + c;
+    }
+    static constexpr int IMG_FULL = IMG_MAIN + LIN_FULL + DIAG_FULL;   // bytes of a whole image (global)
     static constexpr int PART = 2 * HPC * kTileKeys * (int)sizeof(float);   // partial sums of the two column halves
     static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
     static constexpr int NBAR = 2 * NSLOT + 6;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + ONES + LIN_CTA + VEC + PART + RED + CTRL + 1024;
+    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
     // warps that must release a chunk slot before it is refilled
     static constexpr int SLOT_RELEASERS = D == 64 ? kEpiWarps : kEpiWarps / 2;
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
@@ -118,7 +137,7 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
         }
         __syncthreads();
         const int c = c_blk + lane;
-        const int row = j * D + c;
+        const int row = G::col(j, c);
         for (int a0 = warp * 8; a0 < D; a0 += 64) {
             const float4 r0 = __ldg(reinterpret_cast<const float4*>(S + (size_t)c * D + a0));
             const float4 r1 = __ldg(reinterpret_cast<const float4*>(S + (size_t)c * D + a0) + 1);
@@ -137,6 +156,8 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
                         const float x = (own[2 * p + q] + col_s[a][lane]) * quad_scale;
                         const float hi = __bfloat162float(__float2bfloat16_rn(x));
                         val = a < c ? hi : x - hi;
+                    } else if (G::DIAG_MMA) {
+                        val = own[2 * p + q] * quad_scale;           // its bf16 part; the rest in the diagonal blocks
                     }
                     half[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(val));
                 }
@@ -155,12 +176,26 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
         const float m = form.lin ? form.lin[set_head * D + c] * form.lin_scale : 0.f;
         const __nv_bfloat16 hi = __float2bfloat16_rn(m);
         const __nv_bfloat16 lo = __float2bfloat16_rn(m - __bfloat162float(hi));
-        const int row = j * D + c;
+        const int row = G::col(j, c);
         uint8_t* dst = img + G::IMG_MAIN + (size_t)(row / 8) * 256 + (row % 8) * 16;
         *reinterpret_cast<uint4*>(dst) =
             make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
         *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
-        vec[(size_t)uh * D + c] = S[(size_t)c * D + c] * quad_scale;
+        const float dg = S[(size_t)c * D + c] * quad_scale;
+        vec[(size_t)uh * D + c] = dg;
+        if (G::DIAG_MMA) {
+            // block c / 16 (one per MMA step), row n = 16 j + c % 16, K column c % 16: the bf16 of what the
+            // image's diagonal entry left of dg; zeros elsewhere in the row
+            const __nv_bfloat16 lo = __float2bfloat16_rn(dg - __bfloat162float(__float2bfloat16_rn(dg)));
+            const int kk = c % 16, n = 16 * j + kk;
+            uint8_t* blk = img + G::IMG_MAIN + G::LIN_FULL + (size_t)(c / 16) * G::DIAG_BLOCK +
+                           (n / 8) * 256 + (n % 8) * 16;
+            uint32_t w4[4] = {0u, 0u, 0u, 0u};
+            w4[(kk % 8) / 2] = (uint32_t)__bfloat16_as_ushort(lo) << (16 * (kk % 2));
+            const uint4 mine = make_uint4(w4[0], w4[1], w4[2], w4[3]), zero = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(blk) = kk < 8 ? mine : zero;            // K columns 0..7
+            *reinterpret_cast<uint4*>(blk + 128) = kk < 8 ? zero : mine;      // K columns 8..15
+        }
     }
 }
 
@@ -202,6 +237,7 @@ template <int D, bool PAIR>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) {
     using G = Geo<D, PAIR>;
+    static_assert(!(G::DIAG_MMA && PAIR), "the diagonal blocks are laid out for a single CTA");
     extern __shared__ uint8_t smem_raw[];
     // carve shared memory: 1024-byte aligned operand tiles first
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -213,11 +249,12 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     const uint32_t s_lin = s_ones + G::ONES;
     constexpr int kOffVec = kOffOnes + G::ONES + G::LIN_CTA;
     const uint32_t s_vec = base + kOffVec;
-    const float* vec_gen = reinterpret_cast<const float*>(gen_base + kOffVec);
-    float* part_gen = reinterpret_cast<float*>(gen_base + kOffVec + G::VEC);
-    float* red_gen = reinterpret_cast<float*>(gen_base + kOffVec + G::VEC + G::PART);
-    const uint32_t s_bar = base + kOffVec + G::VEC + G::PART + G::RED;
-    uint8_t* bar_gen = gen_base + kOffVec + G::VEC + G::PART + G::RED;
+    const uint32_t s_diag = s_vec + G::VEC;                      // 16 x 16 diagonal blocks (d <= 128)
+    constexpr int kOffPart = kOffVec + G::VEC + G::DIAG_FULL;
+    float* part_gen = reinterpret_cast<float*>(gen_base + kOffPart);
+    float* red_gen = reinterpret_cast<float*>(gen_base + kOffPart + G::PART);
+    const uint32_t s_bar = base + kOffPart + G::PART + G::RED;
+    uint8_t* bar_gen = gen_base + kOffPart + G::PART + G::RED;
     auto full_k = [&](int slot) { return s_bar + 8u * slot; };
     auto empty_k = [&](int slot) { return s_bar + 8u * (G::NSLOT + slot); };
     auto tmem_full = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + a); };
@@ -294,18 +331,21 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                             ok = mbar_wait(empty_k(stage * G::KCH + kc), fill & 1, abort_flag);
                     }
                     if (!ok) break;
-                    const int rows_total = it.hpc * D;
+                    const int rows_total = (G::DIAG_MMA ? G::HPC : it.hpc) * D;     // interleaved heads: every row
                     const int rows = PAIR ? rows_total / 2 : rows_total;
                     const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
                     const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
-                    const uint32_t vec_bytes = (uint32_t)(it.hpc * D * sizeof(float));
+                    // the fp32 diagonal for the epilogue (d = 256) or the diagonal blocks for the tensor cores
+                    const uint32_t vec_bytes = G::DIAG_MMA ? (uint32_t)G::DIAG_FULL
+                                                           : (uint32_t)(it.hpc * D * sizeof(float));
                     mbar_arrive_expect_tx(img_full, (uint32_t)(G::KCH * rows * 128 + rows * 32) + vec_bytes);
                     const uint8_t* img = p.image + (size_t)img_id * G::IMG_FULL;
                     const uint8_t* src = img + (size_t)rank * rows * 128;
                     for (int kc = 0; kc < G::KCH; ++kc)
                         bulk_load(s_img + kc * G::CHUNK_B, src + (size_t)kc * G::CHUNK_B_FULL, rows * 128, img_full);
                     bulk_load(s_lin, img + G::IMG_MAIN + (size_t)rank * rows * 32, rows * 32, img_full);
-                    bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
+                    if (G::DIAG_MMA) bulk_load(s_diag, img + G::IMG_MAIN + G::LIN_FULL, vec_bytes, img_full);
+                    else bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
                     cur_img = img_id;
                 }
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
@@ -354,7 +394,9 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     ++img_loads;
                     cur_img = img_id;
                 }
-                const uint32_t n_cols = (uint32_t)(it.hpc * D);
+                // (interleaved heads: a pass with fewer heads still spans every column; the columns of the
+                // missing heads hold whatever the image rows held and are never read)
+                const uint32_t n_cols = (uint32_t)((G::DIAG_MMA ? G::HPC : it.hpc) * D);
                 const uint32_t idesc = PAIR ? umma_idesc_bf16_m256(n_cols) : umma_idesc_bf16_m128(n_cols);
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
                     const int stage = (int)(tile_no % G::STAGES);
@@ -385,6 +427,17 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         const uint64_t db = umma_desc_k_plain(s_lin);
                         if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, 1u);
                         else umma_bf16(d_tmem, da, db, idesc, 1u);
+                    }
+                    if (G::DIAG_MMA) {
+                        // D[:, c] += k_c * lo(diag_c) for every head: one N = 16 HPC step per 16 channels
+                        const uint32_t idesc_d = umma_idesc_bf16_m128(16 * G::HPC);
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const int slot = stage * G::KCH + ks / 4;
+                            umma_bf16(d_tmem + (uint32_t)(ks * 16 * G::HPC),
+                                      umma_desc_k_sw128(s_k + slot * kChunkA + (ks % 4) * 32),
+                                      umma_desc_k_plain(s_diag + (uint32_t)(ks * G::DIAG_BLOCK)), idesc_d, 1u);
+                        }
                     }
                     if (PAIR) umma_commit_pair(tmem_full(a), 3);
                     else umma_commit(tmem_full(a));
@@ -460,7 +513,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     constexpr int NBW = NB * (32 / BW);
                     auto c0_of = [&](int b) { return half * CBH * 32 + (b / G::HPC) * BW; };
                     auto addr_of = [&](int b) {
-                        return t_lane + (uint32_t)(a * kAccCols + (b % G::HPC) * D + c0_of(b));
+                        return t_lane + (uint32_t)(a * kAccCols + G::col(b % G::HPC, c0_of(b)));
                     };
                     uint32_t dv[2][BW];
                     tmem_ld_cols(addr_of(0), dv[0]);      // head 0 always exists
@@ -484,7 +537,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         // the block's diagonal constants, requested before the accumulator wait so that
                         // their latency is not paid inside the arithmetic
                         uint4 dgv[BW / 4];
-                        if (j < it.hpc) {
+                        if (!G::DIAG_MMA && j < it.hpc) {
 #pragma unroll
                             for (int q = 0; q < BW / 4; ++q) dgv[q] = lds128(s_vec + (uint32_t)((j * D + c0 + 4 * q) * 4));
                         }
@@ -495,9 +548,17 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                             const uint32_t* dd = dv[b & 1];
 #pragma unroll
                             for (int q = 0; q < BW / 4; ++q) {
+                                const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
+                                if (G::DIAG_MMA) {
+                                    // the whole bracket came from the tensor cores: one FMA per element
+                                    acc[j][0] = fma2(k0, make_float2(__uint_as_float(dd[4 * q]), __uint_as_float(dd[4 * q + 1])),
+                                                     acc[j][0]);
+                                    acc[j][1] = fma2(k1, make_float2(__uint_as_float(dd[4 * q + 2]), __uint_as_float(dd[4 * q + 3])),
+                                                     acc[j][1]);
+                                    continue;
+                                }
                                 const float4 dg = make_float4(__uint_as_float(dgv[q].x), __uint_as_float(dgv[q].y),
                                                               __uint_as_float(dgv[q].z), __uint_as_float(dgv[q].w));
-                                const float2 k0 = kf[2 * q], k1 = kf[2 * q + 1];
                                 const float2 t0 = fma2(make_float2(dg.x, dg.y), k0,
                                                        make_float2(__uint_as_float(dd[4 * q]), __uint_as_float(dd[4 * q + 1])));
                                 const float2 t1 = fma2(make_float2(dg.z, dg.w), k1,
@@ -705,7 +766,9 @@ size_t ea_mma_image_bytes(const ea_shape& s) {
     const int Gq = s.n_q_heads / s.n_kv_heads;
     const int hpc = 256 / s.head_dim;
     const size_t subsets = (size_t)((Gq + hpc - 1) / hpc);
-    return (size_t)s.n_units * s.n_kv_heads * subsets * ((size_t)hpc * s.head_dim * s.head_dim * 2 + (size_t)hpc * s.head_dim * 32);
+    const size_t diag_blocks = s.head_dim <= 128 ? (size_t)hpc * (s.head_dim / 16) * 512 : 0;
+    return (size_t)s.n_units * s.n_kv_heads * subsets *
+           ((size_t)hpc * s.head_dim * s.head_dim * 2 + (size_t)hpc * s.head_dim * 32 + diag_blocks);
 }
 
 size_t ea_mma_vec_bytes(const ea_shape& s) {

@@ -35,7 +35,7 @@ from paper_2510_00636_b200 import inputs  # noqa: E402
 # key-slots of that launch (ncu --set full, profiles/logits_mma_kernel_*); None = not captured for
 # the current kernel
 # keyed by (head_dim, query heads per KV head): the log-score write and the sharing of key tiles depend on both
-NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.1018e9 / 2097152, (128, 4): 293.7e6 / 1048576}
+NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.1018e9 / 2097152, (128, 4): 293.9e6 / 1048576}
 
 METRIC = "kv_keys_scored_and_compacted_per_second"
 UNIT = "Gkeys/s"

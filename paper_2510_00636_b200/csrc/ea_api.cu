@@ -29,7 +29,7 @@ ea_status check_shape(const ea_shape* s) {
 ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     ea_ws_plan p;
     size_t off = 0;
-    const size_t U = (size_t)s.n_units, Hq = (size_t)s.n_q_heads, Hkv = (size_t)s.n_kv_heads;
+    const size_t U = (size_t)s.n_units, Hq = (size_t)s.n_q_heads;
     const size_t n = (size_t)s.n_keys, d = (size_t)s.head_dim;
     p.rope_coef = off;  off = ea_align_up(off + U * (d / 2) * 2 * sizeof(float), 256);
     p.logits = off;     off = ea_align_up(off + U * Hq * n * sizeof(float), 256);

@@ -152,6 +152,17 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
     const uint4* q4 = reinterpret_cast<const uint4*>(q);
     uint4* raw4 = reinterpret_cast<uint4*>(raw);
 
+    // this thread's channel of the staged rows (the block's rows, then its columns), its rotation partner
+    // and the two coefficients of x = (R_bar (u - mu))[ch] = t_c (u_ch - mu_ch) + t_s (u_partner - mu_partner)
+    const int t_r = tid % n_rows, t_w = tid / n_rows, t_wstep = 256 / n_rows;
+    const int t_ch = (t_r < BM ? bi * BM : bj * BM - BM) + t_r;
+    int t_m, t_partner;
+    bool t_first;                                                   // t_ch is the first channel of its rotation pair
+    if (layout == EA_ROPE_INTERLEAVED) { t_m = t_ch >> 1; t_first = (t_ch & 1) == 0; t_partner = t_ch ^ 1; }
+    else { t_m = t_ch < HALF ? t_ch : t_ch - HALF; t_first = t_ch < HALF; t_partner = t_first ? t_ch + HALF : t_ch - HALF; }
+    const float t_mu = mu_s[t_ch], t_mu_partner = mu_s[t_partner];
+    const float t_c = c_s[t_m], t_s = t_first ? -s_s[t_m] : s_s[t_m];
+
     for (int w0 = 0; w0 < W; w0 += kKC) {
         __syncthreads();
         // the raw chunk with 128-bit loads (rows past the window read as zero) ...
@@ -162,22 +173,17 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
         }
         __syncthreads();
         // ... then x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
-        for (int e = tid; e < n_rows * kKC; e += 256) {
-            const int w = e / n_rows, r = e % n_rows;              // consecutive threads: consecutive channels
-            const int ch = (r < BM ? bi * BM : bj * BM - BM) + r;
+        // (a thread keeps one channel for the whole kernel: n_rows divides the block size)
+        for (int w = t_w; w < kKC; w += t_wstep) {
             float x = 0.f;
             if (w0 + w < W) {
-                int m, partner;
-                bool first;                                         // ch is the first channel of its rotation pair
-                if (layout == EA_ROPE_INTERLEAVED) { m = ch >> 1; first = (ch & 1) == 0; partner = ch ^ 1; }
-                else { m = ch < HALF ? ch : ch - HALF; first = ch < HALF; partner = first ? ch + HALF : ch - HALF; }
-                const float xa = to_f32(raw[w * D + ch]) - mu_s[ch];
-                const float xb = to_f32(raw[w * D + partner]) - mu_s[partner];
-                x = first ? c_s[m] * xa - s_s[m] * xb : s_s[m] * xb + c_s[m] * xa;
+                const float xa = to_f32(raw[w * D + t_ch]) - t_mu;
+                const float xb = to_f32(raw[w * D + t_partner]) - t_mu_partner;
+                x = t_c * xa + t_s * xb;
             }
             const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-            xt[0][r][w] = hi;
-            xt[1][r][w] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            xt[0][t_r][w] = hi;
+            xt[1][t_r][w] = __float2bfloat16_rn(x - __bfloat162float(hi));
         }
         __syncthreads();
 #pragma unroll

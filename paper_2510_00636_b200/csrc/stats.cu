@@ -174,16 +174,23 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
         __syncthreads();
         // ... then x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
         // (a thread keeps one channel for the whole kernel: n_rows divides the block size)
-        for (int w = t_w; w < kKC; w += t_wstep) {
-            float x = 0.f;
-            if (w0 + w < W) {
-                const float xa = to_f32(raw[w * D + t_ch]) - t_mu;
-                const float xb = to_f32(raw[w * D + t_partner]) - t_mu_partner;
-                x = t_c * xa + t_s * xb;
+        // two neighbouring window rows per step: one 32-bit store per (hi, lo)
+        for (int w = 2 * t_w; w < kKC; w += 2 * t_wstep) {
+            __nv_bfloat162 hi2, lo2;
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                float x = 0.f;
+                if (w0 + w + k < W) {
+                    const float xa = to_f32(raw[(w + k) * D + t_ch]) - t_mu;
+                    const float xb = to_f32(raw[(w + k) * D + t_partner]) - t_mu_partner;
+                    x = t_c * xa + t_s * xb;
+                }
+                const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+                if (k == 0) { hi2.x = hi; lo2.x = lo; } else { hi2.y = hi; lo2.y = lo; }
             }
-            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-            xt[0][t_r][w] = hi;
-            xt[1][t_r][w] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            *reinterpret_cast<__nv_bfloat162*>(&xt[0][t_r][w]) = hi2;
+            *reinterpret_cast<__nv_bfloat162*>(&xt[1][t_r][w]) = lo2;
         }
         __syncthreads();
 #pragma unroll

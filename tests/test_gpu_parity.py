@@ -195,6 +195,31 @@ def test_score_ragged_sizes(ea, oracle, n):
     np.testing.assert_allclose(sc.cpu().numpy(), sc_r, rtol=1e-2)
 
 
+@pytest.mark.parametrize("n", [129, 300, 1000])
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 6, 2), (64, 10, 2)])
+def test_score_ragged_sizes_odd_groups(ea, oracle, n, d, Hq, Hkv):
+    """Ragged caches with a group size that leaves the last pass of the tensor-core kernel partly
+    empty (three query heads per KV head at two heads per pass; five at four per pass)."""
+    import dataclasses
+    cfg = dataclasses.replace(inputs.CONFIGS[0].tempered(2.0), n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d,
+                              window=48, n_keys=n, n_kept=n // 2)
+    q, k, v, pos = inputs.generate_layer(cfg, device="cuda", n_keys=n)
+    shape = _shape(ea, cfg, n_keys=n)
+    ctx = ea.Context.for_shape(shape)
+    mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
+    sc, lg = ea.ea_score(ctx, shape, k, v, mu, sig, cfg.eps, want_logits=True)
+    ctx.sync_status()
+    mu_r, sig_r = oracle.query_stats(inputs.bits(q), pos.numpy(), cfg.n_future, cfg.rope_base)
+    s_r = oracle.logits(inputs.bits(k), mu_r, sig_r)
+    sc_r = oracle.scores(s_r, inputs.bits(v), cfg.eps)
+    delta = parity.logit_error_bound(inputs.bits(k), mu_r, sig_r, 16)
+    bad, _ = parity.check_logits(lg.cpu().numpy(), s_r, delta)
+    assert bad == 0
+    lo, hi = parity.score_range(s_r, delta, inputs.bits(v), cfg.eps, 0)
+    bad, unstable = parity.check_scores(sc.cpu().numpy(), lo, hi)
+    assert bad == 0 and unstable <= max(8, lo.size // 1000)
+
+
 def test_decode_events_below_the_budget_keep_every_key(ea, oracle):
     """Streaming decode: while the cache is within its budget (the first events of the schedule) scores
     are still computed but compaction is the identity; the first event above the budget evicts."""

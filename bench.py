@@ -16,6 +16,7 @@ are independent, no data-path collective exists.
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import subprocess
@@ -272,6 +273,7 @@ class DecodeWorkload:
                 pos_buf = self.pos[e].clone()
                 self._event(ctx, n, kept, window, pos_buf)          # warm-up outside the capture
                 torch.cuda.synchronize()
+                gc.collect()          # no library context may be destroyed (cudaFree) while the capture is open
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     self._event(ctx, n, kept, window, pos_buf)

@@ -32,6 +32,8 @@
  *     launched.  No call aborts, throws or traps the device.  A device-side
  *     wait that runs out of its iteration budget records
  *     EA_ERR_DEVICE_TIMEOUT, which ea_sync_status reports.
+ *   - n_units * n_q_heads <= 65535 per call (EA_ERR_UNSUPPORTED beyond: split
+ *     the units over several calls).
  *   - There is no CPU fallback: on a machine without an sm_100 GPU ea_create
  *     fails with EA_ERR_NOT_SM100 or EA_ERR_CUDA.
  */
@@ -81,9 +83,16 @@ typedef struct ea_shape {
 
 typedef struct ea_ctx ea_ctx;   /* opaque; owns its workspace and a status word */
 
-/* Library version string, e.g. "ea-b200 0.1". */
+/* Library version string, e.g. "ea-b200 0.2". */
 const char* ea_version(void);
 const char* ea_status_string(ea_status s);
+/*
+ * Which CUDA runtime call was behind the calling thread's most recent
+ * EA_ERR_CUDA: "<error name> (<description>) at <source file>:<line>", or ""
+ * if there has been none.  The string belongs to the library and is
+ * overwritten by the thread's next failing call.
+ */
+const char* ea_last_cuda_error(void);
 
 /*
  * Bytes of workspace the three calls need for this shape (the maximum over the
@@ -327,6 +336,22 @@ int64_t ea_n_floor(int64_t n_kept, double safeguard);
  * EA_ERR_CUDA if the stream reports an error), then clears it.
  */
 ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream);
+
+/*
+ * Self-test of the device-timeout route (the paper has no counterpart).  Every
+ * wait inside the library's kernels is bounded; one that gives up raises the
+ * context's status word, which ea_sync_status reports as
+ * EA_ERR_DEVICE_TIMEOUT.  This call launches a one-thread kernel that waits,
+ * with the same bounded wait and a limit of limit_us microseconds
+ * (1 <= limit_us <= 1000, EA_ERR_INVALID_ARG otherwise), on a barrier that
+ * nothing signals, so the wait runs out by construction; no copy is in flight
+ * and nothing is held, the kernel returns by itself and the context stays
+ * usable.  After it, ea_sync_status returns EA_ERR_DEVICE_TIMEOUT once and
+ * EA_OK from then on.  The production waits keep their own limit (2 s: far
+ * longer than any healthy wait, also under a profiler's replay or on a GPU
+ * shared with other processes; a genuine stall surfaces the same way).
+ */
+ea_status ea_selftest_wait_timeout(ea_ctx* ctx, int32_t limit_us, void* cuda_stream);
 
 /*
  * The whole routine on HOST buffers: compress(queries, keys, values) ->

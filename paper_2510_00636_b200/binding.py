@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -34,7 +34,8 @@ class EAError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         name = lib().ea_status_string(status).decode()
-        super().__init__(f"{where} failed: {name} ({status})")
+        detail = lib().ea_last_cuda_error().decode() if status == 4 else ""
+        super().__init__(f"{where} failed: {name} ({status})" + (f": {detail}" if detail else ""))
 
 
 class Shape(ctypes.Structure):
@@ -58,6 +59,7 @@ def lib() -> ctypes.CDLL:
                                   ctypes.c_double)
         sp = ctypes.POINTER(Shape)
         L.ea_version.restype = ctypes.c_char_p
+        L.ea_last_cuda_error.restype = ctypes.c_char_p
         L.ea_status_string.restype = ctypes.c_char_p
         L.ea_status_string.argtypes = [ctypes.c_int]
         L.ea_workspace_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
@@ -81,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.ea_n_floor.restype = i64
         L.ea_select_compact_inplace.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp]
         L.ea_select_compact_inplace.restype = ctypes.c_int
+        L.ea_selftest_wait_timeout.argtypes = [vp, i32, vp]
+        L.ea_selftest_wait_timeout.restype = ctypes.c_int
         L.ea_sync_status.argtypes = [vp, vp]
         L.ea_host_workspace_bytes.argtypes = [sp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         L.ea_compress_host.argtypes = [vp, sp, vp, vp, vp, vp, i32, f64, f32, i32, i32, vp, vp, vp, vp, vp]
@@ -134,7 +138,12 @@ def _dev_tensor(t, dtype, name):
 
 
 class Context:
-    """Owns an ``ea_ctx`` (its workspace lives on ``device``)."""
+    """Owns an ``ea_ctx`` (its workspace lives on ``device``).
+
+    Destroying a context frees device memory.  CUDA forbids that while a stream of the process is
+    being captured into a graph (the capture is invalidated), so keep contexts alive across a
+    capture and run ``gc.collect()`` before opening one if unreferenced contexts may be waiting
+    for the garbage collector."""
 
     def __init__(self, device: int | torch.device = 0, workspace_bytes: int = 0):
         self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
@@ -161,6 +170,11 @@ class Context:
 
     def sync_status(self):
         _check(lib().ea_sync_status(self._h, _stream(self.device)), "ea_sync_status")
+
+    def selftest_wait_timeout(self, limit_us: int = 200):
+        """Launch the self-test kernel whose bounded wait runs out (see ``ea_selftest_wait_timeout``)."""
+        _check(lib().ea_selftest_wait_timeout(self._h, int(limit_us), _stream(self.device)),
+               "ea_selftest_wait_timeout")
 
     def profile_begin(self):
         _check(lib().ea_profile_begin(self._h), "ea_profile_begin")

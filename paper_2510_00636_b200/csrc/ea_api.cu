@@ -1,5 +1,7 @@
 // Host side of the C ABI: argument validation, workspace planning, context
 // lifetime, and the order of kernel launches of each call.
+#include <stdio.h>
+
 #include <new>
 
 #include "ea_internal.h"
@@ -19,12 +21,22 @@ ea_status check_shape(const ea_shape* s) {
         return EA_ERR_INVALID_ARG;
     if (s->cov_norm != EA_COV_POPULATION && s->cov_norm != EA_COV_SAMPLE) return EA_ERR_INVALID_ARG;
     if (s->head_dim != 64 && s->head_dim != 128 && s->head_dim != 256) return EA_ERR_UNSUPPORTED;
-    // grid dimension limits of the per-head launches
-    if ((long long)s->n_units * s->n_q_heads > 65535LL * 1024) return EA_ERR_UNSUPPORTED;
+    // several kernels put one (unit, head) per gridDim.y entry
+    if ((long long)s->n_units * s->n_q_heads > 65535LL) return EA_ERR_UNSUPPORTED;
     return EA_OK;
 }
 
+thread_local char g_last_cuda_error[192] = "";
+
 }  // namespace
+
+void ea_note_cuda_error(cudaError_t err, const char* file, int line) {
+    const char* base = file;
+    for (const char* c = file; *c; ++c)
+        if (*c == '/') base = c + 1;
+    snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s (%s) at %s:%d", cudaGetErrorName(err),
+             cudaGetErrorString(err), base, line);
+}
 
 ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     ea_ws_plan p;
@@ -45,7 +57,9 @@ ea_ws_plan ea_plan_workspace(const ea_shape& s) {
 
 extern "C" {
 
-const char* ea_version(void) { return "ea-b200 0.1"; }
+const char* ea_version(void) { return "ea-b200 0.2"; }
+
+const char* ea_last_cuda_error(void) { return g_last_cuda_error; }
 
 const char* ea_status_string(ea_status s) {
     switch (s) {
@@ -438,7 +452,7 @@ int64_t ea_n_floor(int64_t n_kept, double safeguard) {
 
 ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream) {
     if (!ctx) return EA_ERR_INVALID_ARG;
-    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return EA_ERR_CUDA;
+    EA_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
     const int s = *ctx->status_host;
     *ctx->status_host = 0;
     return s == 0 ? EA_OK : static_cast<ea_status>(s);
@@ -456,11 +470,11 @@ ea_status ea_profile_end(ea_ctx* ctx, void* cuda_stream, double* score_kernel_ms
                          int64_t* timed_launches, int64_t* total_kernel_launches) {
     if (!ctx) return EA_ERR_INVALID_ARG;
     ctx->profiling = false;
-    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return EA_ERR_CUDA;
+    EA_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
     double total = 0.0;
     for (int i = 0; i < ctx->n_events; ++i) {
         float ms = 0.f;
-        if (cudaEventElapsedTime(&ms, ctx->ev_start[i], ctx->ev_stop[i]) != cudaSuccess) return EA_ERR_CUDA;
+        EA_CUDA_TRY(cudaEventElapsedTime(&ms, ctx->ev_start[i], ctx->ev_stop[i]));
         total += (double)ms;
     }
     if (score_kernel_ms) *score_kernel_ms = total;

@@ -55,10 +55,25 @@ struct ea_ws_plan {
 
 ea_ws_plan ea_plan_workspace(const ea_shape& s);
 
+// The CUDA error behind the calling thread's most recent EA_ERR_CUDA (ea_last_cuda_error).
+void ea_note_cuda_error(cudaError_t err, const char* file, int line);
+// EA_OK if no runtime call of this thread has failed since the last check, else EA_ERR_CUDA (noted).
+static inline ea_status ea_check_launch(const char* file, int line) {
+    const cudaError_t err = cudaGetLastError();
+    if (err == cudaSuccess) return EA_OK;
+    ea_note_cuda_error(err, file, line);
+    return EA_ERR_CUDA;
+}
+#define EA_CHECK_LAUNCH() ea_check_launch(__FILE__, __LINE__)
+
 #define EA_CUDA_TRY(expr)                                   \
     do {                                                    \
         cudaError_t err__ = (expr);                         \
-        if (err__ != cudaSuccess) return EA_ERR_CUDA;       \
+        if (err__ != cudaSuccess) {                         \
+            ea_note_cuda_error(err__, __FILE__, __LINE__);  \
+            cudaGetLastError();                             \
+            return EA_ERR_CUDA;                             \
+        }                                                   \
     } while (0)
 
 static inline size_t ea_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

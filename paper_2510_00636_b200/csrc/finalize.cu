@@ -214,7 +214,7 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
             return EA_ERR_UNSUPPORTED;
     }
     ea_count_launches(ctx, lse_ready ? 1 : 2);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 
@@ -223,13 +223,13 @@ ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const floa
     const int rows = s.n_units * s.n_q_heads;
     lse_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(lse_part, rows, n_chunks, lse);
     ea_count_launches(ctx, 1);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_lse(const ea_ctx* ctx, const ea_shape& s, const float* logits, float* lse, cudaStream_t st) {
     lse_kernel<<<s.n_units * s.n_q_heads, kLseThreads, 0, st>>>(logits, s.n_keys, 1, lse);
     ea_count_launches(ctx, 1);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
@@ -238,7 +238,7 @@ ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const floa
     finalize_wo_kernel<<<grid, 256, 0, st>>>(logits, lse, wo_norm2, s.n_q_heads, s.n_kv_heads, s.n_keys,
                                              s.group_mode, epsilon, scores);
     ea_count_launches(ctx, 1);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_wo_gram(const ea_ctx* ctx, const __nv_bfloat16* w_o, int d_model, int n_sets, int Hq, int d,
@@ -248,5 +248,5 @@ ea_status ea_launch_wo_gram(const ea_ctx* ctx, const __nv_bfloat16* w_o, int d_m
     if (grid.y > 65535u || grid.z > 65535u) return EA_ERR_UNSUPPORTED;
     wo_gram_kernel<<<grid, 256, 0, st>>>(w_o, d_model, Hq, d, gram);
     ea_count_launches(ctx, 1);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }

@@ -95,7 +95,7 @@ project_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_constant_
                 // let the copies already in flight land before the CTA's shared memory goes away
                 for (int back = 1; back <= p.stages && back <= kc; ++back) {
                     const int c = kc - back;
-                    mbar_wait(full(c % p.stages), (uint32_t)(c / p.stages) & 1, abort_flag);
+                    mbar_drain(full(c % p.stages), (uint32_t)(c / p.stages) & 1);
                 }
             }
         }
@@ -188,11 +188,10 @@ ea_status ea_launch_project(const ea_ctx* ctx, const ea_shape& s, const __nv_bfl
                                (uint64_t)d_model * 2, (uint64_t)p.n_cols * d_model * 2, 64, kPjTile))
         return EA_ERR_CUDA;
     const int smem = p.stages * stage_bytes + 1024 + 256;
-    if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-        return EA_ERR_CUDA;
+    EA_CUDA_TRY(cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const dim3 grid((unsigned)((p.n_cols + kPjTile - 1) / kPjTile), (unsigned)s.n_units);
     if (grid.y > 65535u) return EA_ERR_UNSUPPORTED;
     project_kernel<<<grid, kPjThreads, smem, st>>>(h_map, w_map, p);
     ea_count_launches(ctx, 1);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }

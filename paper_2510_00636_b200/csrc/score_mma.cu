@@ -26,7 +26,16 @@
 // next.  With PAIR, two CTAs of a cluster work as one (cta_group::2): each stages its own 128 keys
 // and half of the image rows, the leader issues M = 256 MMAs for both, and each CTA runs the
 // epilogue of its own keys; this is what lets head_dim 256 fit in shared memory.
+// Key tiles live in a ring of 16 KiB chunk slots (64 channels of 128 keys).  At head_dim 256 the
+// ring holds little more than two tiles, so a slot must go back to the producer as early as it
+// can: there the epilogue warps copy their part of the key rows into registers while the tile's
+// MMAs are still running, and a slot is free once those warps and the MMAs of its chunk (a
+// tcgen05.commit per chunk) are done with it; the next load then has a whole tile's MMA time to
+// cross HBM.  At head_dim <= 128 the ring is four tiles deep and the epilogue reads the key rows
+// from shared memory as it goes.
 // Every wait is bounded; a wait that gives up raises the context's status word.
+#include <mutex>
+
 #include "ea_internal.h"
 #include "ptx_sm100.cuh"
 
@@ -45,15 +54,16 @@ template <int D, bool PAIR>
 struct Geo {
     static constexpr int HPC = 256 / D;                  // query heads per pass (1, 2 or 4)
     static constexpr int KCH = D / 64;                   // 64-channel (128-byte) chunks per row
-    static constexpr int STAGE = KCH * kChunkA;          // bytes of one key tile
     static constexpr int IMG_ROWS = HPC * D;             // rows of a whole image (accumulator columns)
     static constexpr int CHUNK_B_FULL = IMG_ROWS * 128;  // bytes of one chunk of a whole image (global)
     static constexpr int IMG_MAIN = KCH * CHUNK_B_FULL;  // bytes of the covariance part of a whole image (global)
     static constexpr int ROWS_CTA = PAIR ? IMG_ROWS / 2 : IMG_ROWS;   // image rows one CTA keeps
     static constexpr int CHUNK_B = ROWS_CTA * 128;
     static constexpr int IMG_CTA = KCH * CHUNK_B;
-    static constexpr int STAGES = D == 256 ? 2 : 4;
-    static constexpr int NSLOT = STAGES * KCH;           // ring of 16 KiB chunk slots
+    // The epilogue takes its key rows into registers ahead of the accumulator (see the header).
+    static constexpr bool PRELOAD = D == 256;
+    static constexpr int NSLOT = D == 256 ? 9 : 4 * KCH;   // ring of 16 KiB chunk slots
+    static constexpr int VEC_BUFS = PRELOAD ? 2 : 1;     // the epilogue may still read the previous image's diagonal
     static constexpr int VEC = HPC * D * (int)sizeof(float);       // diagonal vectors of the resident heads
     // linear term: one extra K = 16 MMA step, a constant block of ones times (hi, lo) of mu' per column,
     // both as unswizzled K-major core matrices (8 rows x 16 bytes; 128 bytes on along K, 256 on along rows)
@@ -79,9 +89,12 @@ struct Geo {
     static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
     static constexpr int NBAR = 2 * NSLOT + 6;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + STAGES * STAGE + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
-    // warps that must release a chunk slot before it is refilled
-    static constexpr int SLOT_RELEASERS = D == 64 ? kEpiWarps : kEpiWarps / 2;
+    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + ONES + LIN_CTA + VEC_BUFS * VEC + DIAG_FULL + PART + RED + CTRL + 1024;
+    // arrivals that hand a chunk slot back to the producer: the epilogue warps that read it and,
+    // with PRELOAD, the commit of the chunk's MMAs
+    static constexpr int SLOT_READERS = D == 64 ? kEpiWarps : kEpiWarps / 2;
+    static constexpr int SLOT_RELEASERS = SLOT_READERS + (PRELOAD ? 1 : 0);
+    static_assert(!PRELOAD || KCH >= 2, "each half of the epilogue warps owns whole chunks");
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
@@ -244,13 +257,13 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_img = base;
     const uint32_t s_k = s_img + G::IMG_CTA;
-    constexpr int kOffOnes = G::IMG_CTA + G::STAGES * G::STAGE;
+    constexpr int kOffOnes = G::IMG_CTA + G::NSLOT * kChunkA;
     const uint32_t s_ones = base + kOffOnes;
     const uint32_t s_lin = s_ones + G::ONES;
     constexpr int kOffVec = kOffOnes + G::ONES + G::LIN_CTA;
-    const uint32_t s_vec = base + kOffVec;
-    const uint32_t s_diag = s_vec + G::VEC;                      // 16 x 16 diagonal blocks (d <= 128)
-    constexpr int kOffPart = kOffVec + G::VEC + G::DIAG_FULL;
+    const uint32_t s_vec = base + kOffVec;                       // VEC_BUFS buffers of VEC bytes
+    const uint32_t s_diag = s_vec + G::VEC_BUFS * G::VEC;        // 16 x 16 diagonal blocks (d <= 128)
+    constexpr int kOffPart = kOffVec + G::VEC_BUFS * G::VEC + G::DIAG_FULL;
     float* part_gen = reinterpret_cast<float*>(gen_base + kOffPart);
     float* red_gen = reinterpret_cast<float*>(gen_base + kOffPart + G::PART);
     const uint32_t s_bar = base + kOffPart + G::PART + G::RED;
@@ -270,7 +283,9 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < G::NSLOT; ++s) {
-            mbar_init(full_k(s), 1);
+            // A chunk has landed when this CTA's own copy is in; the leader of a pair also needs the
+            // peer's report that its copy is in (the MMA reads both CTAs' keys).
+            mbar_init(full_k(s), PAIR && leader ? 2 : 1);
             mbar_init(empty_k(s), G::SLOT_RELEASERS);
         }
         for (int a = 0; a < 2; ++a) {
@@ -312,23 +327,28 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     const long long first = p.n_work * my_group / p.n_groups;
     const long long last = p.n_work * (my_group + 1) / p.n_groups;
     constexpr int kKeysPerStep = PAIR ? 2 * kTileKeys : kTileKeys;
+    // Chunk number c = tile_no * KCH + kc of this worker's stream of key tiles lives in ring slot
+    // c % NSLOT, on its (c / NSLOT)-th use.
+    auto slot_of = [](long long c) { return (int)(c % G::NSLOT); };
+    auto use_of = [](long long c) { return (uint32_t)(c / G::NSLOT); };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            long long tile_no = 0, cur_img = -1;
+            long long tile_no = 0, cur_img = -1, issued = 0;      // issued: chunks whose copy has been started
+            int img_no = 0;
             bool ok = true;
             for (long long item = first; ok && item < last; ++item) {
                 const Item it = decode_item(item, my_hs, p, G::HPC);
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
-                    // every tile that used the resident image must have left the epilogue
-                    for (int back = 1; ok && back <= G::STAGES && back <= tile_no; ++back) {
-                        const long long tn = tile_no - back;
-                        const int stage = (int)(tn % G::STAGES);
-                        const uint32_t fill = (uint32_t)(tn / G::STAGES);
-                        for (int kc = 0; ok && kc < G::KCH; ++kc)
-                            ok = mbar_wait(empty_k(stage * G::KCH + kc), fill & 1, abort_flag);
+                    // Every chunk that used the resident image must have been handed back: its MMAs are
+                    // done (PRELOAD: the chunk's commit, which also covers the linear-term step issued
+                    // before it; otherwise the epilogue only runs after the tile's MMAs) and so are the
+                    // epilogues of all tiles but possibly the last one, which reads the other diagonal buffer.
+                    for (int back = 1; ok && back <= G::NSLOT && back <= issued; ++back) {
+                        const long long c = issued - back;
+                        ok = mbar_wait(empty_k(slot_of(c)), use_of(c) & 1, abort_flag);
                     }
                     if (!ok) break;
                     const int rows_total = (G::DIAG_MMA ? G::HPC : it.hpc) * D;     // interleaved heads: every row
@@ -345,35 +365,31 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         bulk_load(s_img + kc * G::CHUNK_B, src + (size_t)kc * G::CHUNK_B_FULL, rows * 128, img_full);
                     bulk_load(s_lin, img + G::IMG_MAIN + (size_t)rank * rows * 32, rows * 32, img_full);
                     if (G::DIAG_MMA) bulk_load(s_diag, img + G::IMG_MAIN + G::LIN_FULL, vec_bytes, img_full);
-                    else bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
+                    else bulk_load(s_vec + (uint32_t)((img_no % G::VEC_BUFS) * G::VEC),
+                                   p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
+                    ++img_no;
                     cur_img = img_id;
                 }
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                    const int stage = (int)(tile_no % G::STAGES);
-                    const uint32_t fill = (uint32_t)(tile_no / G::STAGES);
                     const int key0 = t * kKeysPerStep + (int)rank * kTileKeys;
                     for (int kc = 0; ok && kc < G::KCH; ++kc) {
-                        const int slot = stage * G::KCH + kc;
-                        ok = mbar_wait(empty_k(slot), (fill & 1) ^ 1, abort_flag);
+                        const long long c = tile_no * G::KCH + kc;
+                        const int slot = slot_of(c);
+                        ok = mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        if (PAIR) {
-                            if (leader) mbar_arrive_expect_tx(full_k(slot), 2 * kChunkA);
-                            tma_load_3d_pair(s_k + slot * kChunkA, &k_map, mapa(full_k(slot), 0), kc * 64, key0,
-                                             it.ug);
-                        } else {
-                            mbar_arrive_expect_tx(full_k(slot), kChunkA);
-                            tma_load_3d(s_k + slot * kChunkA, &k_map, full_k(slot), kc * 64, key0, it.ug);
-                        }
+                        mbar_arrive_expect_tx(full_k(slot), kChunkA);
+                        tma_load_3d(s_k + slot * kChunkA, &k_map, full_k(slot), kc * 64, key0, it.ug);
+                        issued = c + 1;
                     }
                 }
             }
-            if (!ok && !PAIR) {
-                // let the copies already in flight land before the CTA's shared memory goes away
-                for (int back = 1; back <= G::STAGES && back <= tile_no; ++back) {
-                    const long long tn = tile_no - back;
-                    for (int kc = 0; kc < G::KCH; ++kc)
-                        mbar_wait(full_k((int)(tn % G::STAGES) * G::KCH + kc), (uint32_t)(tn / G::STAGES) & 1,
-                                  abort_flag);
+            if (!ok) {
+                // Let this CTA's copies already in flight land before its shared memory goes away.  (The
+                // leader of a pair also waits here for the peer's reports, which may never come: the
+                // drain is bounded by time.)
+                for (int back = 1; back <= G::NSLOT && back <= issued; ++back) {
+                    const long long c = issued - back;
+                    mbar_drain(full_k(slot_of(c)), use_of(c) & 1);
                 }
             }
         }
@@ -399,41 +415,45 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 const uint32_t n_cols = (uint32_t)((G::DIAG_MMA ? G::HPC : it.hpc) * D);
                 const uint32_t idesc = PAIR ? umma_idesc_bf16_m256(n_cols) : umma_idesc_bf16_m128(n_cols);
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                    const int stage = (int)(tile_no % G::STAGES);
-                    const uint32_t fill = (uint32_t)(tile_no / G::STAGES);
                     const int a = (int)(tile_no & 1);
                     const uint32_t use = (uint32_t)(tile_no >> 1);
                     ok = mbar_wait<PAIR>(tmem_empty(a), (use & 1) ^ 1, abort_flag);
                     if (!ok) break;
+                    tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(a * kAccCols);
+                    {   // linear term first, overwriting the stage: D = ones . (hi, lo of mu')^T
+                        const uint64_t da = umma_desc_k_plain(s_ones);
+                        const uint64_t db = umma_desc_k_plain(s_lin);
+                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, 0u);
+                        else umma_bf16(d_tmem, da, db, idesc, 0u);
+                    }
 #pragma unroll
                     for (int kc = 0; kc < G::KCH; ++kc) {
-                        const int slot = stage * G::KCH + kc;
-                        ok = ok && mbar_wait<PAIR>(full_k(slot), fill & 1, abort_flag);
+                        const long long c = tile_no * G::KCH + kc;
+                        const int slot = slot_of(c);
+                        ok = ok && mbar_wait<PAIR>(full_k(slot), use_of(c) & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after_sync();
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {
                             const uint64_t da = umma_desc_k_sw128(s_k + slot * kChunkA + ks * 32);
                             const uint64_t db = umma_desc_k_sw128(s_img + kc * G::CHUNK_B + ks * 32);
-                            const uint32_t acc = (kc | ks) ? 1u : 0u;
-                            if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, acc);
-                            else umma_bf16(d_tmem, da, db, idesc, acc);
+                            if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, 1u);
+                            else umma_bf16(d_tmem, da, db, idesc, 1u);
+                        }
+                        if (G::PRELOAD) {
+                            // the slot goes back to the producers of both CTAs once these MMAs have read it
+                            if (PAIR) umma_commit_pair(empty_k(slot), 3);
+                            else umma_commit(empty_k(slot));
                         }
                     }
                     if (!ok) break;
-                    {   // linear term: D += ones . (hi, lo of mu')^T
-                        const uint64_t da = umma_desc_k_plain(s_ones);
-                        const uint64_t db = umma_desc_k_plain(s_lin);
-                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, 1u);
-                        else umma_bf16(d_tmem, da, db, idesc, 1u);
-                    }
                     if (G::DIAG_MMA) {
                         // D[:, c] += k_c * lo(diag_c) for every head: one N = 16 HPC step per 16 channels
                         const uint32_t idesc_d = umma_idesc_bf16_m128(16 * G::HPC);
 #pragma unroll
                         for (int ks = 0; ks < D / 16; ++ks) {
-                            const int slot = stage * G::KCH + ks / 4;
+                            const int slot = slot_of(tile_no * G::KCH + ks / 4);
                             umma_bf16(d_tmem + (uint32_t)(ks * 16 * G::HPC),
                                       umma_desc_k_sw128(s_k + slot * kChunkA + (ks % 4) * 32),
                                       umma_desc_k_plain(s_diag + (uint32_t)(ks * G::DIAG_BLOCK)), idesc_d, 1u);
@@ -444,8 +464,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 }
             }
         } else if (PAIR && lane == 0) {
-            // ---------------------------------------------- peer: report each landed image half
-            long long cur_img = -1;
+            // ------------- peer: report each landed image half and each landed key chunk to the leader
+            long long tile_no = 0, cur_img = -1;
             int img_loads = 0;
             bool ok = true;
             for (long long item = first; ok && item < last; ++item) {
@@ -457,6 +477,13 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     mbar_arrive_cluster(mapa(img_peer, 0));
                     ++img_loads;
                     cur_img = img_id;
+                }
+                for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
+                    for (int kc = 0; ok && kc < G::KCH; ++kc) {
+                        const long long c = tile_no * G::KCH + kc;
+                        ok = mbar_wait(full_k(slot_of(c)), use_of(c) & 1, abort_flag);
+                        if (ok) mbar_arrive_cluster(mapa(full_k(slot_of(c)), 0));
+                    }
                 }
             }
         }
@@ -474,6 +501,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         constexpr int CB = D / 32;                 // 32-column blocks per head
         constexpr int CBH = CB / 2;                // of which this warp handles half
         constexpr int NB = CBH * G::HPC;           // blocks per tile for this warp
+        constexpr int CPH = G::PRELOAD ? G::KCH / 2 : 1;   // PRELOAD: whole chunks owned by this half
         const uint32_t empty_remote = PAIR ? mapa(tmem_empty(0), 0) : 0u;
         long long tile_no = 0, cur_img = -1;
         int img_loads = 0;
@@ -487,6 +515,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 ++img_loads;
                 cur_img = img_id;
             }
+            const uint32_t s_vec_cur = s_vec + (uint32_t)(((img_loads - 1) % G::VEC_BUFS) * G::VEC);
             const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
             const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
             // running (max, sum of exp) of this thread's keys, for the heads this half finishes
@@ -494,22 +523,54 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 #pragma unroll
             for (int j = 0; j < G::HPC; ++j) { m_run[j] = -INFINITY; l_run[j] = 0.f; }
             for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                const int stage = (int)(tile_no % G::STAGES);
                 const int a = (int)(tile_no & 1);
-                bool my_ok = img_ok && mbar_wait<PAIR>(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag);
+                const long long c_tile = tile_no * G::KCH;
+                bool my_ok = img_ok;
+                // PRELOAD: this thread's half of its key row, packed bf16 pairs, taken while the tile's
+                // MMAs are still running; the slots then only wait for those MMAs
+                uint32_t kreg[G::PRELOAD ? D / 4 : 1];
+                if constexpr (G::PRELOAD) {
+#pragma unroll
+                    for (int q = 0; q < CPH; ++q) {
+                        const long long c = c_tile + half * CPH + q;
+                        my_ok = my_ok && mbar_wait(full_k(slot_of(c)), use_of(c) & 1, abort_flag);
+                    }
+                    my_ok = __all_sync(0xffffffffu, my_ok);
+                    if (my_ok) {
+#pragma unroll
+                        for (int q = 0; q < CPH; ++q) {
+                            const int slot = slot_of(c_tile + half * CPH + q);
+                            const uint32_t k_row = s_k + slot * kChunkA + row * 128;
+#pragma unroll
+                            for (int unit = 0; unit < 8; ++unit) {
+                                const uint4 w = lds128(k_row + ((unit ^ (row & 7)) << 4));
+                                kreg[q * 32 + unit * 4 + 0] = w.x;
+                                kreg[q * 32 + unit * 4 + 1] = w.y;
+                                kreg[q * 32 + unit * 4 + 2] = w.z;
+                                kreg[q * 32 + unit * 4 + 3] = w.w;
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) {
+#pragma unroll
+                            for (int q = 0; q < CPH; ++q) mbar_arrive(empty_k(slot_of(c_tile + half * CPH + q)));
+                        }
+                    }
+                }
+                my_ok = my_ok && mbar_wait<PAIR>(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag);
                 my_ok = __all_sync(0xffffffffu, my_ok);
                 float s_out[G::HPC];
                 float* part = part_gen + (tile_no & 1) * (G::HPC * kTileKeys);
                 if (my_ok) {
                     tc_fence_after_sync();
-                    const uint32_t k_row = s_k + stage * G::STAGE + row * 128;
                     float2 acc[G::HPC][2];
 #pragma unroll
                     for (int j = 0; j < G::HPC; ++j) acc[j][0] = acc[j][1] = make_float2(0.f, 0.f);
                     // block b -> (columns c0 .. c0 + BW of head j): heads innermost so the unpacked key values
                     // are reused.  Narrow blocks at d <= 128, where the epilogue is the limit: half the
-                    // registers per block leave the scheduler room to overlap the dependent FMAs.
-                    constexpr int BW = D == 256 ? 32 : 16;
+                    // registers per block leave the scheduler room to overlap the dependent FMAs; narrow
+                    // blocks with PRELOAD too, where the key row already takes D / 4 registers.
+                    constexpr int BW = (D == 256 && !G::PRELOAD) ? 32 : 16;
                     constexpr int NBW = NB * (32 / BW);
                     auto c0_of = [&](int b) { return half * CBH * 32 + (b / G::HPC) * BW; };
                     auto addr_of = [&](int b) {
@@ -523,15 +584,24 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         const int j = b % G::HPC;
                         const int c0 = c0_of(b);
                         if (j == 0) {
+                            if constexpr (G::PRELOAD) {
 #pragma unroll
-                            for (int q = 0; q < BW / 8; ++q) {
-                                const int unit = (c0 % 64) / 8 + q;
-                                const uint4 w = lds128(k_row + (c0 / 64) * kChunkA + ((unit ^ (row & 7)) << 4));
-                                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                                for (int e = 0; e < BW / 2; ++e) {
+                                    const uint32_t w = kreg[(b / G::HPC) * (BW / 2) + e];
+                                    kf[e] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                                }
+                            } else {
+                                const uint32_t k_row = s_k + slot_of(c_tile + c0 / 64) * kChunkA + row * 128;
 #pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
-                                                                __uint_as_float(ww[e] & 0xffff0000u));
+                                for (int q = 0; q < BW / 8; ++q) {
+                                    const int unit = (c0 % 64) / 8 + q;
+                                    const uint4 w = lds128(k_row + ((unit ^ (row & 7)) << 4));
+                                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e)
+                                        kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
+                                                                    __uint_as_float(ww[e] & 0xffff0000u));
+                                }
                             }
                         }
                         // the block's diagonal constants, requested before the accumulator wait so that
@@ -539,7 +609,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         uint4 dgv[BW / 4];
                         if (!G::DIAG_MMA && j < it.hpc) {
 #pragma unroll
-                            for (int q = 0; q < BW / 4; ++q) dgv[q] = lds128(s_vec + (uint32_t)((j * D + c0 + 4 * q) * 4));
+                            for (int q = 0; q < BW / 4; ++q) dgv[q] = lds128(s_vec_cur + (uint32_t)((j * D + c0 + 4 * q) * 4));
                         }
                         tmem_ld_wait();
                         if (b + 1 < NBW && (b + 1) % G::HPC < it.hpc) tmem_ld_cols(addr_of(b + 1), dv[(b + 1) & 1]);
@@ -567,11 +637,13 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                                 acc[j][1] = fma2(k1, t1, acc[j][1]);
                             }
                         }
-                        // hand the 64-channel chunk back to the producer once this warp is done with it
-                        const bool chunk_done = j == G::HPC - 1 && (D == 64 ? b == NBW - 1 : (c0 + BW) % 64 == 0);
-                        if (chunk_done) {
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(empty_k(stage * G::KCH + c0 / 64));
+                        if constexpr (!G::PRELOAD) {
+                            // hand the 64-channel chunk back to the producer once this warp is done with it
+                            const bool chunk_done = j == G::HPC - 1 && (D == 64 ? b == NBW - 1 : (c0 + BW) % 64 == 0);
+                            if (chunk_done) {
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(empty_k(slot_of(c_tile + c0 / 64)));
+                            }
                         }
                     }
                     // the accumulator stage is free again
@@ -702,8 +774,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
 
     sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(form, s.n_q_heads, s.n_kv_heads, image, vec);
     auto kern = logits_mma_kernel<D, PAIR>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM) != cudaSuccess)
-        return EA_ERR_CUDA;
+    EA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
     const long long want = (long long)p.n_groups * p.n_subsets;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * want : want));
@@ -721,8 +792,8 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     cudaEvent_t stop = ea_profile_mark_start(ctx, st);
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, k_map, p);
     ea_profile_mark_stop(ctx, stop, st);
-    if (err != cudaSuccess) return EA_ERR_CUDA;
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    EA_CUDA_TRY(err);
+    return EA_CHECK_LAUNCH();
 }
 
 }  // namespace
@@ -735,10 +806,10 @@ bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint
                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                         CUtensorMapFloatOOBfill);
+    // resolved once, under std::call_once: first calls may come from several host threads
+    static std::once_flag once;
     static encode_tiled_fn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    std::call_once(once, [] {
         void* ptr = nullptr;
         cudaDriverEntryPointQueryResult res;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) == cudaSuccess &&
@@ -746,7 +817,7 @@ bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint
             fn = reinterpret_cast<encode_tiled_fn>(ptr);
         else
             cudaGetLastError();
-    }
+    });
     if (!fn) return false;
     const cuuint64_t dims[3] = {n0, n1, n2};
     const cuuint64_t strides[2] = {stride1, stride2};

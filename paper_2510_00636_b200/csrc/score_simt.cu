@@ -96,5 +96,5 @@ ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv
             return EA_ERR_UNSUPPORTED;
     }
     ea_profile_mark_stop(ctx, stop, st);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }

@@ -578,7 +578,7 @@ static ea_status launch_select(const ea_ctx* ctx, const ea_shape& s, const float
     } else {
         select_kernel<<<heads, kSelThreads, 0, st>>>(scores, s.n_keys, n_kept, plan, kept_idx);
     }
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
@@ -597,7 +597,7 @@ ea_status ea_launch_select_adaptive(const ea_ctx* ctx, const ea_shape& s, const 
                                     cudaStream_t st) {
     const size_t units = (size_t)s.n_units, heads = units * (size_t)s.n_kv_heads;
     const AdaptiveWs a = adaptive_ws(ws, units, heads);
-    if (cudaMemsetAsync(ws, 0, ea_adaptive_ws_bytes(s), st) != cudaSuccess) return EA_ERR_CUDA;
+    EA_CUDA_TRY(cudaMemsetAsync(ws, 0, ea_adaptive_ws_bytes(s), st));
     const unsigned long long places = (unsigned long long)s.n_kv_heads * (unsigned long long)(n_kept - n_floor);
     const dim3 hist_grid((unsigned)heads, (unsigned)((s.n_keys + kAdSpan - 1) / kAdSpan));
     if (hist_grid.y > 65535u) return EA_ERR_UNSUPPORTED;
@@ -609,7 +609,7 @@ ea_status ea_launch_select_adaptive(const ea_ctx* ctx, const ea_shape& s, const 
                                                                 a.above, a.head_kept, head_offsets);
         ea_count_launches(ctx, s.n_keys > 0 ? 2 : 1);
     }
-    if (cudaGetLastError() != cudaSuccess) return EA_ERR_CUDA;
+    if (EA_CHECK_LAUNCH() != EA_OK) return EA_ERR_CUDA;
     const HeadPlan plan = {a.head_kept, head_offsets, s.n_kv_heads, s.n_kv_heads * n_kept};
     // n_kept here only says "some head may keep something"; every head reads its own count
     return launch_select(ctx, s, scores, n_kept, plan, kept_idx, st);
@@ -647,7 +647,7 @@ ea_status ea_launch_gather_adaptive(const ea_ctx* ctx, const ea_shape& s, int n_
         default:
             return EA_ERR_UNSUPPORTED;
     }
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
@@ -678,7 +678,7 @@ ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, con
         default:
             return EA_ERR_UNSUPPORTED;
     }
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
@@ -694,5 +694,5 @@ ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_
         case 256: compact_inplace_kernel<256><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
         default: return EA_ERR_UNSUPPORTED;
     }
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }

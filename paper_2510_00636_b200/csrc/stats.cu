@@ -271,7 +271,7 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
     }
     if (!ok) return EA_ERR_CUDA;
     ea_count_launches(ctx, 2);
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }
 
 ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
@@ -372,5 +372,5 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
                                                                      s->rope_layout, inv_norm, mu_bar, sigma_bar);
             break;
     }
-    return cudaGetLastError() == cudaSuccess ? EA_OK : EA_ERR_CUDA;
+    return EA_CHECK_LAUNCH();
 }

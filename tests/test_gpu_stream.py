@@ -92,6 +92,10 @@ def test_compression_event_replays_as_a_cuda_graph(ea, oracle):
     torch.cuda.current_stream().wait_stream(side)
     graph = torch.cuda.CUDAGraph()
     load(0)
+    # A Context that the garbage collector happens to destroy while the capture is open would call
+    # cudaFree, which invalidates a capture: collect what earlier tests left behind first.
+    import gc
+    gc.collect()
     with torch.cuda.graph(graph):
         event()
     for layer in (1, 2, 0):

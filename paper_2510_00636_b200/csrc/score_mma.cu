@@ -21,18 +21,15 @@
 //   warp 0     TMA producer (one lane): covariance image (bulk copy) and key tiles (tiled, 128B swizzle)
 //   warp 1     MMA issuer (one lane); owns the tensor-memory allocation
 //   warps 2-9  epilogue, two warps per tensor-memory lane quarter: thread <-> accumulator lane <-> key;
-//              each reads half of its key row from the staged tile and the matching accumulator columns
+//              each reads its half of the key row and the matching accumulator columns, the halves of a
+//              key meet in shared memory
 // Tensor memory holds two accumulator stages so the epilogue of one tile overlaps the MMAs of the
 // next.  With PAIR, two CTAs of a cluster work as one (cta_group::2): each stages its own 128 keys
 // and half of the image rows, the leader issues M = 256 MMAs for both, and each CTA runs the
 // epilogue of its own keys; this is what lets head_dim 256 fit in shared memory.
-// Key tiles live in a ring of 16 KiB chunk slots (64 channels of 128 keys).  At head_dim 256 the
-// ring holds little more than two tiles, so a slot must go back to the producer as early as it
-// can: there the epilogue warps copy their part of the key rows into registers while the tile's
-// MMAs are still running, and a slot is free once those warps and the MMAs of its chunk (a
-// tcgen05.commit per chunk) are done with it; the next load then has a whole tile's MMA time to
-// cross HBM.  At head_dim <= 128 the ring is four tiles deep and the epilogue reads the key rows
-// from shared memory as it goes.
+// Key tiles live in a ring of 16 KiB chunk slots (64 channels of 128 keys): two tiles deep at
+// head_dim 256, four at head_dim <= 128.  The epilogue reads the key rows from the slots as it works
+// through the accumulator and hands each slot back as soon as its warps are done with it.
 // Every wait is bounded; a wait that gives up raises the context's status word.
 #include <mutex>
 
@@ -44,8 +41,6 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileKeys = 128;                     // keys per CTA per step
-constexpr int kEpiWarps = 8;
-constexpr int kMmaThreads = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;                      // columns of one accumulator stage
 constexpr int kChunkA = kTileKeys * 128;           // bytes of one 64-channel chunk of a key tile
@@ -60,10 +55,12 @@ struct Geo {
     static constexpr int ROWS_CTA = PAIR ? IMG_ROWS / 2 : IMG_ROWS;   // image rows one CTA keeps
     static constexpr int CHUNK_B = ROWS_CTA * 128;
     static constexpr int IMG_CTA = KCH * CHUNK_B;
-    // The epilogue takes its key rows into registers ahead of the accumulator (see the header).
-    static constexpr bool PRELOAD = D == 256;
-    static constexpr int NSLOT = D == 256 ? 9 : 4 * KCH;   // ring of 16 KiB chunk slots
-    static constexpr int VEC_BUFS = PRELOAD ? 2 : 1;     // the epilogue may still read the previous image's diagonal
+    // Epilogue: EPI_PARTS warps per tensor-memory lane quarter, each with CPP columns of every head.
+    static constexpr int EPI_PARTS = 2;
+    static constexpr int EPI_WARPS = 4 * EPI_PARTS;
+    static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+    static constexpr int CPP = D / EPI_PARTS;
+    static constexpr int NSLOT = (D == 256 ? 2 : 4) * KCH;   // ring of 16 KiB chunk slots: 2 or 4 key tiles
     static constexpr int VEC = HPC * D * (int)sizeof(float);       // diagonal vectors of the resident heads
     // linear term: one extra K = 16 MMA step, a constant block of ones times (hi, lo) of mu' per column,
     // both as unswizzled K-major core matrices (8 rows x 16 bytes; 128 bytes on along K, 256 on along rows)
@@ -73,8 +70,7 @@ struct Geo {
     // At d <= 128 the epilogue is the limit, so the diagonal goes to the tensor cores as well: its bf16
     // part sits on the image's diagonal, and the bf16 rounding of what that leaves is added by one
     // M128 N16 K16 step per (head, 16 channels) against a 16 x 16 diagonal block (unswizzled core
-    // matrices, 512 bytes).  At d = 256 the tensor pipe is the limit and the diagonal stays in fp32 in
-    // the epilogue.
+    // matrices, 512 bytes).  At d = 256 the diagonal stays in fp32 in the epilogue.
     static constexpr bool DIAG_MMA = D <= 128;
     static constexpr int DIAG_BLOCK = 16 * HPC * 32;                    // bytes: 16 HPC rows x 16 bf16
     static constexpr int DIAG_FULL = DIAG_MMA ? (D / 16) * DIAG_BLOCK : 0;   // per whole image
@@ -85,16 +81,14 @@ struct Geo {
         return DIAG_MMA ? (c / 16) * (16 * HPC) + j * 16 + c % 16 : j * D + c;
     }
     static constexpr int IMG_FULL = IMG_MAIN + LIN_FULL + DIAG_FULL;   // bytes of a whole image (global)
-    static constexpr int PART = 2 * HPC * kTileKeys * (int)sizeof(float);   // partial sums of the two column halves
+    // partial sums of the column parts: [tile parity][part][head][key]
+    static constexpr int PART = 2 * EPI_PARTS * HPC * kTileKeys * (int)sizeof(float);
     static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
     static constexpr int NBAR = 2 * NSLOT + 6;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + ONES + LIN_CTA + VEC_BUFS * VEC + DIAG_FULL + PART + RED + CTRL + 1024;
-    // arrivals that hand a chunk slot back to the producer: the epilogue warps that read it and,
-    // with PRELOAD, the commit of the chunk's MMAs
-    static constexpr int SLOT_READERS = D == 64 ? kEpiWarps : kEpiWarps / 2;
-    static constexpr int SLOT_RELEASERS = SLOT_READERS + (PRELOAD ? 1 : 0);
-    static_assert(!PRELOAD || KCH >= 2, "each half of the epilogue warps owns whole chunks");
+    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
+    // epilogue warps that read a chunk slot and hand it back to the producer
+    static constexpr int SLOT_READERS = D == 64 ? EPI_WARPS : 4;
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
@@ -232,7 +226,8 @@ __device__ __forceinline__ Item decode_item(long long w, int hs, const MmaParams
     return it;
 }
 
-// AND of `ok` over all epilogue threads (named barrier 1): keeps their control flow identical.
+// AND of `ok` over all NT epilogue threads (named barrier 1): keeps their control flow identical.
+template <int NT>
 __device__ __forceinline__ bool epi_all(bool ok) {
     uint32_t r;
     asm volatile(
@@ -241,13 +236,13 @@ __device__ __forceinline__ bool epi_all(bool ok) {
         "bar.red.and.pred p, 1, %2, q;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(r)
-        : "r"((uint32_t)ok), "n"(32 * kEpiWarps)
+        : "r"((uint32_t)ok), "n"(NT)
         : "memory");
     return r != 0;
 }
 
 template <int D, bool PAIR>
-__global__ void __launch_bounds__(kMmaThreads, 1)
+__global__ void __launch_bounds__(Geo<D, PAIR>::THREADS, 1)
 logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) {
     using G = Geo<D, PAIR>;
     static_assert(!(G::DIAG_MMA && PAIR), "the diagonal blocks are laid out for a single CTA");
@@ -261,13 +256,14 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     const uint32_t s_ones = base + kOffOnes;
     const uint32_t s_lin = s_ones + G::ONES;
     constexpr int kOffVec = kOffOnes + G::ONES + G::LIN_CTA;
-    const uint32_t s_vec = base + kOffVec;                       // VEC_BUFS buffers of VEC bytes
-    const uint32_t s_diag = s_vec + G::VEC_BUFS * G::VEC;        // 16 x 16 diagonal blocks (d <= 128)
-    constexpr int kOffPart = kOffVec + G::VEC_BUFS * G::VEC + G::DIAG_FULL;
+    const uint32_t s_vec = base + kOffVec;                       // fp32 diagonals (d = 256)
+    const uint32_t s_diag = s_vec + G::VEC;        // 16 x 16 diagonal blocks (d <= 128)
+    constexpr int kOffPart = kOffVec + G::VEC + G::DIAG_FULL;
     float* part_gen = reinterpret_cast<float*>(gen_base + kOffPart);
     float* red_gen = reinterpret_cast<float*>(gen_base + kOffPart + G::PART);
     const uint32_t s_bar = base + kOffPart + G::PART + G::RED;
     uint8_t* bar_gen = gen_base + kOffPart + G::PART + G::RED;
+    // per ring slot: the chunk has landed / its readers are done with it
     auto full_k = [&](int slot) { return s_bar + 8u * slot; };
     auto empty_k = [&](int slot) { return s_bar + 8u * (G::NSLOT + slot); };
     auto tmem_full = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + a); };
@@ -283,14 +279,12 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < G::NSLOT; ++s) {
-            // A chunk has landed when this CTA's own copy is in; the leader of a pair also needs the
-            // peer's report that its copy is in (the MMA reads both CTAs' keys).
-            mbar_init(full_k(s), PAIR && leader ? 2 : 1);
-            mbar_init(empty_k(s), G::SLOT_RELEASERS);
+            mbar_init(full_k(s), 1);
+            mbar_init(empty_k(s), G::SLOT_READERS);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
-            mbar_init(tmem_empty(a), PAIR ? 2 * kEpiWarps : kEpiWarps);
+            mbar_init(tmem_empty(a), PAIR ? 2 * G::EPI_WARPS : G::EPI_WARPS);
         }
         mbar_init(img_full, 1);
         mbar_init(img_peer, 1);
@@ -300,7 +294,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     }
     // constant A operand of the linear-term step: K columns 0 and 1 are one, the rest zero
     // (row r of the tile at (r / 8) * 256 + (r % 8) * 16, K columns 8..15 another 128 bytes on)
-    for (int e = threadIdx.x; e < G::ONES / 16; e += kMmaThreads) {
+    for (int e = threadIdx.x; e < G::ONES / 16; e += G::THREADS) {
         const int piece = e % 16;                       // 16-byte pieces of a 256-byte group of 8 rows
         uint4 v = make_uint4(piece < 8 ? 0x3f803f80u : 0u, 0u, 0u, 0u);   // two bf16 ones, then zeros
         *reinterpret_cast<uint4*>(gen_base + kOffOnes + e * 16) = v;
@@ -336,16 +330,14 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             long long tile_no = 0, cur_img = -1, issued = 0;      // issued: chunks whose copy has been started
-            int img_no = 0;
             bool ok = true;
             for (long long item = first; ok && item < last; ++item) {
                 const Item it = decode_item(item, my_hs, p, G::HPC);
                 const long long img_id = (long long)it.ug * p.n_subsets + it.hs;
                 if (img_id != cur_img) {
-                    // Every chunk that used the resident image must have been handed back: its MMAs are
-                    // done (PRELOAD: the chunk's commit, which also covers the linear-term step issued
-                    // before it; otherwise the epilogue only runs after the tile's MMAs) and so are the
-                    // epilogues of all tiles but possibly the last one, which reads the other diagonal buffer.
+                    // Every chunk that used the resident image must have been handed back: the epilogue warps
+                    // that release a slot only run after the tile's MMAs, and by the time a warp releases its
+                    // last chunk of a tile it has also read the last of the image's diagonal.
                     for (int back = 1; ok && back <= G::NSLOT && back <= issued; ++back) {
                         const long long c = issued - back;
                         ok = mbar_wait(empty_k(slot_of(c)), use_of(c) & 1, abort_flag);
@@ -365,9 +357,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         bulk_load(s_img + kc * G::CHUNK_B, src + (size_t)kc * G::CHUNK_B_FULL, rows * 128, img_full);
                     bulk_load(s_lin, img + G::IMG_MAIN + (size_t)rank * rows * 32, rows * 32, img_full);
                     if (G::DIAG_MMA) bulk_load(s_diag, img + G::IMG_MAIN + G::LIN_FULL, vec_bytes, img_full);
-                    else bulk_load(s_vec + (uint32_t)((img_no % G::VEC_BUFS) * G::VEC),
-                                   p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
-                    ++img_no;
+                    else bulk_load(s_vec, p.vec + ((size_t)u * p.Hq + h0) * D, vec_bytes, img_full);
                     cur_img = img_id;
                 }
                 for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
@@ -377,16 +367,24 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         const int slot = slot_of(c);
                         ok = mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        mbar_arrive_expect_tx(full_k(slot), kChunkA);
-                        tma_load_3d(s_k + slot * kChunkA, &k_map, full_k(slot), kc * 64, key0, it.ug);
+                        if (PAIR) {
+                            // both CTAs' copies are counted on the leader's barrier, which the MMA issuer watches
+                            if (leader) mbar_arrive_expect_tx(full_k(slot), 2 * kChunkA);
+                            tma_load_3d_pair(s_k + slot * kChunkA, &k_map, mapa(full_k(slot), 0), kc * 64, key0,
+                                             it.ug);
+                        } else {
+                            mbar_arrive_expect_tx(full_k(slot), kChunkA);
+                            tma_load_3d(s_k + slot * kChunkA, &k_map, full_k(slot), kc * 64, key0, it.ug);
+                        }
                         issued = c + 1;
                     }
                 }
             }
-            if (!ok) {
-                // Let this CTA's copies already in flight land before its shared memory goes away.  (The
-                // leader of a pair also waits here for the peer's reports, which may never come: the
-                // drain is bounded by time.)
+            if (!ok && leader) {
+                // Let the copies already in flight land before the shared memory goes away.  In a pair the
+                // leader's barriers count both CTAs' bytes, and the peer stays until the teardown's cluster
+                // barrier, which the leader reaches only after this.  Bounded by time: a copy the peer
+                // never started is not waited for beyond that.
                 for (int back = 1; back <= G::NSLOT && back <= issued; ++back) {
                     const long long c = issued - back;
                     mbar_drain(full_k(slot_of(c)), use_of(c) & 1);
@@ -441,11 +439,6 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                             if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, 1u);
                             else umma_bf16(d_tmem, da, db, idesc, 1u);
                         }
-                        if (G::PRELOAD) {
-                            // the slot goes back to the producers of both CTAs once these MMAs have read it
-                            if (PAIR) umma_commit_pair(empty_k(slot), 3);
-                            else umma_commit(empty_k(slot));
-                        }
                     }
                     if (!ok) break;
                     if (G::DIAG_MMA) {
@@ -464,8 +457,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 }
             }
         } else if (PAIR && lane == 0) {
-            // ------------- peer: report each landed image half and each landed key chunk to the leader
-            long long tile_no = 0, cur_img = -1;
+            // ---------------------------------------------- peer: report each landed image half
+            long long cur_img = -1;
             int img_loads = 0;
             bool ok = true;
             for (long long item = first; ok && item < last; ++item) {
@@ -478,30 +471,22 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     ++img_loads;
                     cur_img = img_id;
                 }
-                for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
-                    for (int kc = 0; ok && kc < G::KCH; ++kc) {
-                        const long long c = tile_no * G::KCH + kc;
-                        ok = mbar_wait(full_k(slot_of(c)), use_of(c) & 1, abort_flag);
-                        if (ok) mbar_arrive_cluster(mapa(full_k(slot_of(c)), 0));
-                    }
-                }
             }
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ epilogue
-        // Warp (quarter, half): accumulator lanes 32*quarter.. (thread <-> lane <-> key) and the
-        // 32-column blocks [half*CB/2, (half+1)*CB/2) of every head of the pass.  The two halves of
-        // a key meet in shared memory; head j is finished and stored by half j % 2.
+        // Warp (quarter, part): accumulator lanes 32*quarter.. (thread <-> lane <-> key) and columns
+        // [part * CPP, (part + 1) * CPP) of every head of the pass.  The parts of a key meet in shared
+        // memory and are added in part order; head j is finished and stored by part j % EPI_PARTS.
         const int ew = warp - 2;
         const int quarter = warp % 4;              // the TMEM lanes this warp may read
-        const int half = ew / 4;
+        const int cp = ew / 4;                     // column part
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        constexpr int CB = D / 32;                 // 32-column blocks per head
-        constexpr int CBH = CB / 2;                // of which this warp handles half
-        constexpr int NB = CBH * G::HPC;           // blocks per tile for this warp
-        constexpr int CPH = G::PRELOAD ? G::KCH / 2 : 1;   // PRELOAD: whole chunks owned by this half
+        constexpr int BW = D == 256 ? 32 : 16;                      // accumulator columns per tensor-memory load
+        constexpr int NBW = (G::CPP / BW) * G::HPC;                 // loads per tile for this warp
+        constexpr int kEpiThreads = 32 * G::EPI_WARPS;
         const uint32_t empty_remote = PAIR ? mapa(tmem_empty(0), 0) : 0u;
         long long tile_no = 0, cur_img = -1;
         int img_loads = 0;
@@ -515,10 +500,9 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 ++img_loads;
                 cur_img = img_id;
             }
-            const uint32_t s_vec_cur = s_vec + (uint32_t)(((img_loads - 1) % G::VEC_BUFS) * G::VEC);
             const int u = it.ug / p.Hkv, g = it.ug % p.Hkv;
             const int h0 = g * (p.Hq / p.Hkv) + it.hs * G::HPC;
-            // running (max, sum of exp) of this thread's keys, for the heads this half finishes
+            // running (max, sum of exp) of this thread's keys, for the heads this part finishes
             float m_run[G::HPC], l_run[G::HPC];
 #pragma unroll
             for (int j = 0; j < G::HPC; ++j) { m_run[j] = -INFINITY; l_run[j] = 0.f; }
@@ -526,53 +510,18 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 const int a = (int)(tile_no & 1);
                 const long long c_tile = tile_no * G::KCH;
                 bool my_ok = img_ok;
-                // PRELOAD: this thread's half of its key row, packed bf16 pairs, taken while the tile's
-                // MMAs are still running; the slots then only wait for those MMAs
-                uint32_t kreg[G::PRELOAD ? D / 4 : 1];
-                if constexpr (G::PRELOAD) {
-#pragma unroll
-                    for (int q = 0; q < CPH; ++q) {
-                        const long long c = c_tile + half * CPH + q;
-                        my_ok = my_ok && mbar_wait(full_k(slot_of(c)), use_of(c) & 1, abort_flag);
-                    }
-                    my_ok = __all_sync(0xffffffffu, my_ok);
-                    if (my_ok) {
-#pragma unroll
-                        for (int q = 0; q < CPH; ++q) {
-                            const int slot = slot_of(c_tile + half * CPH + q);
-                            const uint32_t k_row = s_k + slot * kChunkA + row * 128;
-#pragma unroll
-                            for (int unit = 0; unit < 8; ++unit) {
-                                const uint4 w = lds128(k_row + ((unit ^ (row & 7)) << 4));
-                                kreg[q * 32 + unit * 4 + 0] = w.x;
-                                kreg[q * 32 + unit * 4 + 1] = w.y;
-                                kreg[q * 32 + unit * 4 + 2] = w.z;
-                                kreg[q * 32 + unit * 4 + 3] = w.w;
-                            }
-                        }
-                        __syncwarp();
-                        if (lane == 0) {
-#pragma unroll
-                            for (int q = 0; q < CPH; ++q) mbar_arrive(empty_k(slot_of(c_tile + half * CPH + q)));
-                        }
-                    }
-                }
                 my_ok = my_ok && mbar_wait<PAIR>(tmem_full(a), (uint32_t)((tile_no >> 1) & 1), abort_flag);
                 my_ok = __all_sync(0xffffffffu, my_ok);
-                float s_out[G::HPC];
-                float* part = part_gen + (tile_no & 1) * (G::HPC * kTileKeys);
+                float* part = part_gen + (tile_no & 1) * (G::EPI_PARTS * G::HPC * kTileKeys);
                 if (my_ok) {
                     tc_fence_after_sync();
                     float2 acc[G::HPC][2];
 #pragma unroll
                     for (int j = 0; j < G::HPC; ++j) acc[j][0] = acc[j][1] = make_float2(0.f, 0.f);
-                    // block b -> (columns c0 .. c0 + BW of head j): heads innermost so the unpacked key values
-                    // are reused.  Narrow blocks at d <= 128, where the epilogue is the limit: half the
-                    // registers per block leave the scheduler room to overlap the dependent FMAs; narrow
-                    // blocks with PRELOAD too, where the key row already takes D / 4 registers.
-                    constexpr int BW = (D == 256 && !G::PRELOAD) ? 32 : 16;
-                    constexpr int NBW = NB * (32 / BW);
-                    auto c0_of = [&](int b) { return half * CBH * 32 + (b / G::HPC) * BW; };
+                    // load b -> (columns c0 .. c0 + BW of head j): heads innermost so the unpacked key values
+                    // are reused.  Narrow loads at d <= 128, where the epilogue is the limit: few live registers
+                    // leave the scheduler room to overlap the dependent FMAs.
+                    auto c0_of = [&](int b) { return cp * G::CPP + (b / G::HPC) * BW; };
                     auto addr_of = [&](int b) {
                         return t_lane + (uint32_t)(a * kAccCols + G::col(b % G::HPC, c0_of(b)));
                     };
@@ -584,24 +533,16 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         const int j = b % G::HPC;
                         const int c0 = c0_of(b);
                         if (j == 0) {
-                            if constexpr (G::PRELOAD) {
+                            const uint32_t k_row = s_k + slot_of(c_tile + c0 / 64) * kChunkA + row * 128;
 #pragma unroll
-                                for (int e = 0; e < BW / 2; ++e) {
-                                    const uint32_t w = kreg[(b / G::HPC) * (BW / 2) + e];
-                                    kf[e] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-                                }
-                            } else {
-                                const uint32_t k_row = s_k + slot_of(c_tile + c0 / 64) * kChunkA + row * 128;
+                            for (int q = 0; q < BW / 8; ++q) {
+                                const int unit = (c0 % 64) / 8 + q;
+                                const uint4 w = lds128(k_row + ((unit ^ (row & 7)) << 4));
+                                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                                for (int q = 0; q < BW / 8; ++q) {
-                                    const int unit = (c0 % 64) / 8 + q;
-                                    const uint4 w = lds128(k_row + ((unit ^ (row & 7)) << 4));
-                                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e)
-                                        kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
-                                                                    __uint_as_float(ww[e] & 0xffff0000u));
-                                }
+                                for (int e = 0; e < 4; ++e)
+                                    kf[q * 4 + e] = make_float2(__uint_as_float(ww[e] << 16),
+                                                                __uint_as_float(ww[e] & 0xffff0000u));
                             }
                         }
                         // the block's diagonal constants, requested before the accumulator wait so that
@@ -609,7 +550,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         uint4 dgv[BW / 4];
                         if (!G::DIAG_MMA && j < it.hpc) {
 #pragma unroll
-                            for (int q = 0; q < BW / 4; ++q) dgv[q] = lds128(s_vec_cur + (uint32_t)((j * D + c0 + 4 * q) * 4));
+                            for (int q = 0; q < BW / 4; ++q) dgv[q] = lds128(s_vec + (uint32_t)((j * D + c0 + 4 * q) * 4));
                         }
                         tmem_ld_wait();
                         if (b + 1 < NBW && (b + 1) % G::HPC < it.hpc) tmem_ld_cols(addr_of(b + 1), dv[(b + 1) & 1]);
@@ -637,13 +578,11 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                                 acc[j][1] = fma2(k1, t1, acc[j][1]);
                             }
                         }
-                        if constexpr (!G::PRELOAD) {
-                            // hand the 64-channel chunk back to the producer once this warp is done with it
-                            const bool chunk_done = j == G::HPC - 1 && (D == 64 ? b == NBW - 1 : (c0 + BW) % 64 == 0);
-                            if (chunk_done) {
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(empty_k(slot_of(c_tile + c0 / 64)));
-                            }
+                        // hand the 64-channel chunk back to the producer once this warp is done with it
+                        const bool chunk_done = j == G::HPC - 1 && (D == 64 ? b == NBW - 1 : (c0 + BW) % 64 == 0);
+                        if (chunk_done) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(empty_k(slot_of(c_tile + c0 / 64)));
                         }
                     }
                     // the accumulator stage is free again
@@ -654,14 +593,13 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         else mbar_arrive(tmem_empty(a));
                     }
 #pragma unroll
-                    for (int j = 0; j < G::HPC; ++j) {
-                        s_out[j] = (acc[j][0].x + acc[j][1].x) + (acc[j][0].y + acc[j][1].y);
-                        if ((j & 1) != half) part[j * kTileKeys + row] = s_out[j];   // finished by the other half
-                    }
+                    for (int j = 0; j < G::HPC; ++j)
+                        part[(cp * G::HPC + j) * kTileKeys + row] =
+                            (acc[j][0].x + acc[j][1].x) + (acc[j][0].y + acc[j][1].y);
                 }
-                // one named barrier per tile: the halves exchange their partial sums, and a wait
+                // one named barrier per tile: the parts exchange their partial sums, and a wait
                 // that gave up anywhere stops every epilogue warp at the same tile
-                if (!epi_all(my_ok)) {
+                if (!epi_all<kEpiThreads>(my_ok)) {
                     ok = false;
                     break;
                 }
@@ -669,8 +607,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 if (key < p.n) {
 #pragma unroll
                     for (int j = 0; j < G::HPC; ++j)
-                        if ((j & 1) == half && j < it.hpc) {
-                            const float sv = s_out[j] + part[j * kTileKeys + row];
+                        if (j % G::EPI_PARTS == cp && j < it.hpc) {
+                            float sv = part[j * kTileKeys + row];
+#pragma unroll
+                            for (int q = 1; q < G::EPI_PARTS; ++q) sv += part[(q * G::HPC + j) * kTileKeys + row];
                             p.logits[((size_t)u * p.Hq + h0 + j) * (size_t)p.n + key] = sv;
                             const float m_new = fmaxf(m_run[j], sv);
                             l_run[j] = l_run[j] * __expf(m_run[j] - m_new) + __expf(sv - m_new);
@@ -679,10 +619,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 }
             }
             if (!ok) break;
-            // log-sum-exp partial of the work unit: lanes, then the four warps of the finishing half
+            // log-sum-exp partial of the work unit: lanes, then the four warps of the finishing part
 #pragma unroll
             for (int j = 0; j < G::HPC; ++j)
-                if ((j & 1) == half) {
+                if (j % G::EPI_PARTS == cp) {
                     float m = m_run[j], l = l_run[j];
 #pragma unroll
                     for (int off = 16; off > 0; off >>= 1) {
@@ -697,7 +637,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                         red_gen[(j * 4 + quarter) * 2 + 1] = l;
                     }
                 }
-            if (!epi_all(true)) { ok = false; break; }
+            if (!epi_all<kEpiThreads>(true)) { ok = false; break; }
             if (threadIdx.x - 64 < G::HPC && (int)(threadIdx.x - 64) < it.hpc) {
                 const int j = threadIdx.x - 64;
                 float m = -INFINITY, l = 0.f;
@@ -778,7 +718,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     const long long want = (long long)p.n_groups * p.n_subsets;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * want : want));
-    cfg.blockDim = dim3(kMmaThreads);
+    cfg.blockDim = dim3(G::THREADS);
     cfg.dynamicSmemBytes = G::SMEM;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -331,6 +331,32 @@ ea_status ea_select_compact_adaptive(ea_ctx* ctx, const ea_shape* shape, const f
 int64_t ea_n_floor(int64_t n_kept, double safeguard);
 
 /*
+ * Limits the persistent log-score kernel of this context (Eq. 7; one CTA per SM,
+ * each taking the SM's whole register file and shared memory) to n_sms SMs,
+ * so that work launched beside it - another context's memory-bound passes, a
+ * decode step of the serving engine - finds the other SMs free instead of
+ * queueing behind it (the paper has no counterpart).  n_sms = 0 restores the
+ * default, every SM of the device.  2 <= n_sms <= SM count, else
+ * EA_ERR_INVALID_ARG.  Takes effect from the next ea_score / ea_score_wo.
+ */
+ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms);
+
+/*
+ * Runs the value-norm pass of ea_score (the ||v|| of Eq. 9, which does not
+ * depend on the log-scores) on n_sms SMs of its own, beside the tensor-bound
+ * log-score kernel instead of after it (the paper has no counterpart): a
+ * persistent kernel of n_sms CTAs streams V through bulk copies on a stream the
+ * context owns, the log-score kernel takes the other SMs, and a light weighting
+ * pass joins the two.  The scores are those of the default path up to the
+ * rounding of one fp32 square root.  n_sms even, 0 <= n_sms <= SM count - 2
+ * (EA_ERR_INVALID_ARG otherwise); 0 (the default) switches the side pass off.
+ * The first call with n_sms > 0 creates the stream and two events: make it
+ * outside a stream capture.  Applies to ea_score with the tensor-core path
+ * (head_dim 64/128/256 and at least one tile of keys); other calls ignore it.
+ */
+ea_status ea_set_side_sms(ea_ctx* ctx, int32_t n_sms);
+
+/*
  * Synchronises cuda_stream and returns the device-side status recorded since
  * the last call of this function (EA_OK, EA_ERR_DEVICE_TIMEOUT, or
  * EA_ERR_CUDA if the stream reports an error), then clears it.

@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -85,6 +85,10 @@ def lib() -> ctypes.CDLL:
         L.ea_select_compact_inplace.restype = ctypes.c_int
         L.ea_selftest_wait_timeout.argtypes = [vp, i32, vp]
         L.ea_selftest_wait_timeout.restype = ctypes.c_int
+        L.ea_set_sm_budget.argtypes = [vp, i32]
+        L.ea_set_side_sms.argtypes = [vp, i32]
+        L.ea_set_side_sms.restype = ctypes.c_int
+        L.ea_set_sm_budget.restype = ctypes.c_int
         L.ea_sync_status.argtypes = [vp, vp]
         L.ea_host_workspace_bytes.argtypes = [sp, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         L.ea_compress_host.argtypes = [vp, sp, vp, vp, vp, vp, i32, f64, f32, i32, i32, vp, vp, vp, vp, vp]
@@ -175,6 +179,14 @@ class Context:
         """Launch the self-test kernel whose bounded wait runs out (see ``ea_selftest_wait_timeout``)."""
         _check(lib().ea_selftest_wait_timeout(self._h, int(limit_us), _stream(self.device)),
                "ea_selftest_wait_timeout")
+
+    def set_sm_budget(self, n_sms: int = 0):
+        """Limit the persistent log-score kernel to ``n_sms`` SMs (0: all of them)."""
+        _check(lib().ea_set_sm_budget(self._h, int(n_sms)), "ea_set_sm_budget")
+
+    def set_side_sms(self, n_sms: int = 0):
+        """Run the value-norm pass of ``ea_score`` on ``n_sms`` SMs beside the log-score kernel (0: off)."""
+        _check(lib().ea_set_side_sms(self._h, int(n_sms)), "ea_set_side_sms")
 
     def profile_begin(self):
         _check(lib().ea_profile_begin(self._h), "ea_profile_begin")

@@ -50,6 +50,7 @@ ea_ws_plan ea_plan_workspace(const ea_shape& s) {
     p.image = off;      off = ea_align_up(off + (mma ? ea_mma_image_bytes(s) : 0), 1024);
     p.vec = off;        off = ea_align_up(off + (mma ? ea_mma_vec_bytes(s) : 0), 256);
     p.lse_part = off;   off = ea_align_up(off + (mma ? ea_mma_lse_part_bytes(s) : 0), 256);
+    p.vnorm = off;      off = ea_align_up(off + (mma ? U * (size_t)s.n_kv_heads * n * sizeof(float) : 0), 256);
     p.adaptive = off;   off = ea_align_up(off + ea_adaptive_ws_bytes(s), 256);
     p.total = off;
     return p;
@@ -106,6 +107,9 @@ ea_status ea_create(ea_ctx** out_ctx, int device, size_t workspace_bytes) {
     if (!ctx) { cudaSetDevice(prev); return EA_ERR_CUDA; }
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
+    ctx->sm_budget = ctx->sm_count;
+    ctx->side_sms = 0;
+    ctx->side_ready = false;
     ctx->workspace = nullptr;
     ctx->workspace_bytes = workspace_bytes;
     ctx->status_host = nullptr;
@@ -146,6 +150,11 @@ ea_status ea_destroy(ea_ctx* ctx) {
     cudaSetDevice(ctx->device);
     if (ctx->workspace) cudaFree(ctx->workspace);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    if (ctx->side_ready) {
+        cudaStreamDestroy(ctx->st_side);
+        cudaEventDestroy(ctx->ev_fork);
+        cudaEventDestroy(ctx->ev_join);
+    }
     if (ctx->host_ready) {
         cudaStreamDestroy(ctx->st_h2d);
         cudaStreamDestroy(ctx->st_d2h);
@@ -252,11 +261,29 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     if (ea_mma_path_supported(*shape) && shape->group_mode != EA_GROUP_MEAN_LOGIT) {
         // tensor-core log-scores with the log-sum-exp partials from their epilogue
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
+        float* vnorm = reinterpret_cast<float*>(ws + plan.vnorm);
         int n_chunks = 0;
-        st = ea_launch_logits_mma(ctx, *shape, kb, eq7, ws + plan.image,
-                                  reinterpret_cast<float*>(ws + plan.vec), logits, lse_part, &n_chunks, stream);
+        const bool side = ctx->side_sms > 0;
+        if (side) {
+            // the value norms do not depend on the log-scores: their pass over V goes to a few SMs of its
+            // own, on a second stream, and is launched first so that it is resident when the log-score
+            // kernel takes the others
+            EA_CUDA_TRY(cudaEventRecord(ctx->ev_fork, stream));
+            EA_CUDA_TRY(cudaStreamWaitEvent(ctx->st_side, ctx->ev_fork, 0));
+            st = ea_launch_vnorm(ctx, *shape, vb, ctx->side_sms, vnorm, ctx->st_side);
+            if (st == EA_OK) EA_CUDA_TRY(cudaEventRecord(ctx->ev_join, ctx->st_side));
+        }
+        if (st == EA_OK)
+            st = ea_launch_logits_mma(ctx, *shape, kb, eq7, ws + plan.image,
+                                      reinterpret_cast<float*>(ws + plan.vec), logits, lse_part, &n_chunks, stream);
         if (st == EA_OK) st = ea_launch_lse_combine(ctx, *shape, lse_part, n_chunks, lse, stream);
-        if (st == EA_OK) st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, true, scores, stream);
+        if (side) {
+            // always rejoin, whatever happened in between: the caller's stream must not run ahead of the side pass
+            EA_CUDA_TRY(cudaStreamWaitEvent(stream, ctx->ev_join, 0));
+            if (st == EA_OK) st = ea_launch_weight(ctx, *shape, logits, lse, vnorm, epsilon, scores, stream);
+        } else if (st == EA_OK) {
+            st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, true, scores, stream);
+        }
     } else {
         if (ea_mma_path_supported(*shape)) {
             int n_chunks = 0;
@@ -448,6 +475,32 @@ int64_t ea_n_floor(int64_t n_kept, double safeguard) {
     if (f < 0) f = 0;
     if (f > n_kept) f = n_kept;
     return f;
+}
+
+ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    if (n_sms == 0) n_sms = ctx->sm_count;
+    if (n_sms < 2 || n_sms > ctx->sm_count) return EA_ERR_INVALID_ARG;
+    ctx->sm_budget = n_sms;
+    return EA_OK;
+}
+
+ea_status ea_set_side_sms(ea_ctx* ctx, int32_t n_sms) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    if (n_sms < 0 || n_sms % 2 != 0 || n_sms > ctx->sm_count - 2) return EA_ERR_INVALID_ARG;
+    if (n_sms > 0 && !ctx->side_ready) {
+        int prev = 0;
+        EA_CUDA_TRY(cudaGetDevice(&prev));
+        if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+        cudaError_t e = cudaStreamCreateWithFlags(&ctx->st_side, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+        if (prev != ctx->device) cudaSetDevice(prev);
+        EA_CUDA_TRY(e);
+        ctx->side_ready = true;
+    }
+    ctx->side_sms = n_sms;
+    return EA_OK;
 }
 
 ea_status ea_sync_status(ea_ctx* ctx, void* cuda_stream) {

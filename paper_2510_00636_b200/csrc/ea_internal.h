@@ -12,7 +12,12 @@
 
 struct ea_ctx {
     int device;
-    int sm_count;
+    int sm_count;        // SMs of the device
+    int sm_budget;       // SMs the persistent kernels of this context may occupy (ea_set_sm_budget)
+    int side_sms;        // SMs of the value-norm pass that runs beside the log-score kernel (0: no side pass)
+    bool side_ready;     // side stream and events exist
+    cudaStream_t st_side;
+    cudaEvent_t ev_fork, ev_join;
     void* workspace;
     size_t workspace_bytes;
     int* status_host;    // pinned, mapped: device kernels write EA_ERR_DEVICE_TIMEOUT here
@@ -49,6 +54,7 @@ struct ea_ws_plan {
     size_t image;        // bf16 covariance images of the tensor-core log-score kernel (ea_score)
     size_t vec;          // fp32 [U*Hq, d] epilogue vectors of that kernel               (ea_score)
     size_t lse_part;     // fp32 [U*Hq, chunks, 2] log-sum-exp partials of that kernel    (ea_score)
+    size_t vnorm;        // fp32 [U, Hkv, n] value norms (ea_score with a side pass, ea_set_side_sms)
     size_t adaptive;     // radix histograms, search state and per-head counts (ea_select_compact_adaptive)
     size_t total;
 };
@@ -125,6 +131,12 @@ ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_
 // log-sum-exp per softmax row from the per-work-unit partials of the tensor-core kernel
 ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const float* lse_part, int n_chunks,
                                 float* lse, cudaStream_t st);
+
+// ||v|| of every value row on n_ctas SMs (bulk-copy-fed stream), and the weighting that uses them.
+ea_status ea_launch_vnorm(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* v, int n_ctas, float* vnorm,
+                          cudaStream_t st);
+ea_status ea_launch_weight(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
+                           const float* vnorm, float epsilon, float* scores, cudaStream_t st);
 
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
                              const __nv_bfloat16* v, float epsilon, float* lse, bool lse_ready, float* scores,

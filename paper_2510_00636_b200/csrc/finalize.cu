@@ -8,6 +8,7 @@
 // shuffle-reduced), then lane r finishes key r: coalesced log-score loads,
 // exp(s - lse) per query head of the group, (a + eps) * ||v||.
 #include "ea_internal.h"
+#include "ptx_sm100.cuh"
 
 namespace {
 
@@ -120,6 +121,149 @@ finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
 }
 
 
+// ------------------------------------------------------------------------------------------
+// Value norms on a few SMs (Eq. 9's ||v||, the part of the weighting that does not depend on the
+// log-scores), so that the pass over V can run beside the tensor-bound log-score kernel instead of
+// after it.  A persistent CTA per SM streams its contiguous share of the value rows through shared
+// memory with bulk copies (cp.async.bulk: the copy engine keeps about 190 KiB in flight per SM,
+// which register-fed loads cannot).  Every warp serves itself: it owns three 4 KiB slots, waits for
+// a slot's copy, takes the rows into registers, starts the copy of its next chunk into the same slot
+// and only then reduces; no warp ever waits for another one, because each such hand-over costs
+// more than the arithmetic of a chunk.
+//   lane = (row of a group of four, eighth of the row); the eight lanes of a row read consecutive
+//   16-byte pieces (conflict-free), sum squares in fp32 and meet by shuffles; the norms of a chunk
+//   leave as one contiguous run.
+constexpr int kVnChunk = 4096;             // bytes per bulk copy
+constexpr int kVnSlots = 3;                // slots per warp
+constexpr int kVnWarps = 16;
+constexpr int kVnThreads = 32 * kVnWarps;
+constexpr int kVnSmem = kVnWarps * kVnSlots * kVnChunk;
+
+template <int D>
+__global__ void __launch_bounds__(kVnThreads, 1)
+vnorm_stream_kernel(const __nv_bfloat16* __restrict__ v, long long n_rows, float* __restrict__ vnorm,
+                    int* status) {
+    constexpr int ROW_BYTES = 2 * D;
+    constexpr int CR = kVnChunk / ROW_BYTES;           // rows per chunk (8, 16 or 32)
+    constexpr int PPL = D / 64;                        // 16-byte pieces per lane and row (8 lanes per row)
+    constexpr int NG = CR / 4;                         // groups of four rows per chunk
+    extern __shared__ __align__(1024) uint8_t vn_smem[];
+    __shared__ __align__(8) unsigned long long bars[kVnWarps][kVnSlots];
+    __shared__ float norms[kVnWarps][CR];
+    __shared__ int abort_flag;
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (threadIdx.x == 0) {
+        for (int w = 0; w < kVnWarps; ++w)
+            for (int s = 0; s < kVnSlots; ++s) ptx::mbar_init(ptx::smem_u32(&bars[w][s]), 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    // this CTA's chunks: a contiguous range; chunk c of it belongs to warp c % kVnWarps
+    const long long n_chunks = (n_rows + CR - 1) / CR;
+    const long long per = (n_chunks + gridDim.x - 1) / gridDim.x;
+    const long long c0 = per * blockIdx.x;
+    const long long c1 = c0 + per < n_chunks ? c0 + per : n_chunks;
+    const long long mine = c1 - c0 > warp ? (c1 - c0 - warp + kVnWarps - 1) / kVnWarps : 0;   // chunks of this warp
+    const uint32_t s_warp = ptx::smem_u32(vn_smem) + (uint32_t)(warp * kVnSlots * kVnChunk);
+    auto bar = [&](int s) { return ptx::smem_u32(&bars[warp][s]); };
+    auto issue = [&](long long k) {                    // lane 0: start the copy of this warp's k-th chunk
+        const long long row0 = (c0 + warp + k * kVnWarps) * CR;
+        const long long rows = n_rows - row0 < CR ? n_rows - row0 : CR;
+        const uint32_t bytes = (uint32_t)(rows * ROW_BYTES);
+        const int s = (int)(k % kVnSlots);
+        ptx::mbar_arrive_expect_tx(bar(s), bytes);
+        ptx::bulk_load(s_warp + (uint32_t)(s * kVnChunk), reinterpret_cast<const uint8_t*>(v) + row0 * ROW_BYTES, bytes,
+                       bar(s));
+    };
+    if (lane == 0)
+        for (long long k = 0; k < kVnSlots && k < mine; ++k) issue(k);
+    const int rr = lane / 8, q = lane % 8;
+    long long k = 0;
+    bool ok = true;
+    for (; k < mine; ++k) {
+        const int s = (int)(k % kVnSlots);
+        ok = ptx::mbar_wait(bar(s), (uint32_t)(k / kVnSlots) & 1, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t s_rows = s_warp + (uint32_t)(s * kVnChunk);
+        // (rows past the end read whatever the slot held and are not stored)
+        uint4 x[NG][PPL];
+#pragma unroll
+        for (int g = 0; g < NG; ++g)
+#pragma unroll
+            for (int e = 0; e < PPL; ++e)
+                x[g][e] = ptx::lds128(s_rows + (uint32_t)((4 * g + rr) * ROW_BYTES + (e * 8 + q) * 16));
+        float ss[NG];
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+            float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+            for (int e = 0; e < PPL; ++e) {
+                const uint32_t w[4] = {x[g][e].x, x[g][e].y, x[g][e].z, x[g][e].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float2 u = make_float2(__uint_as_float(w[c] << 16), __uint_as_float(w[c] & 0xffff0000u));
+                    acc[c & 1] = ptx::fma2(u, u, acc[c & 1]);
+                }
+            }
+            ss[g] = (acc[0].x + acc[1].x) + (acc[0].y + acc[1].y);
+        }
+        // every lane has consumed its pieces: the slot can take this warp's chunk k + kVnSlots
+        __syncwarp();
+        if (lane == 0 && k + kVnSlots < mine) {
+            ptx::fence_proxy_async_smem();             // the reads above are ordered before the copy engine's writes
+            issue(k + kVnSlots);
+        }
+#pragma unroll
+        for (int off = 4; off > 0; off >>= 1)
+#pragma unroll
+            for (int g = 0; g < NG; ++g) ss[g] += __shfl_xor_sync(0xffffffffu, ss[g], off);
+        if (q == 0) {
+#pragma unroll
+            for (int g = 0; g < NG; ++g) norms[warp][4 * g + rr] = sqrtf(ss[g]);
+        }
+        __syncwarp();
+        const long long row0 = (c0 + warp + k * kVnWarps) * CR;
+#pragma unroll
+        for (int r = lane; r < CR; r += 32)
+            if (row0 + r < n_rows) vnorm[row0 + r] = norms[warp][r];
+        __syncwarp();
+    }
+    if (!ok && lane == 0) {
+        // let this warp's copies already in flight land before the shared memory goes away
+        for (long long j = k; j < k + kVnSlots && j < mine; ++j)
+            ptx::mbar_drain(bar((int)(j % kVnSlots)), (uint32_t)(j / kVnSlots) & 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) *status = (int)EA_ERR_DEVICE_TIMEOUT;
+}
+
+// score = (group reduction of the attention + eps) * ||v|| with the norms already computed; one thread per key.
+__global__ void __launch_bounds__(256)
+weight_kernel(const float* __restrict__ logits, const float* __restrict__ lse, const float* __restrict__ vnorm,
+              int Hq, int Hkv, int n, int group_mode, float epsilon, float* __restrict__ scores) {
+    const int G = Hq / Hkv;
+    const int ug = blockIdx.y;
+    const int u = ug / Hkv, g = ug % Hkv;
+    const int key = blockIdx.x * blockDim.x + threadIdx.x;
+    if (key >= n) return;
+    float a;
+    if (group_mode == EA_GROUP_MEAN_LOGIT) {
+        float x = 0.f;
+        for (int j = 0; j < G; ++j) x += logits[((size_t)u * Hq + (size_t)g * G + j) * n + key];
+        a = expf(x * (1.0f / (float)G) - lse[ug]);
+    } else {
+        a = 0.f;
+        for (int j = 0; j < G; ++j) {
+            const size_t uh = (size_t)u * Hq + (size_t)g * G + j;
+            a += expf(logits[uh * n + key] - lse[uh]);
+        }
+        if (group_mode == EA_GROUP_MEAN_PROB) a *= 1.0f / (float)G;
+    }
+    scores[(size_t)ug * n + key] = (a + epsilon) * vnorm[(size_t)ug * n + key];
+}
+
 // score = group reduction of (a_hat_h + eps) * sqrt(wo_norm2_h) over the query heads of the KV head
 // (Eq. 9 with ||W_o v||); one thread per key.
 __global__ void __launch_bounds__(256)
@@ -217,6 +361,55 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
     return EA_CHECK_LAUNCH();
 }
 
+
+ea_status ea_launch_vnorm(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* v, int n_ctas, float* vnorm,
+                          cudaStream_t st) {
+    const long long n_rows = (long long)s.n_units * s.n_kv_heads * s.n_keys;
+    const int smem = kVnSmem;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_ctas);
+    cfg.blockDim = dim3(kVnThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    // clusters of two keep both SMs of a pair for this kernel, so that the CTA pairs of the log-score
+    // kernel find whole pairs among the others
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = n_ctas % 2 == 0 ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err;
+    switch (s.head_dim) {
+        case 64:
+            EA_CUDA_TRY(cudaFuncSetAttribute(vnorm_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            err = cudaLaunchKernelEx(&cfg, vnorm_stream_kernel<64>, v, n_rows, vnorm, ctx->status_dev);
+            break;
+        case 128:
+            EA_CUDA_TRY(cudaFuncSetAttribute(vnorm_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            err = cudaLaunchKernelEx(&cfg, vnorm_stream_kernel<128>, v, n_rows, vnorm, ctx->status_dev);
+            break;
+        case 256:
+            EA_CUDA_TRY(cudaFuncSetAttribute(vnorm_stream_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            err = cudaLaunchKernelEx(&cfg, vnorm_stream_kernel<256>, v, n_rows, vnorm, ctx->status_dev);
+            break;
+        default:
+            return EA_ERR_UNSUPPORTED;
+    }
+    EA_CUDA_TRY(err);
+    ea_count_launches(ctx, 1);
+    return EA_CHECK_LAUNCH();
+}
+
+ea_status ea_launch_weight(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
+                           const float* vnorm, float epsilon, float* scores, cudaStream_t st) {
+    dim3 grid((unsigned)((s.n_keys + 255) / 256), (unsigned)(s.n_units * s.n_kv_heads));
+    weight_kernel<<<grid, 256, 0, st>>>(logits, lse, vnorm, s.n_q_heads, s.n_kv_heads, s.n_keys, s.group_mode,
+                                        epsilon, scores);
+    ea_count_launches(ctx, 1);
+    return EA_CHECK_LAUNCH();
+}
 
 ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const float* lse_part, int n_chunks,
                                 float* lse, cudaStream_t st) {

@@ -47,18 +47,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Wait for the phase with the given parity to complete.  The wait is bounded: after `limit_ns`
 // (or kWaitPolls polls) it raises *abort_flag and gives up; it also gives up as soon as another
-// thread has raised the flag.  Returns true when the phase completed.
+// thread has raised the flag.  Returns true when the phase completed.  The clock and the flag are
+// looked at once every CHECK polls only: reading %globaltimer costs a good fraction of a
+// microsecond, which a producer that waits before every copy cannot afford per wait.
 constexpr uint64_t kWaitNs = 2000000000ull;
 constexpr uint32_t kWaitPolls = 1u << 28;
+template <uint32_t CHECK = 1024>
 __device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   uint64_t limit_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    uint64_t t0 = 0;
     for (uint32_t it = 1; it < kWaitPolls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0u) {
+        if ((it & (CHECK - 1)) == 0u) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > limit_ns) break;
+            const uint64_t now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
@@ -75,11 +79,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // (the abort flag is already up), and it raises nothing.
 constexpr uint64_t kDrainNs = 20000000ull;
 __device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    uint64_t t0 = 0;
     for (uint32_t it = 1; it < kWaitPolls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0u && globaltimer_ns() - t0 > kDrainNs) break;
+        if ((it & 255u) == 0u) {
+            const uint64_t now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kDrainNs) break;
+        }
     }
     return false;
 }

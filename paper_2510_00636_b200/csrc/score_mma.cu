@@ -684,7 +684,9 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     using G = Geo<D, PAIR>;
     const int Gq = s.n_q_heads / s.n_kv_heads;
     constexpr int keys_per_step = PAIR ? 2 * kTileKeys : kTileKeys;
-    const int workers = PAIR ? ctx->sm_count / 2 : ctx->sm_count;     // CTAs or CTA pairs
+    // CTAs or CTA pairs, one per SM; the SMs of a side pass (ea_set_side_sms) are left to it
+    const int sms = ctx->sm_budget < ctx->sm_count - ctx->side_sms ? ctx->sm_budget : ctx->sm_count - ctx->side_sms;
+    const int workers = PAIR ? sms / 2 : sms;
     MmaParams p;
     p.vec = vec;
     p.image = image;

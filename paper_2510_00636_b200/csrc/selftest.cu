@@ -15,7 +15,7 @@ __global__ void wait_timeout_kernel(unsigned long long limit_ns, int* status) {
     abort_flag = 0;
     ptx::mbar_init(ptx::smem_u32(&bar), 1);
     ptx::fence_mbar_init();
-    const bool ok = ptx::mbar_wait_limited(ptx::smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    const bool ok = ptx::mbar_wait_limited<8>(ptx::smem_u32(&bar), 0u, &abort_flag, limit_ns);
     if (!ok && abort_flag) *status = (int)EA_ERR_DEVICE_TIMEOUT;
 }
 

@@ -356,3 +356,34 @@ def test_host_buffer_entry_point_matches_device_calls(ea, chunk):
     with pytest.raises(ea.EAError) as e:
         ea.ea_compress_host(small, shape, hq, hk, hv, pos, cfg.n_future, cfg.rope_base, cfg.eps, cfg.n_kept, chunk)
     assert e.value.status == 3
+
+
+@pytest.mark.parametrize("cfg_id,side,budget", [(1, 16, 0), (0, 8, 0), (1, 0, 64), (1, 24, 100)])
+def test_side_pass_and_sm_budget_leave_the_result_unchanged(ea, cfg_id, side, budget):
+    """The value-norm pass on SMs of its own (ea_set_side_sms) and a log-score kernel limited to part of
+    the device (ea_set_sm_budget) are scheduling choices: log-scores bitwise equal, scores equal up to the
+    rounding of the norm's square root, same kept set on ties-free data."""
+    cfg = inputs.CONFIGS[cfg_id].tempered(2.0)
+    q, k, v, pos = inputs.generate_layer(cfg, device="cuda")
+    shape = _shape(ea, cfg)
+    ctx = ea.Context.for_shape(shape)
+    mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
+    sc0, lg0 = ea.ea_score(ctx, shape, k, v, mu, sig, cfg.eps, want_logits=True)
+    sc0, lg0 = sc0.clone(), lg0.clone()
+    ctx.set_side_sms(side)
+    ctx.set_sm_budget(budget)
+    for _ in range(2):
+        sc1, lg1 = ea.ea_score(ctx, shape, k, v, mu, sig, cfg.eps, want_logits=True)
+        ctx.sync_status()
+        assert torch.equal(lg0, lg1)
+        torch.testing.assert_close(sc1, sc0, rtol=1e-6, atol=0.0)
+    ctx.set_side_sms(0)
+    ctx.set_sm_budget(0)
+    sc2 = ea.ea_score(ctx, shape, k, v, mu, sig, cfg.eps)
+    ctx.sync_status()
+    assert torch.equal(sc2, sc0)
+    for bad in (3, -2, 1000):
+        with pytest.raises(ea.EAError):
+            ctx.set_side_sms(bad)
+    with pytest.raises(ea.EAError):
+        ctx.set_sm_budget(1)

@@ -511,3 +511,76 @@ def test_oracle_on_tiny_config(oracle):
     assert out["kept_idx"].shape == (1, 2, 256)
     assert np.all(np.isfinite(out["logits"])) and np.all(np.isfinite(out["scores"]))
     assert np.all(np.diff(out["kept_idx"], axis=-1) > 0)
+
+
+# ------------------------------------------------------------------------------------------
+# Streaming driver (oracle/ea_stream.py): plumbing around the pinned functions.
+def _stream_inputs(seed, U=1, Hq=4, Hkv=2, d=64, n0=40, W=16):
+    rng = np.random.default_rng(seed)
+    def bf(x):
+        return (x.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    k0, v0 = bf(rng.normal(size=(U, Hkv, n0, d))), bf(rng.normal(size=(U, Hkv, n0, d)))
+    return rng, bf, k0, v0
+
+
+def test_stream_single_event_is_compress_on_the_concatenated_inputs(oracle):
+    from oracle.ea_stream import StreamOracle
+    rng, bf, k0, v0 = _stream_inputs(1)
+    k1, v1 = bf(rng.normal(size=(1, 2, 24, 64))), bf(rng.normal(size=(1, 2, 24, 64)))
+    q = bf(rng.normal(size=(1, 4, 16, 64)) + 0.3)
+    st = StreamOracle(k0, v0, window=16, budget=32)
+    st.append(k1, v1)
+    st.push_queries(q)
+    got = st.compress([64], 8, 1e4, 0.02)
+    want = oracle.compress(q, np.concatenate([k0, k1], 2), np.concatenate([v0, v1], 2), np.array([64]), 8, 1e4,
+                           0.02, 32)
+    assert np.array_equal(got["kept_idx"], want["kept_idx"])
+    assert np.array_equal(got["scores"], want["scores"])
+    st.keep(got["kept_idx"])
+    assert st.n_keys == 32 and np.array_equal(st.k, want["k_out"]) and np.array_equal(st.v, want["v_out"])
+
+
+def test_stream_window_is_the_tail_of_everything_pushed(oracle):
+    from oracle.ea_stream import StreamOracle
+    rng, bf, k0, v0 = _stream_inputs(2)
+    st = StreamOracle(k0, v0, window=16, budget=1000)
+    pushed = []
+    for m in (5, 7, 3, 20, 1, 40):          # partly filled, exactly full, wrapped several times in one push
+        q = bf(rng.normal(size=(1, 4, m, 64)))
+        pushed.append(q)
+        st.push_queries(q)
+        everything = np.concatenate(pushed, axis=2)
+        assert np.array_equal(st.q, everything[:, :, -16:])
+        assert st.q.shape[2] == min(16, everything.shape[2])
+    # statistics depend on the set of rows only: any rotation of the window gives the same mean and covariance
+    mu, sig = oracle.mean_cov(st.q)
+    mu_r, sig_r = oracle.mean_cov(np.roll(st.q, 5, axis=2))
+    np.testing.assert_allclose(mu, mu_r, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(sig, sig_r, rtol=0, atol=1e-14)
+
+
+def test_stream_events_compose_as_index_maps(oracle):
+    """After two events the cache holds original rows: following the kept indices back through both events
+    names them, and below the budget an event keeps every row."""
+    from oracle.ea_stream import StreamOracle
+    rng, bf, k0, v0 = _stream_inputs(3, n0=20)
+    st = StreamOracle(k0, v0, window=16, budget=48)
+    origin = np.broadcast_to(np.arange(20), (1, 2, 20)).copy()       # which original row sits where
+    all_k = k0
+    for e, n_new in enumerate((12, 30, 30)):
+        k1, v1 = bf(rng.normal(size=(1, 2, n_new, 64))), bf(rng.normal(size=(1, 2, n_new, 64)))
+        st.append(k1, v1)
+        st.push_queries(bf(rng.normal(size=(1, 4, 9, 64)) + 0.1 * e))
+        origin = np.concatenate([origin, np.broadcast_to(np.arange(all_k.shape[2], all_k.shape[2] + n_new),
+                                                         (1, 2, n_new))], axis=2)
+        all_k = np.concatenate([all_k, k1], axis=2)
+        out = st.compress([all_k.shape[2]], 8, 1e4, 0.02)
+        idx = out["kept_idx"]
+        if e == 0:
+            assert st.n_keys == 32 and np.array_equal(idx, np.broadcast_to(np.arange(32), (1, 2, 32)))
+        assert idx.shape[2] == min(st.n_keys, 48)
+        assert (np.diff(idx, axis=2) > 0).all()
+        st.keep(idx)
+        origin = np.take_along_axis(origin, idx.astype(np.int64), axis=2)
+        for g in range(2):
+            assert np.array_equal(st.k[0, g], all_k[0, g][origin[0, g]])

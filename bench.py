@@ -33,10 +33,13 @@ import torch  # noqa: E402
 from paper_2510_00636_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the log-score kernel divided by the
-# key-slots of that launch (ncu --set full, profiles/logits_mma_kernel_*); None = not captured for
-# the current kernel
-# keyed by (head_dim, query heads per KV head): the log-score write and the sharing of key tiles depend on both
+# key-slots of that launch (one ncu --set full capture per shape on a few layers, clocks not locked),
+# keyed by (head_dim, query heads per KV head): the log-score write and the sharing of key tiles depend
+# on both.  NCU_CAPTURE_SOURCE is the fingerprint of the kernel source that was captured.
 NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.1018e9 / 2097152, (128, 4): 293.9e6 / 1048576}
+NCU_CAPTURE_SOURCE = "to-be-recorded"
+# nominal figures of the part, reported beside the measured denominators
+NOMINAL_HBM_GBS, NOMINAL_TFLOPS = 8000.0, 2250.0
 
 METRIC = "kv_keys_scored_and_compacted_per_second"
 UNIT = "Gkeys/s"
@@ -169,6 +172,16 @@ class Workload:
                                    cfg.window)
         return self.ea.Context.for_shape(shape, self.device.index)
 
+    def release_outputs(self):
+        """Drop the output tensors (the host-buffer leg only needs a few input layers)."""
+        for name in ("mu", "sigma", "scores", "k_out", "v_out", "head_off"):
+            setattr(self, name, None)
+
+    def release_all(self):
+        for name in list(vars(self)):
+            if isinstance(getattr(self, name), (torch.Tensor, list, dict)):
+                setattr(self, name, None)
+
     def step(self, ctx, units_per_call):
         """One pass of the whole path over every unit, `units_per_call` units per library call."""
         ea, cfg = self.ea, self.cfg
@@ -204,83 +217,99 @@ class Workload:
 
 
 class DecodeWorkload:
-    """The streaming-decode config: one step replays the 28 compression events of a generation that
-    grows every sequence's cache from 2048 to 16384 keys in steps of 512 with a 4096-key budget
-    (inputs.decode_schedule).  Every distinct cache length has its own resident synthetic cache (all
-    28 layers x batch 8 folded into the units of one call); the window queries rotate through
-    `n_phases` slowly turning query means."""
+    """The streaming-decode config on ONE carried cache: one step replays the 28 compression events of a
+    generation that grows every sequence's cache from 2048 to 16384 keys in steps of 512 with a 4096-key
+    budget (inputs.decode_schedule).  All 28 layers x batch 8 are the units of one call.  Every event
+    appends 512 new pairs behind the kept ones in the fixed buffer (ea_cache_append), pushes the window's
+    worth of new queries into the ring (ea_window_push), takes the ring's statistics, scores the cache and
+    compacts it in place to the budget.  The new tokens rotate through `n_phases` pre-generated draws with
+    slowly turning query means; a step starts from 2048 valid rows of whatever the buffer holds (rows kept
+    by the previous step: synthetic rows of the same distribution)."""
 
     def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False):
         import dataclasses
         self.cfg, self.device, self.ea = cfg, device, ea
         self.use_graph, self.graphs = use_graph, {}
         self.events = inputs.decode_schedule()
+        self.every = self.events[0][1] - 2048
+        self.cap = max(n for _, n, _ in self.events)
         L, B = cfg.n_layers, cfg.batch
         U, Hq, Hkv, d, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
         bf, f32 = torch.bfloat16, torch.float32
         self.n_units = U
-        self.caches, self.windows = {}, []
-        for n in sorted({n for _, n, _ in self.events}):
-            k = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
-            v = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
-            for layer in range(L):
-                _, kk, vv, _ = inputs.generate_layer(dataclasses.replace(cfg, window=1), layer=layer, device=device,
-                                                     n_keys=n)
-                k[layer * B:(layer + 1) * B], v[layer * B:(layer + 1) * B] = kk, vv
-            kept = min(n, cfg.n_kept)
-            self.caches[n] = dict(
-                k=k, v=v, scores=torch.empty((U, Hkv, n), dtype=f32, device=device),
-                idx=torch.empty((U, Hkv, kept), dtype=torch.int32, device=device),
-                k_out=torch.empty((U, Hkv, kept, d), dtype=bf, device=device),
-                v_out=torch.empty((U, Hkv, kept, d), dtype=bf, device=device))
+        self.k = torch.empty((U, Hkv, self.cap, d), dtype=bf, device=device)
+        self.v = torch.empty((U, Hkv, self.cap, d), dtype=bf, device=device)
+        for layer in range(L):
+            _, kk, vv, _ = inputs.generate_layer(dataclasses.replace(cfg, window=1), layer=layer, device=device,
+                                                 n_keys=self.cap, draw=1)
+            self.k[layer * B:(layer + 1) * B], self.v[layer * B:(layer + 1) * B] = kk, vv
+        self.new_k, self.new_v, self.new_q = [], [], []
         for ph in range(n_phases):
-            q = torch.empty((U, Hq, W, d), dtype=bf, device=device)
+            nk = torch.empty((U, Hkv, self.every, d), dtype=bf, device=device)
+            nv = torch.empty_like(nk)
+            nq = torch.empty((U, Hq, W, d), dtype=bf, device=device)
+            pos = 2048 + ph * self.every
             for layer in range(L):
-                qq, _, _, _ = inputs.generate_layer(cfg, layer=layer, device=device, n_keys=1,
-                                                    q_phase=2 * 3.141592653589793 / 64 * ph)
-                q[layer * B:(layer + 1) * B] = qq
-            self.windows.append(q)
+                qq, kk, vv, _ = inputs.generate_layer(cfg, layer=layer, device=device, n_keys=self.every, draw=2 + ph,
+                                                      key_positions=torch.arange(pos, pos + self.every),
+                                                      q_phase=2 * 3.141592653589793 / 64 * ph)
+                sl = slice(layer * B, (layer + 1) * B)
+                nk[sl], nv[sl], nq[sl] = kk, vv, qq
+            self.new_k.append(nk), self.new_v.append(nv), self.new_q.append(nq)
+        self.ring = torch.zeros((U, Hq, W, d), dtype=bf, device=device)
+        self.pushed = torch.zeros((U,), dtype=torch.int64, device=device)
         self.pos = [torch.full((U,), pos, dtype=torch.int64, device=device) for pos, _, _ in self.events]
         self.mu = torch.empty((U, Hq, d), dtype=f32, device=device)
         self.sigma = torch.empty((U, Hq, d, d), dtype=f32, device=device)
-        # for the caller: the largest shape decides the workspace
-        self.k = self.caches[max(self.caches)]["k"]
+        self.scores = torch.empty((U, Hkv, self.cap), dtype=f32, device=device)
+        self.idx = torch.empty((U, Hkv, cfg.n_kept), dtype=torch.int32, device=device)
+
+    def _shape(self, n):
+        cfg = self.cfg
+        return self.ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, n, cfg.window,
+                                  kv_capacity=self.cap)
 
     def make_ctx(self, units_per_call):
-        cfg = self.cfg
-        shape = self.ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, max(self.caches),
-                                   cfg.window)
-        return self.ea.Context.for_shape(shape, self.device.index)
+        return self.ea.Context.for_shape(self._shape(self.cap), self.device.index)
 
-    def _event(self, ctx, n, kept, window, pos):
+    def _event(self, ctx, n, kept, ph, pos):
         ea, cfg = self.ea, self.cfg
-        c = self.caches[n]
-        shape = ea.make_shape(self.n_units, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, n, cfg.window)
-        ea.ea_query_stats(ctx, shape, window, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
-        ea.ea_score(ctx, shape, c["k"], c["v"], self.mu, self.sigma, cfg.eps, c["scores"])
-        ea.ea_select_compact(ctx, shape, c["scores"], kept, c["k"], c["v"], c["idx"], c["k_out"], c["v_out"])
+        shape = self._shape(n)
+        scores = self.scores.view(-1)[:self.n_units * cfg.n_kv_heads * n].view(self.n_units, cfg.n_kv_heads, n)
+        idx = self.idx.view(-1)[:self.n_units * cfg.n_kv_heads * kept].view(self.n_units, cfg.n_kv_heads, kept)
+        ea.ea_cache_append(ctx, self._shape(n - self.every), self.k, self.v, self.new_k[ph], self.new_v[ph])
+        ea.ea_window_push(ctx, shape, self.ring, self.pushed, self.new_q[ph])
+        ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
+        ea.ea_score(ctx, shape, self.k, self.v, self.mu, self.sigma, cfg.eps, scores)
+        ea.ea_select_compact_inplace(ctx, shape, scores, kept, self.k, self.v, idx)
 
     def step(self, ctx, units_per_call):
         for e, (pos, n, kept) in enumerate(self.events):
-            window = self.windows[e % len(self.windows)]
+            ph = e % len(self.new_q)
             if not self.use_graph:
-                self._event(ctx, n, kept, window, self.pos[e])
+                self._event(ctx, n, kept, ph, self.pos[e])
                 continue
-            # one CUDA graph per distinct event (cache length, window buffer); the position is read from a
+            # one CUDA graph per distinct event (cache length, new-token buffers); the position is read from a
             # device buffer that is refreshed before each replay
-            key = (n, e % len(self.windows))
+            key = (n, ph)
             if key not in self.graphs:
                 pos_buf = self.pos[e].clone()
-                self._event(ctx, n, kept, window, pos_buf)          # warm-up outside the capture
+                self._event(ctx, n, kept, ph, pos_buf)          # warm-up outside the capture
                 torch.cuda.synchronize()
                 gc.collect()          # no library context may be destroyed (cudaFree) while the capture is open
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
-                    self._event(ctx, n, kept, window, pos_buf)
+                    self._event(ctx, n, kept, ph, pos_buf)
                 self.graphs[key] = (g, pos_buf)
             g, pos_buf = self.graphs[key]
             pos_buf.copy_(self.pos[e], non_blocking=True)
             g.replay()
+
+    def release_all(self):
+        self.graphs = {}
+        for name in list(vars(self)):
+            if isinstance(getattr(self, name), (torch.Tensor, list, dict)) and name != "events":
+                setattr(self, name, None)
 
     def work(self):
         cfg = self.cfg
@@ -389,6 +418,111 @@ def run_reference(args, cfg):
     }))
 
 
+def source_fingerprint():
+    """Hash of the log-score kernel's source: the DRAM-traffic figure of a capture only describes that source."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2510_00636_b200", "csrc", "score_mma.cu")
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_workload, free_first=None):
+    """Builds the workload of `cfg` in HBM, times `steps` steps after `warmup`, returns the figures of the line."""
+    if free_first is not None:
+        free_first.release_all()
+        free_first = None
+        gc.collect()
+        torch.cuda.empty_cache()
+    decode = cfg.cfg_id == 4
+    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph) if decode else Workload(cfg, device, ea, args.head_adaptive,
+                                                                 args.hidden_stats, args.with_wo)
+    upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
+    ctx = wl.make_ctx(upc)
+    if args.side_sms:
+        ctx.set_side_sms(args.side_sms)
+    slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg)
+    if args.with_wo:
+        alg_flops *= 2                 # v^T (W_o^T W_o) v per query head is a second quadratic form
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(warmup):
+        wl.step(ctx, upc)
+    ctx.sync_status()
+
+    barrier(world)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ctx.profile_begin()
+    t_host0 = time.time()
+    ev0.record()
+    for _ in range(steps):
+        wl.step(ctx, upc)
+    ev1.record()
+    score_ms, score_launches, total_launches = ctx.profile_end()
+    torch.cuda.synchronize()
+    t_host1 = time.time()
+    barrier(world)
+    clocks = sampler.stop(t_host0, t_host1)
+    ms_local = ev0.elapsed_time(ev1) / steps
+    ms = max_over_ranks(ms_local, world, device)
+    ctx.sync_status()
+    if decode and args.graph:
+        # replays do not pass through the library's launch counter or its kernel events: take both from one
+        # untimed step of the same launches made directly (every timed step replayed exactly these)
+        wl.use_graph = False
+        ctx.profile_begin()
+        wl.step(ctx, upc)
+        score_ms, score_launches, total_launches = ctx.profile_end()
+        total_launches *= steps
+        wl.use_graph = True
+
+    # roofline of the dominant kernel (the log-score kernel, Eq. 7)
+    n_calls = len(wl.events) if decode else (wl.n_units + upc - 1) // upc
+    avg_score_ms = score_ms / max(1, score_launches)
+    # (with --with-wo the kernel runs twice per call, once per quadratic form, each with the FLOPs of Eq. 7)
+    flops_per_launch = alg_flops / (2 if args.with_wo else 1) / n_calls
+    bytes_per_launch = slots * 2 * cfg.head_dim / n_calls            # the K rows this kernel must read
+    t_tensor = flops_per_launch / (peaks["tflops"] * 1e12)
+    t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        achieved = flops_per_launch / (avg_score_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["tflops"], "frac_nominal": achieved / NOMINAL_TFLOPS}
+    else:
+        achieved = bytes_per_launch / (avg_score_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "frac_nominal": achieved / NOMINAL_HBM_GBS}
+    # DRAM bytes per launch from an ncu capture of this kernel on a few layers of the same shapes, scaled by
+    # the key-slots of a launch (traffic is proportional to them); null when the kernel's source is no
+    # longer the one that was captured
+    captured = NCU_DRAM_BYTES_PER_KEY_SLOT.get((cfg.head_dim, cfg.group))
+    fresh = captured is not None and NCU_CAPTURE_SOURCE == source_fingerprint()
+    traffic = captured * slots / n_calls if fresh else None
+    sm_mhz = clocks.get("sm_mhz")
+    roofline.update({"traffic": traffic, "kernel": "log-score kernel (k.mu/sqrt(d) + k'Sigma k/2d), kernel-only figure",
+                     "kernel_ms": avg_score_ms, "launches_timed": score_launches,
+                     # device time x median SM clock of the timed region: compares runs at different power-capped clocks
+                     "kernel_mcycles": avg_score_ms * sm_mhz / 1e3 if sm_mhz else None,
+                     "peak_source": peaks["source"] + " (sustained bf16 matmul)"})
+    # whole-path roofline: the slower of the K.Sigma FLOPs at tensor peak and the K/V bytes at HBM bandwidth
+    t_path = max(alg_flops / (peaks["tflops"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9))
+    t_path_nominal = max(alg_flops / (NOMINAL_TFLOPS * 1e12), alg_bytes / (NOMINAL_HBM_GBS * 1e9))
+    out = {"ms": ms, "slots": slots, "units_per_call": upc, "roofline": roofline, "clocks": clocks,
+           "gpu_launches": int(total_launches),
+           "path_roofline": {"t_roof_ms": t_path * 1e3, "frac": t_path / (ms * 1e-3), "t_roof_nominal_ms": t_path_nominal * 1e3,
+                             "frac_nominal": t_path_nominal / (ms * 1e-3), "step_mcycles": ms * sm_mhz / 1e3 if sm_mhz else None,
+                             "alg_bytes": alg_bytes, "alg_flops": alg_flops, "peak_source": peaks["source"],
+                             "nominal": "%.0f GB/s, %.0f TFLOP/s dense bf16" % (NOMINAL_HBM_GBS, NOMINAL_TFLOPS)},
+           "workload": wl if keep_workload else None}
+    if not keep_workload:
+        wl.release_all()
+        del wl, ctx
+        gc.collect()
+        torch.cuda.empty_cache()
+    return out
+
+
 # ------------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -409,6 +543,10 @@ def main():
                     help="prefill configs: weight by ||W_o v|| (ea_score_wo) with an output projection of this width")
     ap.add_argument("--graph", action="store_true",
                     help="decode config: replay each compression event as a captured CUDA graph")
+    ap.add_argument("--side-sms", type=int, default=0,
+                    help="run the value-norm pass on this many SMs beside the log-score kernel (ea_set_side_sms)")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="default run: skip the device-resident figures of the 32k and the decode workloads")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -432,82 +570,14 @@ def main():
     from paper_2510_00636_b200 import binding as ea
     ea.lib()
 
-    decode = cfg.cfg_id == 4
     variant = args.head_adaptive is not None or args.hidden_stats or args.with_wo
-    if variant and decode:
+    if variant and cfg.cfg_id == 4:
         raise SystemExit("--head-adaptive, --hidden-stats and --with-wo apply to the prefill configs")
-    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph) if decode else Workload(cfg, device, ea, args.head_adaptive,
-                                                                 args.hidden_stats, args.with_wo)
-    upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
-    ctx = wl.make_ctx(upc)
-    slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg)
-    if variant:
-        args.skip_e2e = True           # the host-buffer entry point runs the three basic calls
-    if args.with_wo:
-        alg_flops *= 2                 # v^T (W_o^T W_o) v per query head is a second quadratic form
-    if decode:
-        args.skip_e2e = True           # the host-buffer leg is defined for the prefill configs
+    if variant or cfg.cfg_id == 4:
+        args.skip_e2e = True           # the host-buffer entry point runs the three basic calls on a prefill cache
     peaks = measured_peaks()
-
-    sampler = ClockSampler(local)
-    sampler.start()
-    for _ in range(args.warmup):
-        wl.step(ctx, upc)
-    ctx.sync_status()
-
-    barrier(world)
-    torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ctx.profile_begin()
-    t_host0 = time.time()
-    ev0.record()
-    for _ in range(args.steps):
-        wl.step(ctx, upc)
-    ev1.record()
-    score_ms, score_launches, total_launches = ctx.profile_end()
-    torch.cuda.synchronize()
-    t_host1 = time.time()
-    barrier(world)
-    clocks = sampler.stop(t_host0, t_host1)
-    ms_local = ev0.elapsed_time(ev1) / args.steps
-    ms = max_over_ranks(ms_local, world, device)
-    ctx.sync_status()
-    if decode and args.graph:
-        # replays do not pass through the library's launch counter or its kernel events: take both from one
-        # untimed step of the same launches made directly (every timed step replayed exactly these)
-        wl.use_graph = False
-        ctx.profile_begin()
-        wl.step(ctx, upc)
-        score_ms, score_launches, total_launches = ctx.profile_end()
-        total_launches *= args.steps
-        wl.use_graph = True
-
-    # roofline of the dominant kernel (the log-score kernel, Eq. 7)
-    n_calls = len(wl.events) if decode else (wl.n_units + upc - 1) // upc
-    avg_score_ms = score_ms / max(1, score_launches)
-    # (with --with-wo the kernel runs twice per call, once per quadratic form, each with the FLOPs of Eq. 7)
-    flops_per_launch = alg_flops / (2 if args.with_wo else 1) / n_calls
-    bytes_per_launch = slots * 2 * cfg.head_dim / n_calls            # the K rows this kernel must read
-    t_tensor = flops_per_launch / (peaks["tflops"] * 1e12)
-    t_hbm = bytes_per_launch / (peaks["hbm_gbs"] * 1e9)
-    if t_tensor >= t_hbm:
-        achieved = flops_per_launch / (avg_score_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["tflops"]}
-    else:
-        achieved = bytes_per_launch / (avg_score_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"]}
-    # DRAM bytes per launch from the ncu capture of this kernel (profiles/): measured on a 2-layer
-    # case of the same shapes and scaled by the key-slots of a launch (traffic is proportional to them)
-    traffic_per_slot = NCU_DRAM_BYTES_PER_KEY_SLOT.get((cfg.head_dim, cfg.group))
-    traffic = None if traffic_per_slot is None else traffic_per_slot * slots / n_calls
-    roofline.update({"traffic": traffic, "kernel": "log-score kernel (k.mu/sqrt(d) + k'Sigma k/2d)",
-                     "kernel_ms": avg_score_ms, "launches_timed": score_launches,
-                     "peak_source": peaks["source"] + " (sustained bf16 matmul)"})
-    # whole-path roofline: the slower of the K.Sigma FLOPs at tensor peak and the K/V bytes at HBM bandwidth
-    t_path = max(alg_flops / (peaks["tflops"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9))
-    path_frac = t_path / (ms * 1e-3)
+    m = measure(args, cfg, ea, device, world, local, peaks, args.steps, args.warmup, keep_workload=True)
+    wl, slots, ms = m.pop("workload"), m["slots"], m["ms"]
 
     result = {
         "metric": METRIC, "value": world * slots / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
@@ -521,19 +591,37 @@ def main():
                    "statistics": "window queries given" if not args.hidden_stats else
                                  "hidden states through W_Q, d_model %d" % args.hidden_stats,
                    "value_weight": "||v||" if not args.with_wo else "||W_o v||, d_model %d" % args.with_wo,
-                   "cuda_graph": bool(decode and args.graph), "key_slots_per_step": slots, "units_per_call": upc, "parallelism": f"replicas x{world}",
+                   "cuda_graph": bool(cfg.cfg_id == 4 and args.graph), "key_slots_per_step": slots,
+                   "units_per_call": m["units_per_call"], "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (K+V %.1f GB per step)" % (slots * 4 * cfg.head_dim / 1e9)},
         "ms_per_128k_compression": ms if cfg.cfg_id == 3 else None,
-        "path_roofline": {"t_roof_ms": t_path * 1e3, "frac": path_frac, "alg_bytes": alg_bytes,
-                          "alg_flops": alg_flops, "peak_source": peaks["source"]},
-        "roofline": roofline,
-        "gpu_launches": int(total_launches),
-        "clocks": clocks,
+        "path_roofline": m["path_roofline"],
+        "roofline": m["roofline"],
+        "gpu_launches": m["gpu_launches"],
+        "clocks": m["clocks"],
     }
+    if cfg.cfg_id == 4:
+        result["config"]["cache"] = "one carried buffer per sequence, compacted in place, 512 pairs appended per event"
 
     # end to end from host buffers through ea_compress_host (rank-local; max over ranks)
     if not args.skip_e2e:
         result["e2e"] = run_e2e(args, cfg, wl, ea, device, world, slots)
+
+    # the other full-size workloads, device-resident only, in the same line (the headline stays the 128k config)
+    if args.other_configs and cfg.cfg_id == 3 and not args.layers and not variant and world == 1:
+        others = {}
+        for other_id in (2, 4):
+            ocfg = inputs.CONFIGS[other_id]
+            om = measure(args, ocfg, ea, device, world, local, peaks, max(5, args.steps // 2), 3, keep_workload=False,
+                         free_first=wl)
+            wl = None
+            others[ocfg.name] = {"ms_per_step": om["ms"], "value": om["slots"] / (om["ms"] * 1e-3) / 1e9, "unit": UNIT,
+                                 "path_roofline_frac": om["path_roofline"]["frac"],
+                                 "path_roofline_frac_nominal": om["path_roofline"]["frac_nominal"],
+                                 "kernel_frac": om["roofline"]["frac"], "kernel_ms": om["roofline"]["kernel_ms"],
+                                 "kernel_mcycles": om["roofline"]["kernel_mcycles"], "sm_mhz": om["clocks"]["sm_mhz"],
+                                 "gpu_launches": om["gpu_launches"]}
+        result["other_configs"] = others
 
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
         n_sample = oracle_sample(cfg)

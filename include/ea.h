@@ -79,6 +79,12 @@ typedef struct ea_shape {
     int32_t rope_layout; /* EA_ROPE_*                                                  */
     int32_t group_mode;  /* EA_GROUP_*                                                 */
     int32_t cov_norm;    /* EA_COV_*                                                   */
+    int32_t kv_capacity; /* rows per KV head in the K/V BUFFERS when the cache lives in a
+                            larger, fixed buffer (streaming decode): head g of unit u starts
+                            at row (u * Hkv + g) * kv_capacity and its first n_keys rows are
+                            the cache.  0 = dense (kv_capacity = n_keys).  Must be 0 or
+                            >= n_keys.  Scores, log-scores and kept indices stay dense in
+                            n_keys; gathered outputs (k_out, v_out) are dense in n_kept.   */
 } ea_shape;
 
 typedef struct ea_ctx ea_ctx;   /* opaque; owns its workspace and a status word */
@@ -280,8 +286,8 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
  * length becomes n_kept; new pairs are appended from there).  kept_idx still
  * refers to the positions before the call.
  *
- * k, v      bf16 [n_units, Hkv, n, d], 16-byte aligned, modified in place;
- *           two distinct buffers
+ * k, v      bf16 [n_units, Hkv, n, d] (rows per head: kv_capacity if set), 16-byte
+ *           aligned, modified in place; two distinct buffers
  * kept_idx  int32 [n_units, Hkv, n_kept]  (output)
  * The call records only stream work and no allocation, so a sequence of
  * ea_query_stats / ea_score / ea_select_compact_inplace can be captured into
@@ -290,6 +296,49 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
 ea_status ea_select_compact_inplace(ea_ctx* ctx, const ea_shape* shape, const float* scores,
                                     int32_t n_kept, void* k, void* v, int32_t* kept_idx,
                                     void* cuda_stream);
+
+/*
+ * Streaming decode: one cache buffer and one window buffer carried through
+ * consecutive compression events (the decoding set-up of the "Implementation
+ * details" paragraph: a buffer of the most recent 128 states, compression
+ * every 512 generated tokens down to a fixed budget).
+ *
+ * The cache of a head lives in a fixed range of kv_capacity rows (see
+ * ea_shape) of which the first n_keys are valid.  One event is
+ *   ea_cache_append            n_keys -> n_keys + n_new rows per head
+ *   ea_window_push             the queries generated since the last event
+ *   ea_query_stats_ring        statistics of what the window ring holds
+ *   ea_score                   on the shape with the new n_keys
+ *   ea_select_compact_inplace  back to the budget, kept rows moved to the front
+ * after which the caller's n_keys is n_kept.  All five only enqueue stream
+ * work on device-resident state, so an event of a given shape can be captured
+ * into a CUDA graph once and replayed.
+ *
+ * ea_cache_append
+ *   k, v          bf16 [n_units, Hkv, kv_capacity, d], modified in place: rows
+ *                 n_keys .. n_keys + n_new - 1 of every head receive the new pairs
+ *   k_new, v_new  bf16 [n_units, Hkv, n_new, d] (K POST-RoPE at its absolute position)
+ *   n_keys + n_new <= kv_capacity, else EA_ERR_INVALID_ARG
+ * ea_window_push
+ *   q_ring        bf16 [n_units, Hq, W, d], W = shape->window: a ring per query head
+ *   ring_pushed   int64 [n_units] DEVICE: rows pushed so far per unit (start at 0);
+ *                 row j of this call goes to ring row (ring_pushed + j) mod W, then
+ *                 the counters advance by n_new.  The window is the last
+ *                 min(ring_pushed, W) rows pushed.
+ *   q_new         bf16 [n_units, Hq, n_new, d] PRE-RoPE queries, oldest first
+ * ea_query_stats_ring
+ *   ea_query_stats over the rows the ring holds: min(ring_pushed[u], W) of them
+ *   (a partly filled ring is read by its first rows, a wrapped one as it lies:
+ *   mean and covariance do not depend on the order).  A unit with fewer than
+ *   one row (two for EA_COV_SAMPLE) gets mu_bar = 0, sigma_bar = 0.
+ */
+ea_status ea_cache_append(ea_ctx* ctx, const ea_shape* shape, void* k, void* v, const void* k_new,
+                          const void* v_new, int32_t n_new, void* cuda_stream);
+ea_status ea_window_push(ea_ctx* ctx, const ea_shape* shape, void* q_ring, int64_t* ring_pushed,
+                         const void* q_new, int32_t n_new, void* cuda_stream);
+ea_status ea_query_stats_ring(ea_ctx* ctx, const ea_shape* shape, const void* q_ring,
+                              const int64_t* ring_pushed, const int64_t* pos_next, int32_t n_future,
+                              double rope_base, float* mu_bar, float* sigma_bar, void* cuda_stream);
 
 /*
  * Head-adaptive eviction and compaction (the "Head-Adaptive Compression"

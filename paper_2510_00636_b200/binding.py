@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_cache_append", "ea_window_push", "ea_query_stats_ring",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -41,7 +41,7 @@ class EAError(RuntimeError):
 class Shape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_units", "n_q_heads", "n_kv_heads", "head_dim", "n_keys", "window", "rope_layout",
-        "group_mode", "cov_norm")]
+        "group_mode", "cov_norm", "kv_capacity")]
 
 
 _lib = None
@@ -85,6 +85,11 @@ def lib() -> ctypes.CDLL:
         L.ea_select_compact_inplace.restype = ctypes.c_int
         L.ea_selftest_wait_timeout.argtypes = [vp, i32, vp]
         L.ea_selftest_wait_timeout.restype = ctypes.c_int
+        L.ea_cache_append.argtypes = [vp, sp, vp, vp, vp, vp, i32, vp]
+        L.ea_window_push.argtypes = [vp, sp, vp, vp, vp, i32, vp]
+        L.ea_query_stats_ring.argtypes = [vp, sp, vp, vp, vp, i32, f64, vp, vp, vp]
+        for name in ("ea_cache_append", "ea_window_push", "ea_query_stats_ring"):
+            getattr(L, name).restype = ctypes.c_int
         L.ea_set_sm_budget.argtypes = [vp, i32]
         L.ea_set_side_sms.argtypes = [vp, i32]
         L.ea_set_side_sms.restype = ctypes.c_int
@@ -122,9 +127,9 @@ def ea_workspace_bytes(shape: Shape) -> int:
 
 
 def make_shape(n_units, n_q_heads, n_kv_heads, head_dim, n_keys, window, rope_layout=ROPE_HALF_SPLIT,
-               group_mode=GROUP_MEAN_PROB, cov_norm=COV_POPULATION) -> Shape:
+               group_mode=GROUP_MEAN_PROB, cov_norm=COV_POPULATION, kv_capacity=0) -> Shape:
     return Shape(n_units, n_q_heads, n_kv_heads, head_dim, n_keys, window, rope_layout, group_mode,
-                 cov_norm)
+                 cov_norm, kv_capacity)
 
 
 def _ptr(t):
@@ -212,6 +217,41 @@ def ea_query_stats(ctx: Context, shape: Shape, q_win, pos_next, n_future: int, r
     _check(lib().ea_query_stats(ctx._h, ctypes.byref(shape), _ptr(q_win), _ptr(pos_next), int(n_future),
                                 float(rope_base), _ptr(mu_bar), _ptr(sigma_bar), _stream(ctx.device)),
            "ea_query_stats")
+    return mu_bar, sigma_bar
+
+
+def ea_cache_append(ctx: Context, shape: Shape, k, v, k_new, v_new):
+    """Append ``k_new, v_new`` [U,Hkv,n_new,d] behind the ``shape.n_keys`` rows each head holds in ``k, v``
+    [U,Hkv,kv_capacity,d] (in place)."""
+    for t, name in ((k, "k"), (v, "v"), (k_new, "k_new"), (v_new, "v_new")):
+        _dev_tensor(t, torch.bfloat16, name)
+    _check(lib().ea_cache_append(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(k_new), _ptr(v_new),
+                                 int(k_new.shape[2]), _stream(ctx.device)), "ea_cache_append")
+
+
+def ea_window_push(ctx: Context, shape: Shape, q_ring, ring_pushed, q_new):
+    """Push ``q_new`` [U,Hq,n_new,d] into the ring ``q_ring`` [U,Hq,W,d]; ``ring_pushed`` int64 [U] (device) counts."""
+    _dev_tensor(q_ring, torch.bfloat16, "q_ring")
+    _dev_tensor(q_new, torch.bfloat16, "q_new")
+    _dev_tensor(ring_pushed, torch.int64, "ring_pushed")
+    _check(lib().ea_window_push(ctx._h, ctypes.byref(shape), _ptr(q_ring), _ptr(ring_pushed), _ptr(q_new),
+                                int(q_new.shape[2]), _stream(ctx.device)), "ea_window_push")
+
+
+def ea_query_stats_ring(ctx: Context, shape: Shape, q_ring, ring_pushed, pos_next, n_future: int, rope_base: float,
+                        mu_bar=None, sigma_bar=None):
+    """``ea_query_stats`` over the rows a window ring holds -> (mu_bar, sigma_bar)."""
+    _dev_tensor(q_ring, torch.bfloat16, "q_ring")
+    _dev_tensor(ring_pushed, torch.int64, "ring_pushed")
+    _dev_tensor(pos_next, torch.int64, "pos_next")
+    U, Hq, d = shape.n_units, shape.n_q_heads, shape.head_dim
+    if mu_bar is None:
+        mu_bar = torch.empty((U, Hq, d), dtype=torch.float32, device=q_ring.device)
+    if sigma_bar is None:
+        sigma_bar = torch.empty((U, Hq, d, d), dtype=torch.float32, device=q_ring.device)
+    _check(lib().ea_query_stats_ring(ctx._h, ctypes.byref(shape), _ptr(q_ring), _ptr(ring_pushed), _ptr(pos_next),
+                                     int(n_future), float(rope_base), _ptr(mu_bar), _ptr(sigma_bar),
+                                     _stream(ctx.device)), "ea_query_stats_ring")
     return mu_bar, sigma_bar
 
 

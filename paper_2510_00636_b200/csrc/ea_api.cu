@@ -20,6 +20,7 @@ ea_status check_shape(const ea_shape* s) {
     if (s->group_mode < EA_GROUP_MEAN_PROB || s->group_mode > EA_GROUP_MEAN_LOGIT)
         return EA_ERR_INVALID_ARG;
     if (s->cov_norm != EA_COV_POPULATION && s->cov_norm != EA_COV_SAMPLE) return EA_ERR_INVALID_ARG;
+    if (s->kv_capacity != 0 && s->kv_capacity < s->n_keys) return EA_ERR_INVALID_ARG;
     if (s->head_dim != 64 && s->head_dim != 128 && s->head_dim != 256) return EA_ERR_UNSUPPORTED;
     // several kernels put one (unit, head) per gridDim.y entry
     if ((long long)s->n_units * s->n_q_heads > 65535LL) return EA_ERR_UNSUPPORTED;
@@ -263,7 +264,7 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
         float* vnorm = reinterpret_cast<float*>(ws + plan.vnorm);
         int n_chunks = 0;
-        const bool side = ctx->side_sms > 0;
+        const bool side = ctx->side_sms > 0 && ea_kv_cap(*shape) == shape->n_keys;   // the side pass streams a dense V
         if (side) {
             // the value norms do not depend on the log-scores: their pass over V goes to a few SMs of its
             // own, on a second stream, and is launched first so that it is resident when the log-score
@@ -375,7 +376,7 @@ ea_status ea_select_compact(ea_ctx* ctx, const ea_shape* shape, const float* sco
     if (!aligned16(scores) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
         return EA_ERR_INVALID_ARG;
     if (do_gather) {
-        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys *
+        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) *
                                 shape->head_dim * sizeof(__nv_bfloat16);
         const size_t out_bytes = (size_t)shape->n_units * shape->n_kv_heads * n_kept *
                                  shape->head_dim * sizeof(__nv_bfloat16);
@@ -408,7 +409,7 @@ ea_status ea_select_compact_inplace(ea_ctx* ctx, const ea_shape* shape, const fl
     if (!scores || !kept_idx || !k || !v) return EA_ERR_INVALID_ARG;
     if (!aligned16(scores) || !aligned16(k) || !aligned16(v)) return EA_ERR_INVALID_ARG;
     {
-        const size_t bytes = (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys * shape->head_dim *
+        const size_t bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) * shape->head_dim *
                              sizeof(__nv_bfloat16);
         const char* a = static_cast<const char*>(k);
         const char* b = static_cast<const char*>(v);
@@ -443,7 +444,7 @@ ea_status ea_select_compact_adaptive(ea_ctx* ctx, const ea_shape* shape, const f
     if (!aligned16(scores) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
         return EA_ERR_INVALID_ARG;
     if (do_gather) {
-        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys *
+        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) *
                                 shape->head_dim * sizeof(__nv_bfloat16);
         const size_t out_bytes = (size_t)shape->n_units * shape->n_kv_heads * n_kept *
                                  shape->head_dim * sizeof(__nv_bfloat16);

@@ -71,6 +71,7 @@ ea_status ea_compress_host(ea_ctx* ctx, const ea_shape* shape, const void* q_win
     if (shape->n_units == 0) return EA_OK;
     if (!q_win || !k || !v || !pos_next || !kept_idx || !k_out || !v_out) return EA_ERR_INVALID_ARG;
     if (shape->n_keys < 1 || shape->window < 1 || n_future < 1) return EA_ERR_INVALID_ARG;
+    if (shape->kv_capacity != 0 && shape->kv_capacity != shape->n_keys) return EA_ERR_UNSUPPORTED;   // host arrays are dense
     if (ctx->workspace_bytes < need) return EA_ERR_WORKSPACE;
 
     int prev = 0;

@@ -83,11 +83,18 @@ static inline ea_status ea_check_launch(const char* file, int line) {
     } while (0)
 
 static inline size_t ea_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// Rows per KV head in the K/V buffers (the cache is the first n_keys of them).
+static inline int ea_kv_cap(const ea_shape& s) { return s.kv_capacity > 0 ? s.kv_capacity : s.n_keys; }
 
 // ---- launchers (each returns EA_OK or EA_ERR_CUDA from cudaGetLastError) ----
 ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
                           const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
                           float* mu_bar, float* sigma_bar, cudaStream_t st);
+
+// The same statistics over a ring of window rows: pushed[u] rows written so far, at most s.window of them valid.
+ea_status ea_launch_stats_ring(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_ring,
+                               const int64_t* pushed, const int64_t* pos_next, int n_future, double rope_base,
+                               float* rope_coef, float* mu_bar, float* sigma_bar, cudaStream_t st);
 
 // What the log-score kernels evaluate per (query head h, row x of the KV head it reads):
 //   lin_scale * lin_h . x + quad_scale * x^T quad_h x

@@ -66,7 +66,7 @@ constexpr int kFinThreads = 256;
 template <int D>
 __global__ void __launch_bounds__(kFinThreads)
 finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
-                const __nv_bfloat16* __restrict__ v, int Hq, int Hkv, int n, int group_mode,
+                const __nv_bfloat16* __restrict__ v, int Hq, int Hkv, int n, int cap, int group_mode,
                 float epsilon, float* __restrict__ scores) {
     constexpr int LPR = D / 8;          // lanes per value row (one uint4 = 8 bf16 each)
     constexpr int RPS = 32 / LPR;       // rows per load step
@@ -78,7 +78,7 @@ finalize_kernel(const float* __restrict__ logits, const float* __restrict__ lse,
     const int key0 = (blockIdx.x * (kFinThreads / 32) + warp) * 32;
     if (key0 >= n) return;
 
-    const uint4* vrow = reinterpret_cast<const uint4*>(v + ((size_t)ug * n + key0) * D);
+    const uint4* vrow = reinterpret_cast<const uint4*>(v + ((size_t)ug * cap + key0) * D);
     float my_sumsq = 0.f;
 #pragma unroll 4
     for (int t = 0; t < STEPS; ++t) {
@@ -342,16 +342,16 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
     switch (s.head_dim) {
         case 64:
             finalize_kernel<64><<<grid, kFinThreads, 0, st>>>(logits, lse, v, s.n_q_heads, s.n_kv_heads,
-                                                             s.n_keys, s.group_mode, epsilon, scores);
+                                                             s.n_keys, ea_kv_cap(s), s.group_mode, epsilon, scores);
             break;
         case 128:
             finalize_kernel<128><<<grid, kFinThreads, 0, st>>>(logits, lse, v, s.n_q_heads,
-                                                              s.n_kv_heads, s.n_keys, s.group_mode,
+                                                              s.n_kv_heads, s.n_keys, ea_kv_cap(s), s.group_mode,
                                                               epsilon, scores);
             break;
         case 256:
             finalize_kernel<256><<<grid, kFinThreads, 0, st>>>(logits, lse, v, s.n_q_heads,
-                                                              s.n_kv_heads, s.n_keys, s.group_mode,
+                                                              s.n_kv_heads, s.n_keys, ea_kv_cap(s), s.group_mode,
                                                               epsilon, scores);
             break;
         default:

@@ -671,10 +671,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 
 // ------------------------------------------------------------------------------------------
 // K as a rank-3 tensor (d, n, unit*kv_head); one box is 64 channels x 128 keys, 128-byte swizzle.
-// Rows past n read as zero.
-bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, long long heads) {
+// Rows past n read as zero; heads are kv_capacity rows apart.
+bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, int cap, long long heads) {
     return ea_tensor_map_bf16_3d(map, k, (uint64_t)d, (uint64_t)n, (uint64_t)heads, (uint64_t)d * 2,
-                                 (uint64_t)n * d * 2, 64, kTileKeys);
+                                 (uint64_t)cap * d * 2, 64, kTileKeys);
 }
 
 template <int D, bool PAIR>
@@ -712,7 +712,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     *n_chunks_out = p.n_chunks * (PAIR ? 2 : 1);
 
     CUtensorMap k_map;
-    if (!make_k_map(&k_map, k, D, s.n_keys, (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
+    if (!make_k_map(&k_map, k, D, s.n_keys, ea_kv_cap(s), (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
 
     sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(form, s.n_q_heads, s.n_kv_heads, image, vec);
     auto kern = logits_mma_kernel<D, PAIR>;

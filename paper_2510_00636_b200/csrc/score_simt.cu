@@ -13,7 +13,7 @@ constexpr int kKeysPerCta = (kThreads / 32) * kKeysPerWarp;   // 64
 
 template <int D>
 __global__ void __launch_bounds__(kThreads)
-logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form, int Hq, int Hkv, int n,
+logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form, int Hq, int Hkv, int n, int cap,
                    float* __restrict__ logits) {
     constexpr int CT = D / 32;
     __shared__ __nv_bfloat16 k_s[kKeysPerCta][D];
@@ -21,7 +21,7 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form,
     const int uh = blockIdx.y;
     const int u = uh / Hq, h = uh % Hq, g = h / (Hq / Hkv);
     const int key0 = blockIdx.x * kKeysPerCta;
-    const __nv_bfloat16* kk = k + ((size_t)u * Hkv + g) * (size_t)n * D;
+    const __nv_bfloat16* kk = k + ((size_t)u * Hkv + g) * (size_t)cap * D;
     const size_t set_head = (size_t)(u / form.units_per_set) * Hq + h;
     const float* S = form.quad + set_head * D * D;
     const float* mu = form.lin ? form.lin + set_head * D : nullptr;
@@ -81,15 +81,15 @@ ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv
     switch (s.head_dim) {
         case 64:
             logits_simt_kernel<64><<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads,
-                                                             s.n_kv_heads, s.n_keys, logits);
+                                                             s.n_kv_heads, s.n_keys, ea_kv_cap(s), logits);
             break;
         case 128:
             logits_simt_kernel<128><<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads,
-                                                              s.n_kv_heads, s.n_keys, logits);
+                                                              s.n_kv_heads, s.n_keys, ea_kv_cap(s), logits);
             break;
         case 256: {
             auto kern = logits_simt_kernel<256>;
-            kern<<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads, s.n_kv_heads, s.n_keys, logits);
+            kern<<<grid, kThreads, 0, st>>>(k, form, s.n_q_heads, s.n_kv_heads, s.n_keys, ea_kv_cap(s), logits);
             break;
         }
         default:

@@ -341,7 +341,7 @@ select_cluster_kernel(const float* __restrict__ scores, int n, int n_kept, int s
 }
 
 template <int D>
-__global__ void gather_kernel(const int32_t* __restrict__ kept_idx, long long n_rows_out, int n,
+__global__ void gather_kernel(const int32_t* __restrict__ kept_idx, long long n_rows_out, int n,   // n: rows per head in k, v
                               int n_kept, const uint4* __restrict__ k, const uint4* __restrict__ v,
                               uint4* __restrict__ k_out, uint4* __restrict__ v_out) {
     constexpr int LPR = D / 8;                 // 16-byte pieces per row
@@ -633,15 +633,15 @@ ea_status ea_launch_gather_adaptive(const ea_ctx* ctx, const ea_shape& s, int n_
     uint4* vo = reinterpret_cast<uint4*>(v_out);
     switch (s.head_dim) {
         case 64:
-            gather_adaptive_kernel<64><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, s.n_keys, s.n_kv_heads,
+            gather_adaptive_kernel<64><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, ea_kv_cap(s), s.n_kv_heads,
                                                                  unit_stride, k4, v4, ko, vo);
             break;
         case 128:
-            gather_adaptive_kernel<128><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, s.n_keys, s.n_kv_heads,
+            gather_adaptive_kernel<128><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, ea_kv_cap(s), s.n_kv_heads,
                                                                   unit_stride, k4, v4, ko, vo);
             break;
         case 256:
-            gather_adaptive_kernel<256><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, s.n_keys, s.n_kv_heads,
+            gather_adaptive_kernel<256><<<grid, threads, 0, st>>>(kept_idx, head_offsets, rows, ea_kv_cap(s), s.n_kv_heads,
                                                                   unit_stride, k4, v4, ko, vo);
             break;
         default:
@@ -667,13 +667,13 @@ ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, con
     uint4* vo = reinterpret_cast<uint4*>(v_out);
     switch (s.head_dim) {
         case 64:
-            gather_kernel<64><<<grid, threads, 0, st>>>(kept_idx, rows, s.n_keys, n_kept, k4, v4, ko, vo);
+            gather_kernel<64><<<grid, threads, 0, st>>>(kept_idx, rows, ea_kv_cap(s), n_kept, k4, v4, ko, vo);
             break;
         case 128:
-            gather_kernel<128><<<grid, threads, 0, st>>>(kept_idx, rows, s.n_keys, n_kept, k4, v4, ko, vo);
+            gather_kernel<128><<<grid, threads, 0, st>>>(kept_idx, rows, ea_kv_cap(s), n_kept, k4, v4, ko, vo);
             break;
         case 256:
-            gather_kernel<256><<<grid, threads, 0, st>>>(kept_idx, rows, s.n_keys, n_kept, k4, v4, ko, vo);
+            gather_kernel<256><<<grid, threads, 0, st>>>(kept_idx, rows, ea_kv_cap(s), n_kept, k4, v4, ko, vo);
             break;
         default:
             return EA_ERR_UNSUPPORTED;
@@ -689,9 +689,9 @@ ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_
     uint4* k4 = reinterpret_cast<uint4*>(k);
     uint4* v4 = reinterpret_cast<uint4*>(v);
     switch (s.head_dim) {
-        case 64: compact_inplace_kernel<64><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
-        case 128: compact_inplace_kernel<128><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
-        case 256: compact_inplace_kernel<256><<<grid, kIpThreads, 0, st>>>(kept_idx, s.n_keys, n_kept, k4, v4); break;
+        case 64: compact_inplace_kernel<64><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
+        case 128: compact_inplace_kernel<128><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
+        case 256: compact_inplace_kernel<256><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
         default: return EA_ERR_UNSUPPORTED;
     }
     return EA_CHECK_LAUNCH();

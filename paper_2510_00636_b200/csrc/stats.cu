@@ -64,7 +64,8 @@ __device__ __forceinline__ float to_f32(float x) { return x; }
 template <int D, typename QT>
 __global__ void __launch_bounds__(256)
 stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
-                 int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar) {
+                 int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar,
+                 int w_cap, const long long* __restrict__ pushed, int cov_sample) {
     constexpr int HALF = D / 2;
     constexpr int BM = D < 128 ? D : 128;          // block edge
     constexpr int NB1 = D / BM;                    // blocks per edge (1 or 2)
@@ -89,7 +90,27 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
     const int bj = NB1 == 1 ? 0 : (blockIdx.y == 0 ? 0 : 1);
     const bool diag = bi == bj;
     const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
-    const QT* q = q_win + (size_t)uh * W * D;
+    // A window kept as a ring of w_cap rows (pushed != nullptr): the rows written so far, at most
+    // w_cap of them, are the window; mean and covariance do not depend on their order, so a
+    // wrapped ring is read as it lies and a partly filled one by its first rows.
+    if (pushed) {
+        const long long p = pushed[u];
+        W = p < (long long)w_cap ? (int)p : w_cap;
+        if (W < 1 + cov_sample) {
+            // nothing to estimate from: zero statistics (uniform expected attention)
+            if (blockIdx.y == 0)
+                for (int c = tid; c < D; c += 256) mu_bar[(size_t)uh * D + c] = 0.f;
+            const int r0 = NB1 == 1 ? 0 : (blockIdx.y == 2 ? BM : 0), c0 = NB1 == 1 ? 0 : (blockIdx.y == 0 ? 0 : BM);
+            for (int e = tid; e < BM * BM; e += 256) {
+                const int a = r0 + e / BM, c = c0 + e % BM;
+                sigma_bar[(size_t)uh * D * D + (size_t)a * D + c] = 0.f;
+                sigma_bar[(size_t)uh * D * D + (size_t)c * D + a] = 0.f;
+            }
+            return;
+        }
+        inv_norm = 1.0f / (float)(W - cov_sample);
+    }
+    const QT* q = q_win + (size_t)uh * w_cap * D;
 
     for (int m = tid; m < HALF; m += 256) {
         c_s[m] = coef[2 * ((size_t)u * HALF + m)];
@@ -246,7 +267,7 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
 template <typename QT>
 static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_win, const int64_t* pos_next,
                               int n_future, double rope_base, float* rope_coef, float* mu_bar, float* sigma_bar,
-                              cudaStream_t st) {
+                              cudaStream_t st, const int64_t* pushed = nullptr) {
     const int d = s.head_dim, half = d / 2;
     const int n_coef = s.n_units * half;
     rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, st>>>(pos_next, s.n_units, half, d, n_future,
@@ -259,7 +280,9 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return false;
         kern<<<dim3(heads, blocks_y), 256, smem, st>>>(q_win, rope_coef, s.n_q_heads, s.window, s.rope_layout,
-                                                       inv_norm, mu_bar, sigma_bar);
+                                                       inv_norm, mu_bar, sigma_bar, s.window,
+                                                       reinterpret_cast<const long long*>(pushed),
+                                                       s.cov_norm == EA_COV_SAMPLE ? 1 : 0);
         return true;
     };
     bool ok;
@@ -278,6 +301,12 @@ ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
                           const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
                           float* mu_bar, float* sigma_bar, cudaStream_t st) {
     return launch_stats(ctx, s, q_win, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st);
+}
+
+ea_status ea_launch_stats_ring(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_ring,
+                               const int64_t* pushed, const int64_t* pos_next, int n_future, double rope_base,
+                               float* rope_coef, float* mu_bar, float* sigma_bar, cudaStream_t st) {
+    return launch_stats(ctx, s, q_ring, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st, pushed);
 }
 
 ea_status ea_launch_stats_f32(const ea_ctx* ctx, const ea_shape& s, const float* q_win, const int64_t* pos_next,
@@ -355,21 +384,21 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
     switch (d) {
         case 64:
             stats_mma_kernel<64, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<64, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                    s->rope_layout, inv_norm, mu_bar, sigma_bar);
+                                                                    s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0);
             break;
         case 128:
             if (cudaFuncSetAttribute(stats_mma_kernel<128, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      stats_smem_bytes<128, __nv_bfloat16>()) != cudaSuccess)
                 return EA_ERR_CUDA;
             stats_mma_kernel<128, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<128, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar);
+                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0);
             break;
         default:
             if (cudaFuncSetAttribute(stats_mma_kernel<256, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      stats_smem_bytes<256, __nv_bfloat16>()) != cudaSuccess)
                 return EA_ERR_CUDA;
             stats_mma_kernel<256, __nv_bfloat16><<<dim3(heads, 3), 256, stats_smem_bytes<256, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar);
+                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0);
             break;
     }
     return EA_CHECK_LAUNCH();

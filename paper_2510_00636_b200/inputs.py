@@ -112,12 +112,14 @@ def rope_half_split(x: torch.Tensor, positions: torch.Tensor, rope_base: float) 
 
 def generate_layer(cfg: EAConfig, layer: int = 0, device="cpu", n_keys: int | None = None,
                    key_positions: torch.Tensor | None = None, pos_next: int | None = None,
-                   q_phase: float | None = None):
+                   q_phase: float | None = None, draw: int = 0):
     """One layer of synthetic activations.
 
     Returns ``(q_win [B,Hq,W,d], k [B,Hkv,n,d], v [B,Hkv,n,d], pos_next [B] int64)``; the three
     tensors are bf16 on ``device``.  ``q_phase`` (streaming config) rotates the query offsets
-    between two fixed directions: ``off_q = cos(phase) A + sin(phase) B``.
+    between two fixed directions: ``off_q = cos(phase) A + sin(phase) B``.  ``draw`` > 0 gives further
+    independent draws of the noise with the layer's outlier channels, offsets and query factor unchanged
+    (the tokens generated between two compression events of a stream).
     """
     n = cfg.n_keys if n_keys is None else n_keys
     B, Hq, Hkv, d, W = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
@@ -132,8 +134,15 @@ def generate_layer(cfg: EAConfig, layer: int = 0, device="cpu", n_keys: int | No
     scale = torch.ones(d, device=dev)
     scale[perm[: cfg.n_outliers]] = cfg.outlier_scale
 
-    # keys
+    # what belongs to the layer (drawn first, from the layer's seed): channel offsets and the query factor
     off_k = 0.5 * randn(B, Hkv, 1, d)
+    if draw:
+        off_a = 0.5 * randn(B, Hq, 1, d)
+        off_b = 0.5 * randn(B, Hq, 1, d)
+        F = randn(B, Hq, cfg.q_rank, d) / math.sqrt(cfg.q_rank)
+        gen.manual_seed(1000 * cfg.cfg_id + layer + 7919 * draw)      # the noise of this draw
+
+    # keys
     k_pre = randn(B, Hkv, n, d)
     if cfg.drift_sigma > 0:
         k_pre += torch.cumsum(cfg.drift_sigma * randn(B, Hkv, n, d), dim=2)
@@ -144,10 +153,12 @@ def generate_layer(cfg: EAConfig, layer: int = 0, device="cpu", n_keys: int | No
     del k_pre
 
     # window queries (pre-RoPE)
-    off_a = 0.5 * randn(B, Hq, 1, d)
-    off_b = 0.5 * randn(B, Hq, 1, d)
+    if not draw:
+        off_a = 0.5 * randn(B, Hq, 1, d)
+        off_b = 0.5 * randn(B, Hq, 1, d)
     off_q = off_a if q_phase is None else math.cos(q_phase) * off_a + math.sin(q_phase) * off_b
-    F = randn(B, Hq, cfg.q_rank, d) / math.sqrt(cfg.q_rank)
+    if not draw:
+        F = randn(B, Hq, cfg.q_rank, d) / math.sqrt(cfg.q_rank)
     y = randn(B, Hq, W, cfg.q_rank)
     q = ((randn(B, Hq, W, d) + y @ F + off_q) * scale).to(torch.bfloat16)
 

@@ -107,3 +107,147 @@ def test_compression_event_replays_as_a_cuda_graph(ea, oracle):
         own = oracle.select(scores.cpu().numpy().astype(np.float64), cfg.n_kept)
         assert np.array_equal(idx.cpu().numpy(), own)
     ctx.sync_status()
+
+
+def test_one_cache_carried_through_consecutive_events(ea, oracle):
+    """Streaming decode on ONE cache buffer and ONE window ring: every event appends the new pairs behind the
+    kept ones, pushes the new queries into the ring (partly filled, wrapped, more than a ring at once), takes
+    the statistics of what the ring holds, scores the cache at its absolute positions and compacts in place
+    to the budget; the last events run as replays of one captured CUDA graph.  Checked event by event against
+    the oracle's streaming driver on the same bits: statistics, log-scores and scores within the tolerance
+    protocol (every slot stable on these tempered inputs, so scores are held to relative 1e-2 directly), the
+    kept set against the oracle's ranges and bit-exactly against the oracle's selection on the GPU's own
+    scores, and the cache contents bit-exactly.  So that one borderline index cannot derail the comparison of
+    later events, the oracle's cache then continues from the rows the GPU kept (stated in the assertion)."""
+    import dataclasses
+    import gc
+    import parity
+    from oracle.ea_stream import StreamOracle
+    base = inputs.CONFIGS[4].tempered(2.0)
+    budget, every, n0 = 1024, 384, 640
+    cap = budget + every
+    cfg = dataclasses.replace(base, n_layers=1, batch=2, n_keys=n0, n_kept=budget)
+    U, Hq, Hkv, d, W = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
+    dev = torch.device("cuda")
+    _, k0, v0, _ = inputs.generate_layer(cfg, layer=3, device=dev, n_keys=n0, draw=1)
+    k = torch.zeros((U, Hkv, cap, d), dtype=torch.bfloat16, device=dev)
+    v = torch.zeros_like(k)
+    k[:, :, :n0], v[:, :, :n0] = k0, v0
+    ring = torch.zeros((U, Hq, W, d), dtype=torch.bfloat16, device=dev)
+    pushed = torch.zeros((U,), dtype=torch.int64, device=dev)
+    st = StreamOracle(inputs.bits(k0), inputs.bits(v0), window=W, budget=budget)
+    big = ea.make_shape(U, Hq, Hkv, d, cap, W, kv_capacity=cap)
+    ctx = ea.Context.for_shape(big)
+    mu = torch.empty((U, Hq, d), device=dev)
+    sigma = torch.empty((U, Hq, d, d), device=dev)
+    # staging buffers (fixed addresses, so that a captured event can be replayed on new contents)
+    k_new, v_new = (torch.empty((U, Hkv, every, d), dtype=torch.bfloat16, device=dev) for _ in range(2))
+    q_slots = {m: torch.empty((U, Hq, m, d), dtype=torch.bfloat16, device=dev) for m in (100, 200, 184, 384)}
+    pos = torch.empty((U,), dtype=torch.int64, device=dev)
+    pushes = [(100,), (200, 184), (384,), (384,), (384,)]          # below a ring, wrapping, more than a ring at once
+    n_cur, position = n0, n0
+    graph = None
+    for e, push in enumerate(pushes):
+        n = n_cur + every
+        n_kept = min(n, budget)
+        position += every
+        _, kn, vn, _ = inputs.generate_layer(cfg, layer=3, device=dev, n_keys=every, draw=2 + e,
+                                             key_positions=torch.arange(position - every, position))
+        k_new.copy_(kn), v_new.copy_(vn)
+        q_parts = []
+        for i, m in enumerate(push):
+            cfg_q = dataclasses.replace(cfg, window=m)
+            qn, _, _, _ = inputs.generate_layer(cfg_q, layer=3, device=dev, n_keys=1, draw=100 + 10 * e + i,
+                                                q_phase=0.1 * e)
+            q_slots[m].copy_(qn)
+            q_parts.append(inputs.bits(qn))
+        pos.fill_(position)
+        shape_old = ea.make_shape(U, Hq, Hkv, d, n_cur, W, kv_capacity=cap)
+        shape = ea.make_shape(U, Hq, Hkv, d, n, W, kv_capacity=cap)
+        scores = torch.empty((U, Hkv, n), device=dev)
+        logits = torch.empty((U, Hq, n), device=dev)
+        idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, device=dev)
+
+        def event():
+            ea.ea_cache_append(ctx, shape_old, k, v, k_new, v_new)
+            for m in push:
+                ea.ea_window_push(ctx, shape, ring, pushed, q_slots[m])
+            ea.ea_query_stats_ring(ctx, shape, ring, pushed, pos, cfg.n_future, cfg.rope_base, mu, sigma)
+            ea.ea_score(ctx, shape, k, v, mu, sigma, cfg.eps, scores, logits)
+            ea.ea_select_compact_inplace(ctx, shape, scores, n_kept, k, v, idx)
+
+        if e < 3:
+            event()
+        else:
+            if graph is None:
+                # events 2, 3 and 4 have one shape: capture it once (event 2 already ran it eagerly), replay twice
+                gc.collect()
+                graph = torch.cuda.CUDAGraph()
+                g_scores, g_logits, g_idx = scores, logits, idx
+                with torch.cuda.graph(graph):
+                    event()
+            graph.replay()
+            scores, logits, idx = g_scores, g_logits, g_idx
+        ctx.sync_status()
+
+        # the oracle's side of the same event
+        st.append(inputs.bits(kn), inputs.bits(vn))
+        for qb in q_parts:
+            st.push_queries(qb)
+        ref = st.compress(np.full((U,), position), cfg.n_future, cfg.rope_base, cfg.eps)
+        assert int(pushed[0]) == sum(sum(p) for p in pushes[:e + 1])
+        sb, sb_ref = sigma.cpu().numpy().astype(np.float64), ref["sigma_bar"]
+        dg = np.sqrt(np.einsum("uhaa->uha", sb_ref))
+        assert (np.abs(sb - sb_ref) / (dg[..., :, None] * dg[..., None, :] + 1e-30)).max() < 2e-5, f"event {e}"
+        assert (np.abs(mu.cpu().numpy() - ref["mu_bar"]) / (dg + 1e-30)).max() < 2e-5, f"event {e}"
+        delta = parity.logit_error_bound(st.k, ref["mu_bar"], ref["sigma_bar"], 16)
+        bad, _ = parity.check_logits(logits.cpu().numpy(), ref["logits"], delta)
+        assert bad == 0, f"event {e}: {bad} log-scores off"
+        lo, hi = parity.score_range(ref["logits"], delta, st.v, cfg.eps, 0)
+        sc = scores.cpu().numpy()
+        bad, unstable = parity.check_scores(sc, lo, hi)
+        assert bad == 0 and unstable == 0, f"event {e}"
+        np.testing.assert_allclose(sc, ref["scores"], rtol=1e-2, atol=0.0)
+        got = idx.cpu().numpy()
+        missing, present, free = parity.check_kept(got, lo, hi, n_kept)
+        assert missing == 0 and present == 0, f"event {e}"
+        assert np.array_equal(got, oracle.select(sc.astype(np.float64), n_kept)), f"event {e}"
+        if n_kept == n:
+            assert np.array_equal(got, np.broadcast_to(np.arange(n, dtype=np.int32), got.shape))
+        # cache contents after the event: the rows the GPU kept, in order, at the front of every head's range;
+        # the oracle's cache continues from those rows
+        st.keep(got)
+        assert np.array_equal(inputs.bits(k[:, :, :n_kept]), st.k), f"event {e}: key cache differs"
+        assert np.array_equal(inputs.bits(v[:, :, :n_kept]), st.v), f"event {e}: value cache differs"
+        print(f"event {e}: n {n} -> {n_kept}, free indices {free}, differ from oracle's own selection "
+              f"{int((got != ref['kept_idx']).any(-1).sum())} heads")
+        n_cur = n_kept
+
+
+def test_ring_statistics_partly_filled_and_wrapped(ea, oracle):
+    """ea_query_stats_ring against the oracle's statistics of the last min(pushed, W) rows, for a ring that
+    is empty (zero statistics), holds one row, is partly filled, exactly full and wrapped."""
+    torch.manual_seed(5)
+    U, Hq, d, W = 2, 3, 64, 16
+    shape = ea.make_shape(U, Hq, 1, d, 0, W)
+    ctx = ea.Context.for_shape(shape)
+    ring = torch.zeros((U, Hq, W, d), dtype=torch.bfloat16, device="cuda")
+    pushed = torch.zeros((U,), dtype=torch.int64, device="cuda")
+    pos = torch.tensor([100, 7], dtype=torch.int64, device="cuda")
+    mu, sig = ea.ea_query_stats_ring(ctx, shape, ring, pushed, pos, 8, 1e4)
+    ctx.sync_status()
+    assert float(mu.abs().max()) == 0.0 and float(sig.abs().max()) == 0.0
+    everything = None
+    for m in (1, 6, 9, 5, 40):
+        q = (torch.randn(U, Hq, m, d, device="cuda") * 2 + 0.5).to(torch.bfloat16)
+        ea.ea_window_push(ctx, shape, ring, pushed, q)
+        everything = q if everything is None else torch.cat([everything, q], dim=2)
+        mu, sig = ea.ea_query_stats_ring(ctx, shape, ring, pushed, pos, 8, 1e4)
+        ctx.sync_status()
+        tail = inputs.bits(everything[:, :, -W:])
+        mu_r, sig_r = oracle.query_stats(tail, pos.cpu().numpy(), 8, 1e4)
+        sig = sig.cpu().numpy().astype(np.float64)
+        tot = np.sqrt(np.einsum("uhaa->uh", sig_r))[..., None, None] ** 2 / d + 1e-12
+        assert (np.abs(sig - sig_r) / tot).max() < 1e-4, m
+        np.testing.assert_allclose(mu.cpu().numpy(), mu_r, atol=2e-5 * (1 + np.abs(mu_r).max()))
+        assert pushed.tolist() == [everything.shape[2]] * U

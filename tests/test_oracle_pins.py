@@ -584,3 +584,75 @@ def test_stream_events_compose_as_index_maps(oracle):
         origin = np.take_along_axis(origin, idx.astype(np.int64), axis=2)
         for g in range(2):
             assert np.array_equal(st.k[0, g], all_k[0, g][origin[0, g]])
+
+
+# ------------------------------------------------------------------------------------------
+# Quantised cache (oracle/ea_quant.py)
+def test_e4m3_decoder_against_a_library_conversion_of_every_code():
+    """All 256 codes: the formula of the format against torch's float8_e4m3fn -> float32 conversion."""
+    import torch
+    from oracle import ea_quant
+    codes = np.arange(256, dtype=np.uint8)
+    want = torch.from_numpy(codes).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    got = ea_quant.e4m3_decode(codes)
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.isnan(got).sum() == 2
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok], want[ok])
+    assert got[ok].max() == 448.0 and np.abs(got[ok][got[ok] != 0]).min() == 2.0 ** -9
+    # and back: every finite value re-encodes to its own code (up to the sign of zero)
+    back = torch.from_numpy(got[ok].astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(back, codes[ok])
+
+
+def _quant_case(seed, U=2, Hq=4, Hkv=2, d=64, n=96, W=24):
+    import torch
+    rng = np.random.default_rng(seed)
+    def bf(x):
+        return (x.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    q = bf(rng.normal(size=(U, Hq, W, d)) * 0.7 + 0.2)
+    k = rng.normal(size=(U, Hkv, n, d)) * (1 + 3 * (rng.random(d) < 0.05))
+    v = rng.normal(size=(U, Hkv, n, d)) * np.exp(0.5 * rng.normal(size=(U, Hkv, n, 1)))
+    k_scale = (np.abs(k).max(2) / 448.0).astype(np.float32)                  # per channel
+    v_scale = (np.abs(v).max(3) / 448.0).astype(np.float32)                  # per token
+    enc = lambda x: torch.from_numpy(x.astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    return q, enc(k / k_scale[:, :, None, :]), k_scale, enc(v / v_scale[..., None]), v_scale
+
+
+def test_quantised_scoring_equals_scoring_with_the_key_scales_folded_into_the_statistics(oracle):
+    """k = diag(s) k_q, so mu.k = (s*mu).k_q and k^T Sigma k = k_q^T (diag(s) Sigma diag(s)) k_q: an exact
+    identity, which is also how a kernel can consume the codes without ever forming the scaled keys."""
+    from oracle import ea_quant
+    q, kq, ks, vq, vs = _quant_case(11)
+    pos = np.array([96, 200])
+    mu, sig = oracle.query_stats(q, pos, 16, 1e4)
+    direct = ea_quant.logits(ea_quant.dequant_k(kq, ks), mu, sig)
+    G = mu.shape[1] // kq.shape[1]
+    s_q = np.repeat(ks.astype(np.float64), G, axis=1)                       # [U, Hq, d]
+    folded = ea_quant.logits(ea_quant.e4m3_decode(kq), mu * s_q, sig * s_q[..., :, None] * s_q[..., None, :])
+    np.testing.assert_allclose(folded, direct, rtol=1e-12, atol=1e-12)
+    # value side: ||s_i v_q|| = s_i ||v_q||
+    sc = ea_quant.scores(direct, ea_quant.dequant_v(vq, vs), 0.02)
+    unit = ea_quant.scores(direct, ea_quant.e4m3_decode(vq), 0.0) * vs
+    sc0 = ea_quant.scores(direct, ea_quant.dequant_v(vq, vs), 0.0)
+    np.testing.assert_allclose(unit, sc0, rtol=1e-12)
+    assert (sc > sc0).all()
+
+
+def test_quantised_oracle_with_unit_scales_is_the_bf16_oracle(oracle):
+    """E4M3 values are bf16 values: with all scales one, the quantised path must reproduce the pinned C oracle
+    run on the same numbers as bf16 bits, through every step including the kept rows."""
+    from oracle import ea_quant
+    q, kq, ks, vq, vs = _quant_case(12)
+    ks[:], vs[:] = 1.0, 1.0
+    to_bf16 = lambda codes: (ea_quant.e4m3_decode(codes).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    pos = np.array([96, 96])
+    got = ea_quant.compress(q, kq, ks, vq, vs, pos, 16, 1e4, 0.02, 40)
+    want = oracle.compress(q, to_bf16(kq), to_bf16(vq), pos, 16, 1e4, 0.02, 40)
+    np.testing.assert_allclose(got["logits"], want["logits"], rtol=1e-11, atol=1e-11)
+    np.testing.assert_allclose(got["scores"], want["scores"], rtol=1e-11)
+    assert np.array_equal(got["kept_idx"], want["kept_idx"])
+    assert np.array_equal(to_bf16(got["k_out"]), want["k_out"]) and np.array_equal(to_bf16(got["v_out"]), want["v_out"])
+    for mode in (1, 2):
+        s = got["logits"]
+        np.testing.assert_allclose(ea_quant.scores(s, ea_quant.e4m3_decode(vq), 0.02, mode),
+                                   oracle.scores(s, to_bf16(vq), 0.02, group_mode=mode), rtol=1e-11)

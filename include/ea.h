@@ -260,6 +260,42 @@ ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const v
                       float* logits_opt, void* cuda_stream);
 
 /*
+ * The same scores on a quantised cache.  The paper calls quantisation
+ * orthogonal to eviction and combinable with it (Related Works,
+ * "Quantization") and fixes no format; this library's reading: keys and values
+ * are FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no
+ * infinities, largest finite value 448) with fp32 scales,
+ *   k[u,g,i,c] = decode(k_q8[u,g,i,c]) * k_scale[u,g,c]     one scale per channel
+ *   v[u,g,i,c] = decode(v_q8[u,g,i,c]) * v_scale[u,g,i]     one scale per token
+ * and the scores are Eq. 7, 8, 9 of ea_score on these k, v.  The key scales
+ * are folded into mu_bar and sigma_bar (mu.k = (s*mu).x and
+ * k^T Sigma k = x^T diag(s) Sigma diag(s) x for the code row x), so the tensor-
+ * core kernel runs on the codes, widened to bf16 without rounding; the value
+ * norm is v_scale_i ||x_i||.
+ *
+ * k_q8, v_q8  uint8 [n_units, Hkv, n, d] E4M3 codes, 16-byte aligned, dense
+ *             (kv_capacity must be 0 or n_keys: EA_ERR_UNSUPPORTED otherwise)
+ * k_scale     fp32 [n_units, Hkv, d];   v_scale  fp32 [n_units, Hkv, n]
+ * k_scratch   bf16 [n_units, Hkv, n, d]  caller-owned scratch; holds the
+ *             widened key codes on return
+ * the other arguments as for ea_score.
+ */
+ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, const float* k_scale,
+                      const void* v_q8, const float* v_scale, const float* mu_bar,
+                      const float* sigma_bar, float epsilon, void* k_scratch, float* scores,
+                      float* logits_opt, void* cuda_stream);
+/*
+ * ea_select_compact on a quantised cache: the same selection, then the kept
+ * code rows and the value scales of their tokens are gathered (the key scales
+ * belong to the channels and stay as they are).
+ * k_out, v_out  uint8 [n_units, Hkv, n_kept, d];  v_scale_out fp32 [n_units, Hkv, n_kept]
+ */
+ea_status ea_select_compact_q8(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                               int32_t n_kept, const void* k_q8, const void* v_q8,
+                               const float* v_scale, int32_t* kept_idx, void* k_out, void* v_out,
+                               float* v_scale_out, void* cuda_stream);
+
+/*
  * Eviction and compaction: per (unit, KV head) keep the n_kept pairs with the
  * highest score; among equal scores the lowest index wins; kept indices are
  * emitted in ascending order (the cache keeps its temporal order) and the

@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_cache_append", "ea_window_push", "ea_query_stats_ring",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_select_compact_q8",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -90,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.ea_query_stats_ring.argtypes = [vp, sp, vp, vp, vp, i32, f64, vp, vp, vp]
         for name in ("ea_cache_append", "ea_window_push", "ea_query_stats_ring"):
             getattr(L, name).restype = ctypes.c_int
+        L.ea_score_q8.argtypes = [vp, sp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp]
+        L.ea_select_compact_q8.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.ea_score_q8.restype = L.ea_select_compact_q8.restype = ctypes.c_int
         L.ea_set_sm_budget.argtypes = [vp, i32]
         L.ea_set_side_sms.argtypes = [vp, i32]
         L.ea_set_side_sms.restype = ctypes.c_int
@@ -311,6 +314,43 @@ def ea_score(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, epsilon: float
     _check(lib().ea_score(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(mu_bar), _ptr(sigma_bar),
                           float(epsilon), _ptr(scores), _ptr(logits), _stream(ctx.device)), "ea_score")
     return (scores, logits) if (want_logits or logits is not None) else scores
+
+
+def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar, sigma_bar, epsilon: float,
+                k_scratch=None, scores=None, logits=None, want_logits: bool = False):
+    """Scores of a quantised cache: k_q8, v_q8 uint8 [U,Hkv,n,d] (E4M3 codes), k_scale fp32 [U,Hkv,d],
+    v_scale fp32 [U,Hkv,n] -> scores fp32 [U,Hkv,n] (and the log-scores if asked)."""
+    _dev_tensor(k_q8, torch.uint8, "k_q8")
+    _dev_tensor(v_q8, torch.uint8, "v_q8")
+    _dev_tensor(k_scale, torch.float32, "k_scale")
+    _dev_tensor(v_scale, torch.float32, "v_scale")
+    U, Hq, Hkv, n, d = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys, shape.head_dim
+    dev = k_q8.device
+    if k_scratch is None:
+        k_scratch = torch.empty((U, Hkv, n, d), dtype=torch.bfloat16, device=dev)
+    if scores is None:
+        scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=dev)
+    if logits is None and want_logits:
+        logits = torch.empty((U, Hq, n), dtype=torch.float32, device=dev)
+    _check(lib().ea_score_q8(ctx._h, ctypes.byref(shape), _ptr(k_q8), _ptr(k_scale), _ptr(v_q8), _ptr(v_scale),
+                             _ptr(mu_bar), _ptr(sigma_bar), float(epsilon), _ptr(k_scratch), _ptr(scores),
+                             _ptr(logits), _stream(ctx.device)), "ea_score_q8")
+    return (scores, logits) if (want_logits or logits is not None) else scores
+
+
+def ea_select_compact_q8(ctx: Context, shape: Shape, scores, n_kept: int, k_q8, v_q8, v_scale):
+    """-> (kept_idx int32 [U,Hkv,n_kept], k_out, v_out uint8 [U,Hkv,n_kept,d], v_scale_out fp32 [U,Hkv,n_kept])."""
+    _dev_tensor(scores, torch.float32, "scores")
+    U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
+    dev = scores.device
+    idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, device=dev)
+    k_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.uint8, device=dev)
+    v_out = torch.empty_like(k_out)
+    vs_out = torch.empty((U, Hkv, n_kept), dtype=torch.float32, device=dev)
+    _check(lib().ea_select_compact_q8(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k_q8), _ptr(v_q8),
+                                      _ptr(v_scale), _ptr(idx), _ptr(k_out), _ptr(v_out), _ptr(vs_out),
+                                      _stream(ctx.device)), "ea_select_compact_q8")
+    return idx, k_out, v_out, vs_out
 
 
 def ea_wo_gram(ctx: Context, w_o, n_q_heads: int, head_dim: int, wo_gram=None):

@@ -342,7 +342,7 @@ ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const v
     const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
     const ea_quad_form eq7 = ea_eq7_form(*shape, mu_bar, sigma_bar);
     // ||W_o^h v||^2 = v^T (W_o^h^T W_o^h) v: the same kernels, the value rows in place of the keys
-    const ea_quad_form norm2 = {nullptr, wo_gram, shape->n_units / n_weight_sets, 0.0f, 1.0f};
+    const ea_quad_form norm2 = {nullptr, wo_gram, shape->n_units / n_weight_sets, 0.0f, 1.0f, nullptr};
     if (ea_mma_path_supported(*shape)) {
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
         float* vec = reinterpret_cast<float*>(ws + plan.vec);

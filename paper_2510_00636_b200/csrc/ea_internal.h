@@ -105,9 +105,12 @@ struct ea_quad_form {
     const float* quad;       // fp32 [sets * Hq, d, d]
     int units_per_set;       // unit u reads set u / units_per_set
     float lin_scale, quad_scale;
+    // rows given as codes x with the real row diag(ch_scale) x (quantised keys): fp32 [units * Hkv, d] or
+    // nullptr.  The scales are folded into lin and quad as they are read (lin_c s_c, quad_ac s_a s_c).
+    const float* ch_scale;
 };
 static inline ea_quad_form ea_eq7_form(const ea_shape& s, const float* mu_bar, const float* sigma_bar) {
-    ea_quad_form f = {mu_bar, sigma_bar, 1, 1.0f / sqrtf((float)s.head_dim), 0.5f / (float)s.head_dim};
+    ea_quad_form f = {mu_bar, sigma_bar, 1, 1.0f / sqrtf((float)s.head_dim), 0.5f / (float)s.head_dim, nullptr};
     return f;
 }
 
@@ -154,8 +157,21 @@ ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* 
 ea_status ea_launch_wo_gram(const ea_ctx* ctx, const __nv_bfloat16* w_o, int d_model, int n_sets, int Hq, int d,
                             float* gram, cudaStream_t st);
 ea_status ea_launch_lse(const ea_ctx* ctx, const ea_shape& s, const float* logits, float* lse, cudaStream_t st);
+// one softmax row per KV head over the mean of its group's log-scores (EA_GROUP_MEAN_LOGIT)
+ea_status ea_launch_lse_grouped(const ea_ctx* ctx, const ea_shape& s, const float* logits, float* lse, cudaStream_t st);
 ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
                                 const float* wo_norm2, float epsilon, float* scores, cudaStream_t st);
+
+// Quantised cache (FP8 E4M3 codes with scales): key codes widened to bf16 (exact), the weighting on value codes
+// with one scale per token, and the gather of code rows with their value scales.
+ea_status ea_launch_dequant_k(const ea_ctx* ctx, const ea_shape& s, const uint8_t* k_q8, __nv_bfloat16* k_codes,
+                              cudaStream_t st);
+ea_status ea_launch_finalize_q8(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
+                                const uint8_t* v_q8, const float* v_scale, float epsilon, float* scores,
+                                cudaStream_t st);
+ea_status ea_launch_gather_q8(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
+                              const uint8_t* k_q8, const uint8_t* v_q8, const float* v_scale, uint8_t* k_out,
+                              uint8_t* v_out, float* v_scale_out, cudaStream_t st);
 
 ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
                            int32_t* kept_idx, cudaStream_t st);

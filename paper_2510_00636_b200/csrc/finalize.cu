@@ -425,6 +425,12 @@ ea_status ea_launch_lse(const ea_ctx* ctx, const ea_shape& s, const float* logit
     return EA_CHECK_LAUNCH();
 }
 
+ea_status ea_launch_lse_grouped(const ea_ctx* ctx, const ea_shape& s, const float* logits, float* lse, cudaStream_t st) {
+    lse_kernel<<<s.n_units * s.n_kv_heads, kLseThreads, 0, st>>>(logits, s.n_keys, s.n_q_heads / s.n_kv_heads, lse);
+    ea_count_launches(ctx, 1);
+    return EA_CHECK_LAUNCH();
+}
+
 ea_status ea_launch_finalize_wo(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
                                 const float* wo_norm2, float epsilon, float* scores, cudaStream_t st) {
     dim3 grid((unsigned)((s.n_keys + 255) / 256), (unsigned)(s.n_units * s.n_kv_heads));

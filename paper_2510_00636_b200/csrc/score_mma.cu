@@ -125,6 +125,8 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
     const float* S = form.quad + set_head * D * D;
     uint8_t* img = image + ((size_t)(u * Hkv + g) * n_subsets + hs) * G::IMG_FULL;   // 16-byte aligned
     const float quad_scale = form.quad_scale;  // 1/(2d) for Eq. 7, a power of two: the scaling is exact
+    // per-channel scales of quantised rows (1 when the rows are the real keys)
+    const float* cs = form.ch_scale ? form.ch_scale + (size_t)(u * Hkv + g) * D : nullptr;
 
     // Image rows in blocks of 32: the block needs S[c][:] (its own rows) and S[:][c] (its columns).  The
     // columns go through shared memory, loaded as 128-byte row segments, so that every global sector
@@ -145,6 +147,7 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
         __syncthreads();
         const int c = c_blk + lane;
         const int row = G::col(j, c);
+        const float s_c = cs ? cs[c] : 1.f;
         for (int a0 = warp * 8; a0 < D; a0 += 64) {
             const float4 r0 = __ldg(reinterpret_cast<const float4*>(S + (size_t)c * D + a0));
             const float4 r1 = __ldg(reinterpret_cast<const float4*>(S + (size_t)c * D + a0) + 1);
@@ -160,11 +163,12 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
                     if (a != c) {
                         // the two mirrored entries together carry (S_ca + S_ac) * quad_scale, split into a
                         // bf16 and the bf16 rounding of its remainder
-                        const float x = (own[2 * p + q] + col_s[a][lane]) * quad_scale;
+                        const float s_ac = cs ? s_c * cs[a] : 1.f;
+                        const float x = (own[2 * p + q] + col_s[a][lane]) * quad_scale * s_ac;
                         const float hi = __bfloat162float(__float2bfloat16_rn(x));
                         val = a < c ? hi : x - hi;
                     } else if (G::DIAG_MMA) {
-                        val = own[2 * p + q] * quad_scale;           // its bf16 part; the rest in the diagonal blocks
+                        val = own[2 * p + q] * quad_scale * s_c * s_c;   // its bf16 part; the rest in the diagonal blocks
                     }
                     half[q] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(val));
                 }
@@ -180,7 +184,8 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
     // K columns 0 and 1, zeros elsewhere; unswizzled core-matrix layout (8 rows x 16 bytes, K columns
     // 8..15 another 128 bytes on, next 8 rows 256 bytes on)
     for (int c = threadIdx.x; c < D; c += blockDim.x) {
-        const float m = form.lin ? form.lin[set_head * D + c] * form.lin_scale : 0.f;
+        const float sc = cs ? cs[c] : 1.f;
+        const float m = form.lin ? form.lin[set_head * D + c] * form.lin_scale * sc : 0.f;
         const __nv_bfloat16 hi = __float2bfloat16_rn(m);
         const __nv_bfloat16 lo = __float2bfloat16_rn(m - __bfloat162float(hi));
         const int row = G::col(j, c);
@@ -188,7 +193,7 @@ sigma_image_kernel(const ea_quad_form form, int Hq, int Hkv, uint8_t* __restrict
         *reinterpret_cast<uint4*>(dst) =
             make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
         *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
-        const float dg = S[(size_t)c * D + c] * quad_scale;
+        const float dg = S[(size_t)c * D + c] * quad_scale * sc * sc;
         vec[(size_t)uh * D + c] = dg;
         if (G::DIAG_MMA) {
             // block c / 16 (one per MMA step), row n = 16 j + c % 16, K column c % 16: the bf16 of what the

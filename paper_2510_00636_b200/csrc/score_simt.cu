@@ -25,6 +25,11 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form,
     const size_t set_head = (size_t)(u / form.units_per_set) * Hq + h;
     const float* S = form.quad + set_head * D * D;
     const float* mu = form.lin ? form.lin + set_head * D : nullptr;
+    // per-channel scales of quantised rows, folded into the form as it is read
+    const float* cs = form.ch_scale ? form.ch_scale + ((size_t)u * Hkv + g) * D : nullptr;
+    float cs_r[CT];
+#pragma unroll
+    for (int j = 0; j < CT; ++j) cs_r[j] = cs ? cs[(threadIdx.x % 32) + 32 * j] : 1.f;
 
     for (int e = threadIdx.x; e < kKeysPerCta * D; e += kThreads) {
         int r = e / D, c = e % D;
@@ -43,7 +48,7 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form,
     for (int a = 0; a < D; ++a) {
         float srow[CT];
 #pragma unroll
-        for (int j = 0; j < CT; ++j) srow[j] = S[(size_t)a * D + lane + 32 * j];
+        for (int j = 0; j < CT; ++j) srow[j] = S[(size_t)a * D + lane + 32 * j] * (cs ? cs[a] * cs_r[j] : 1.f);
 #pragma unroll
         for (int i = 0; i < kKeysPerWarp; ++i) {
             const float ka = __bfloat162float(kw[i][a]);
@@ -56,7 +61,7 @@ logits_simt_kernel(const __nv_bfloat16* __restrict__ k, const ea_quad_form form,
     const float inv_2d = form.quad_scale;
     float mu_r[CT];
 #pragma unroll
-    for (int j = 0; j < CT; ++j) mu_r[j] = mu ? mu[lane + 32 * j] * inv_sqrt_d : 0.f;
+    for (int j = 0; j < CT; ++j) mu_r[j] = mu ? mu[lane + 32 * j] * inv_sqrt_d * cs_r[j] : 0.f;
 #pragma unroll
     for (int i = 0; i < kKeysPerWarp; ++i) {
         float acc = 0.f;

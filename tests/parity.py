@@ -29,7 +29,7 @@ def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
-def logit_error_bound(k_bits, mu_bar, sigma_bar, sigma_operand_bits: int):
+def logit_error_bound(k_bits, mu_bar, sigma_bar, sigma_operand_bits: int, k_values=None):
     """Per (unit, query head, key) bound on the CUDA path's log-score error.
 
     Three sources, added:
@@ -41,7 +41,7 @@ def logit_error_bound(k_bits, mu_bar, sigma_bar, sigma_operand_bits: int):
         Sigma_bb) (W fp32 additions), again six standard deviations of the summed effect,
         6 * 2^-20 * sum_a k_a^2 Sigma_aa / (2d).
     """
-    k = bf16_to_f64(k_bits)                                  # [U, Hkv, n, d]
+    k = bf16_to_f64(k_bits) if k_values is None else np.asarray(k_values, dtype=np.float64)   # [U, Hkv, n, d]
     U, Hkv, n, d = k.shape
     Hq = mu_bar.shape[1]
     G = Hq // Hkv
@@ -77,12 +77,13 @@ def attention_range(s, delta):
     return lo, hi
 
 
-def score_range(s_or, delta, v_bits, eps, group_mode=0):
+def score_range(s_or, delta, v_bits, eps, group_mode=0, v_values=None):
     """[lo, hi] of the oracle score (a + eps) * ||v|| under the log-score perturbation."""
     U, Hq, n = s_or.shape
-    Hkv = v_bits.shape[1]
+    Hkv = (v_bits if v_values is None else v_values).shape[1]
     G = Hq // Hkv
-    vnorm = np.sqrt((bf16_to_f64(v_bits) ** 2).sum(-1))       # [U, Hkv, n]
+    vv = bf16_to_f64(v_bits) if v_values is None else np.asarray(v_values, dtype=np.float64)
+    vnorm = np.sqrt((vv ** 2).sum(-1))                        # [U, Hkv, n]
     if group_mode == 2:
         s_g = s_or.reshape(U, Hkv, G, n).mean(2)
         d_g = delta.reshape(U, Hkv, G, n).mean(2)

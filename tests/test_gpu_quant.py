@@ -1,0 +1,113 @@
+"""Quantised cache (FP8 E4M3 codes with scales) through the C ABI against the quantised oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import parity
+from paper_2510_00636_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ea():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2510_00636_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+@pytest.mark.parametrize("cfg_id,scale,eps,n,mode", [(0, 2.0, 0.02, None, 0), (1, 2.0, 0.02, None, 0), (1, 3.0, 0.0, None, 0),
+                                                     (1, 20.0, 0.02, None, 0), (0, 2.0, 0.02, 100, 0), (3, 2.0, 0.02, 3000, 0),
+                                                     (0, 2.0, 0.02, None, 1), (0, 2.0, 0.02, None, 2)])
+def test_quantised_whole_path(ea, oracle, cfg_id, scale, eps, n, mode):
+    """Window statistics, scores of the quantised cache and compaction of code rows with their value scales,
+    against the fp64 oracle on the same codes and scales: log-scores and scores within the tolerance protocol
+    (and scores to relative 1e-2 directly where the softmax is spread), the kept set against the oracle's
+    ranges and bit-exactly against the oracle's selection on the GPU's own scores, gathered codes and scales
+    bit-exactly."""
+    from oracle import ea_quant
+    cfg = inputs.CONFIGS[cfg_id].tempered(scale, eps)
+    if n is not None:
+        cfg = dataclasses.replace(cfg, n_layers=1, n_keys=n, n_kept=n // 2)
+    q, k, v, pos = inputs.generate_layer(cfg, device="cuda")
+    kq, ks, vq, vs = inputs.quantize_e4m3(k, v)
+    shape = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window, group_mode=mode)
+    ctx = ea.Context.for_shape(shape)
+    mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
+    sc, lg = ea.ea_score_q8(ctx, shape, kq, ks, vq, vs, mu, sig, cfg.eps, want_logits=True)
+    idx, ko, vo, vso = ea.ea_select_compact_q8(ctx, shape, sc, cfg.n_kept, kq, vq, vs)
+    ctx.sync_status()
+    ref = ea_quant.compress(inputs.bits(q), _np(kq), _np(ks), _np(vq), _np(vs), pos.numpy(), cfg.n_future, cfg.rope_base,
+                            cfg.eps, cfg.n_kept, group_mode=mode)
+    k_real, v_real = ea_quant.dequant_k(_np(kq), _np(ks)), ea_quant.dequant_v(_np(vq), _np(vs))
+    delta = parity.logit_error_bound(None, ref["mu_bar"], ref["sigma_bar"], 16, k_values=k_real)
+    bad, worst = parity.check_logits(_np(lg), ref["logits"], delta)
+    assert bad == 0, (bad, worst)
+    lo, hi = parity.score_range(ref["logits"], delta, None, cfg.eps, mode, v_values=v_real)
+    bad, unstable = parity.check_scores(_np(sc), lo, hi)
+    assert bad == 0
+    if scale <= 3.0:
+        assert unstable == 0
+        np.testing.assert_allclose(_np(sc), ref["scores"], rtol=1e-2, atol=0.0)
+    else:
+        assert unstable <= max(8, lo.size // 1000)
+    got = _np(idx)
+    missing, present, free = parity.check_kept(got, lo, hi, cfg.n_kept)
+    assert missing == 0 and present == 0
+    assert np.array_equal(got, oracle.select(_np(sc).astype(np.float64), cfg.n_kept))
+    i64 = got.astype(np.int64)
+    assert np.array_equal(_np(ko), np.take_along_axis(_np(kq), i64[..., None], axis=2))
+    assert np.array_equal(_np(vo), np.take_along_axis(_np(vq), i64[..., None], axis=2))
+    assert np.array_equal(_np(vso), np.take_along_axis(_np(vs), i64, axis=2))
+    print(dict(logit_worst_rel=worst, free=free,
+               score_worst_rel=float((np.abs(_np(sc) - ref["scores"]) / np.maximum(ref["scores"], 1e-300)).max())))
+
+
+def test_unit_scales_reproduce_the_bf16_path_bitwise(ea):
+    """With all scales one the quantised entry points see the same numbers as the bf16 ones: same log-scores
+    bit for bit (the codes are widened without rounding, the folded scales are ones)."""
+    cfg = inputs.CONFIGS[1].tempered(2.0)
+    q, k, v, pos = inputs.generate_layer(cfg, device="cuda")
+    kq, ks, vq, vs = inputs.quantize_e4m3(k, v)
+    ks.fill_(1.0), vs.fill_(1.0)
+    k16 = kq.view(torch.float8_e4m3fn).to(torch.bfloat16)
+    v16 = vq.view(torch.float8_e4m3fn).to(torch.bfloat16)
+    shape = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window)
+    ctx = ea.Context.for_shape(shape)
+    mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
+    sc8, lg8 = ea.ea_score_q8(ctx, shape, kq, ks, vq, vs, mu, sig, cfg.eps, want_logits=True)
+    sc8, lg8 = sc8.clone(), lg8.clone()
+    sc16, lg16 = ea.ea_score(ctx, shape, k16, v16, mu, sig, cfg.eps, want_logits=True)
+    ctx.sync_status()
+    assert torch.equal(lg8, lg16)
+    torch.testing.assert_close(sc8, sc16, rtol=1e-6, atol=0.0)
+
+
+def test_quantised_calls_validate_their_arguments(ea):
+    cfg = inputs.CONFIGS[0]
+    q, k, v, pos = inputs.generate_layer(cfg, device="cuda")
+    kq, ks, vq, vs = inputs.quantize_e4m3(k, v)
+    shape = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window)
+    ctx = ea.Context.for_shape(shape)
+    mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
+    sc = ea.ea_score_q8(ctx, shape, kq, ks, vq, vs, mu, sig, cfg.eps)
+    strided = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window,
+                            kv_capacity=cfg.n_keys + 8)
+    with pytest.raises(ea.EAError) as e:
+        ea.ea_score_q8(ctx, strided, kq, ks, vq, vs, mu, sig, cfg.eps)
+    assert e.value.status == 2
+    with pytest.raises(ea.EAError) as e:
+        ea.ea_select_compact_q8(ctx, shape, sc, cfg.n_keys + 1, kq, vq, vs)
+    assert e.value.status == 1
+    with pytest.raises(ea.EAError) as e:
+        ea.ea_score_q8(ea.Context(0, 256), shape, kq, ks, vq, vs, mu, sig, cfg.eps)
+    assert e.value.status == 3
+    ctx.sync_status()

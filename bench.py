@@ -124,29 +124,40 @@ class ClockSampler:
 class Workload:
     """All layers of one config resident in HBM, plus preallocated outputs."""
 
-    def __init__(self, cfg: inputs.EAConfig, device, ea, safeguard=None, hidden_dm=None, wo_dm=None):
+    def __init__(self, cfg: inputs.EAConfig, device, ea, safeguard=None, hidden_dm=None, wo_dm=None, fp8=False):
         self.cfg, self.device, self.ea = cfg, device, ea
+        self.fp8 = fp8                      # cache held as FP8 E4M3 codes with scales (ea_score_q8 / ea_select_compact_q8)
         self.safeguard = safeguard          # None: n_kept per head; else head-adaptive with this safeguard share
         self.hidden_dm = hidden_dm          # statistics from hidden states of this width through W_Q
         self.wo_dm = wo_dm                  # ||W_o v|| weighting with an output projection of this width
         L, B = cfg.n_layers, cfg.batch
         U, Hq, Hkv, d, n, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window
         bf, f32 = torch.bfloat16, torch.float32
-        self.k = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
-        self.v = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
+        kv_dtype = torch.uint8 if fp8 else bf
+        self.k = torch.empty((U, Hkv, n, d), dtype=kv_dtype, device=device)
+        self.v = torch.empty((U, Hkv, n, d), dtype=kv_dtype, device=device)
         self.q = torch.empty((U, Hq, W, d), dtype=bf, device=device)
         self.pos = torch.empty((U,), dtype=torch.int64, device=device)
+        if fp8:
+            self.k_scale = torch.empty((U, Hkv, d), dtype=f32, device=device)
+            self.v_scale = torch.empty((U, Hkv, n), dtype=f32, device=device)
+            self.k_scratch = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
         for layer in range(L):
             q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device=device)
             sl = slice(layer * B, (layer + 1) * B)
-            self.q[sl], self.k[sl], self.v[sl], self.pos[sl] = q, k, v, pos.to(device)
+            self.q[sl], self.pos[sl] = q, pos.to(device)
+            if fp8:
+                self.k[sl], self.k_scale[sl], self.v[sl], self.v_scale[sl] = inputs.quantize_e4m3(k, v)
+            else:
+                self.k[sl], self.v[sl] = k, v
             del q, k, v
         self.mu = torch.empty((U, Hq, d), dtype=f32, device=device)
         self.sigma = torch.empty((U, Hq, d, d), dtype=f32, device=device)
         self.scores = torch.empty((U, Hkv, n), dtype=f32, device=device)
         self.idx = torch.empty((U, Hkv, cfg.n_kept), dtype=torch.int32, device=device)
-        self.k_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
-        self.v_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=bf, device=device)
+        self.k_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=kv_dtype, device=device)
+        self.v_out = torch.empty((U, Hkv, cfg.n_kept, d), dtype=kv_dtype, device=device)
+        self.v_scale_out = torch.empty((U, Hkv, cfg.n_kept), dtype=f32, device=device) if fp8 else None
         self.head_off = torch.empty((U, Hkv + 1), dtype=torch.int32, device=device)
         self.n_units = U
         gen = torch.Generator(device=device).manual_seed(1234)
@@ -196,6 +207,13 @@ class Workload:
             else:
                 ea.ea_query_stats(ctx, shape, self.q[u0:u1], self.pos[u0:u1], cfg.n_future, cfg.rope_base,
                                   self.mu[u0:u1], self.sigma[u0:u1])
+            if self.fp8:
+                ea.ea_score_q8(ctx, shape, self.k[u0:u1], self.k_scale[u0:u1], self.v[u0:u1], self.v_scale[u0:u1],
+                               self.mu[u0:u1], self.sigma[u0:u1], cfg.eps, self.k_scratch[u0:u1], self.scores[u0:u1])
+                ea.ea_select_compact_q8(ctx, shape, self.scores[u0:u1], cfg.n_kept, self.k[u0:u1], self.v[u0:u1],
+                                        self.v_scale[u0:u1], out=(self.idx[u0:u1], self.k_out[u0:u1],
+                                                                  self.v_out[u0:u1], self.v_scale_out[u0:u1]))
+                continue
             if self.wo_dm:
                 if self.wo_gram is None:
                     self.wo_gram = ea.ea_wo_gram(ctx, self.w_o, cfg.n_q_heads, cfg.head_dim)
@@ -319,12 +337,14 @@ class DecodeWorkload:
         return slots, bytes_, slots * 2 * cfg.head_dim ** 2 * cfg.group
 
 
-def algorithmic_work(cfg: inputs.EAConfig):
-    """Per step: key-slots, algorithmic HBM bytes (read K, read V, write kept K and V) and the
-    FLOPs of the quadratic form k^T Sigma k for each query head (2 d^2 G per key-slot)."""
+def algorithmic_work(cfg: inputs.EAConfig, fp8: bool = False):
+    """Per step: key-slots, algorithmic HBM bytes (read K, read V, write kept K and V; with an FP8 cache one
+    byte per element plus the fp32 value scale of each token) and the FLOPs of the quadratic form
+    k^T Sigma k for each query head (2 d^2 G per key-slot)."""
     slots = cfg.key_slots
     d, G = cfg.head_dim, cfg.group
-    bytes_ = slots * 4 * d + cfg.n_units * cfg.n_kv_heads * cfg.n_kept * 4 * d
+    row = 2 * d + 4 if fp8 else 4 * d
+    bytes_ = slots * row + cfg.n_units * cfg.n_kv_heads * cfg.n_kept * row
     flops = slots * 2 * d * d * G
     return slots, bytes_, flops
 
@@ -435,12 +455,12 @@ def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_work
         torch.cuda.empty_cache()
     decode = cfg.cfg_id == 4
     wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph) if decode else Workload(cfg, device, ea, args.head_adaptive,
-                                                                 args.hidden_stats, args.with_wo)
+                                                                 args.hidden_stats, args.with_wo, args.kv_dtype == "fp8")
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
     if args.side_sms:
         ctx.set_side_sms(args.side_sms)
-    slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg)
+    slots, alg_bytes, alg_flops = wl.work() if decode else algorithmic_work(cfg, args.kv_dtype == "fp8")
     if args.with_wo:
         alg_flops *= 2                 # v^T (W_o^T W_o) v per query head is a second quadratic form
 
@@ -547,6 +567,9 @@ def main():
                     help="run the value-norm pass on this many SMs beside the log-score kernel (ea_set_side_sms)")
     ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
                     help="default run: skip the device-resident figures of the 32k and the decode workloads")
+    ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
+                    help="prefill configs: cache held as FP8 E4M3 codes with scales (ea_score_q8, ea_select_compact_q8); "
+                         "the device-resident line only, with the algorithmic bytes of that format")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -570,7 +593,7 @@ def main():
     from paper_2510_00636_b200 import binding as ea
     ea.lib()
 
-    variant = args.head_adaptive is not None or args.hidden_stats or args.with_wo
+    variant = args.head_adaptive is not None or args.hidden_stats or args.with_wo or args.kv_dtype == "fp8"
     if variant and cfg.cfg_id == 4:
         raise SystemExit("--head-adaptive, --hidden-stats and --with-wo apply to the prefill configs")
     if variant or cfg.cfg_id == 4:
@@ -591,6 +614,7 @@ def main():
                    "statistics": "window queries given" if not args.hidden_stats else
                                  "hidden states through W_Q, d_model %d" % args.hidden_stats,
                    "value_weight": "||v||" if not args.with_wo else "||W_o v||, d_model %d" % args.with_wo,
+                   "kv_dtype": args.kv_dtype,
                    "cuda_graph": bool(cfg.cfg_id == 4 and args.graph), "key_slots_per_step": slots,
                    "units_per_call": m["units_per_call"], "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (K+V %.1f GB per step)" % (slots * 4 * cfg.head_dim / 1e9)},

@@ -338,15 +338,19 @@ def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar
     return (scores, logits) if (want_logits or logits is not None) else scores
 
 
-def ea_select_compact_q8(ctx: Context, shape: Shape, scores, n_kept: int, k_q8, v_q8, v_scale):
-    """-> (kept_idx int32 [U,Hkv,n_kept], k_out, v_out uint8 [U,Hkv,n_kept,d], v_scale_out fp32 [U,Hkv,n_kept])."""
+def ea_select_compact_q8(ctx: Context, shape: Shape, scores, n_kept: int, k_q8, v_q8, v_scale, out=None):
+    """-> (kept_idx int32 [U,Hkv,n_kept], k_out, v_out uint8 [U,Hkv,n_kept,d], v_scale_out fp32 [U,Hkv,n_kept]);
+    ``out`` may hand in these four tensors."""
     _dev_tensor(scores, torch.float32, "scores")
     U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
     dev = scores.device
-    idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, device=dev)
-    k_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.uint8, device=dev)
-    v_out = torch.empty_like(k_out)
-    vs_out = torch.empty((U, Hkv, n_kept), dtype=torch.float32, device=dev)
+    if out is not None:
+        idx, k_out, v_out, vs_out = out
+    else:
+        idx = torch.empty((U, Hkv, n_kept), dtype=torch.int32, device=dev)
+        k_out = torch.empty((U, Hkv, n_kept, d), dtype=torch.uint8, device=dev)
+        v_out = torch.empty_like(k_out)
+        vs_out = torch.empty((U, Hkv, n_kept), dtype=torch.float32, device=dev)
     _check(lib().ea_select_compact_q8(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k_q8), _ptr(v_q8),
                                       _ptr(v_scale), _ptr(idx), _ptr(k_out), _ptr(v_out), _ptr(vs_out),
                                       _stream(ctx.device)), "ea_select_compact_q8")

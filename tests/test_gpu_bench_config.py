@@ -72,34 +72,50 @@ def test_all_layers_in_one_call_sampled_heads(ea, oracle, cfg_id, samples):
 
 
 def test_decode_events_in_one_call_sampled_heads(ea, oracle):
-    """The streaming config as bench.py replays it (224 units per call, 28 events): after one step the
-    buffers hold the results of the last event; sampled heads of it against the oracle."""
+    """The streaming config as bench.py runs it (224 units per call, 28 events on one carried cache): every
+    event but the last as the benchmark issues them, then the last one call by call with the cache and the
+    window ring snapshotted before scoring; sampled heads of it against the oracle, and the compacted cache
+    against the oracle's gather of the snapshot."""
     import bench
     cfg = inputs.CONFIGS[4]
     dev = torch.device("cuda", 0)
     wl = bench.DecodeWorkload(cfg, dev, ea)
     ctx = wl.make_ctx(wl.n_units)
-    wl.step(ctx, wl.n_units)
-    ctx.sync_status()
+    for e, (pos, n, kept) in enumerate(wl.events[:-1]):
+        wl._event(ctx, n, kept, e % len(wl.new_q), wl.pos[e])
     e = len(wl.events) - 1
     pos, n, kept = wl.events[e]
-    c, q = wl.caches[n], wl.windows[e % len(wl.windows)]
+    ph = e % len(wl.new_q)
+    shape = wl._shape(n)
+    ea.ea_cache_append(ctx, wl._shape(n - wl.every), wl.k, wl.v, wl.new_k[ph], wl.new_v[ph])
+    ea.ea_window_push(ctx, shape, wl.ring, wl.pushed, wl.new_q[ph])
+    ctx.sync_status()
+    assert int(wl.pushed[0]) == cfg.window * len(wl.events)
+    samples = [(0, 0), (101, 2), (223, 3)]
+    snap = {(u, g): (inputs.bits(wl.k[u:u + 1, g:g + 1, :n]), inputs.bits(wl.v[u:u + 1, g:g + 1, :n])) for u, g in samples}
+    scores = torch.empty((wl.n_units, cfg.n_kv_heads, n), device=dev)
+    idx = torch.empty((wl.n_units, cfg.n_kv_heads, kept), dtype=torch.int32, device=dev)
+    ea.ea_query_stats_ring(ctx, shape, wl.ring, wl.pushed, wl.pos[e], cfg.n_future, cfg.rope_base, wl.mu, wl.sigma)
+    ea.ea_score(ctx, shape, wl.k, wl.v, wl.mu, wl.sigma, cfg.eps, scores)
+    ea.ea_select_compact_inplace(ctx, shape, scores, kept, wl.k, wl.v, idx)
+    ctx.sync_status()
     G = cfg.group
-    for u, g in [(0, 0), (101, 2), (223, 3)]:
+    for u, g in samples:
         hq = slice(g * G, (g + 1) * G)
-        qb, kb, vb = inputs.bits(q[u:u + 1, hq]), inputs.bits(c["k"][u:u + 1, g:g + 1]), inputs.bits(c["v"][u:u + 1, g:g + 1])
+        kb, vb = snap[(u, g)]
+        qb = inputs.bits(wl.ring[u:u + 1, hq])
         ref = oracle.compress(qb, kb, vb, np.array([pos], np.int64), cfg.n_future, cfg.rope_base, cfg.eps, kept)
         delta = parity.logit_error_bound(kb, ref["mu_bar"], ref["sigma_bar"], 16)
         lo, hi = parity.score_range(ref["logits"], delta, vb, cfg.eps, 0)
-        got = c["scores"][u:u + 1, g:g + 1].cpu().numpy()
+        got = scores[u:u + 1, g:g + 1].cpu().numpy()
         bad, unstable = parity.check_scores(got, lo, hi)
         assert bad == 0 and unstable <= max(8, lo.size // 1000), (u, g, bad, unstable)
-        idx = c["idx"][u:u + 1, g:g + 1].cpu().numpy()
-        missing, present, _ = parity.check_kept(idx, lo, hi, kept)
+        own_idx = idx[u:u + 1, g:g + 1].cpu().numpy()
+        missing, present, _ = parity.check_kept(own_idx, lo, hi, kept)
         assert missing == 0 and present == 0, (u, g, missing, present)
         own = oracle.select(got.astype(np.float64), kept)
-        assert np.array_equal(idx, own)
-        assert np.array_equal(inputs.bits(c["k_out"][u:u + 1, g:g + 1]), oracle.gather(kb, own))
-        assert np.array_equal(inputs.bits(c["v_out"][u:u + 1, g:g + 1]), oracle.gather(vb, own))
+        assert np.array_equal(own_idx, own)
+        assert np.array_equal(inputs.bits(wl.k[u:u + 1, g:g + 1, :kept]), oracle.gather(kb, own))
+        assert np.array_equal(inputs.bits(wl.v[u:u + 1, g:g + 1, :kept]), oracle.gather(vb, own))
     del wl
     torch.cuda.empty_cache()

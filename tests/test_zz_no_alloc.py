@@ -56,6 +56,34 @@ def test_static_scratch_call_matches_context_call_twice_in_a_row(ea):
         assert torch.equal(mu, mu_ref) and torch.equal(sig, sig_ref)
 
 
+@pytest.mark.parametrize("d,layout,U", [(64, 0, 3), (64, 1, 512), (128, 1, 256), (256, 0, 4), (256, 1, 128)])
+def test_static_scratch_call_every_head_dim_up_to_the_limit(ea, d, layout, U):
+    """Each head_dim has its own launch shape (one block row at 64 and 128, three at 256), both rotation
+    pairings, and the largest problem the fixed array admits (n_units * head_dim / 2 == the stated maximum);
+    a second call right behind the first must neither change the result nor take any device memory."""
+    Hq, W, T = 2, 40, 64
+    if U * d // 2 > ea.STATIC_MAX_ROPE_PAIRS:
+        pytest.skip("beyond the fixed array")
+    at_limit = U * d // 2 == ea.STATIC_MAX_ROPE_PAIRS
+    q = _window(U, Hq, W, d, 100 + d + layout)
+    pos = torch.arange(U, dtype=torch.int64, device="cuda") * 37 + 5
+    shape = ea.make_shape(U, Hq, 1, d, 0, W, rope_layout=layout)
+    ctx = ea.Context.for_shape(shape)
+    mu_ref, sig_ref = ea.ea_query_stats(ctx, shape, q, pos, T, 1e6)
+    ctx.sync_status()
+    mu, sig = torch.empty_like(mu_ref), torch.empty_like(sig_ref)
+    ea.ea_query_stats_static(shape, q, pos, T, 1e6, mu, sig)
+    torch.cuda.synchronize()
+    assert torch.equal(mu, mu_ref) and torch.equal(sig, sig_ref), (d, layout, U, at_limit)
+    free_before, _ = torch.cuda.mem_get_info()
+    mu.fill_(0), sig.fill_(0)
+    ea.ea_query_stats_static(shape, q, pos, T, 1e6, mu, sig)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the call took device memory"
+    assert torch.equal(mu, mu_ref) and torch.equal(sig, sig_ref)
+
+
 def test_static_scratch_call_refuses_oversized_and_bad_shapes(ea):
     L = ea.lib()
     too_many = ea.STATIC_MAX_ROPE_PAIRS // 64 + 1            # units at head_dim 128

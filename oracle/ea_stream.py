@@ -19,6 +19,26 @@ import numpy as np
 from oracle import ea_oracle
 
 
+def fill_holes(kept_idx, n_kept: int):
+    """Unordered in-place compaction as an index map.  ``kept_idx`` [..., n_kept] ascending kept positions of a
+    cache of n rows -> ``where`` [..., n_kept]: the original row that ends up at position j when every kept row
+    below ``n_kept`` stays where it is and the kept rows at or beyond ``n_kept`` (ascending) move into the
+    evicted positions below ``n_kept`` (ascending).  The kept SET is unchanged, only the order is."""
+    idx = np.asarray(kept_idx)
+    out = np.empty_like(idx)
+    flat_in, flat_out = idx.reshape(-1, idx.shape[-1]), out.reshape(-1, idx.shape[-1])
+    for h in range(flat_in.shape[0]):
+        kept = [int(i) for i in flat_in[h]]
+        stay = set(i for i in kept if i < n_kept)
+        movers = [i for i in kept if i >= n_kept]
+        holes = [p for p in range(n_kept) if p not in stay]
+        where = list(range(n_kept))
+        for p, src in zip(holes, movers):
+            where[p] = src
+        flat_out[h] = where
+    return out
+
+
 class StreamOracle:
     """Caches ``k, v`` uint16 [U, Hkv, n, d] (bf16 bit patterns) and pushed queries uint16 [U, Hq, m, d]."""
 

@@ -656,3 +656,28 @@ def test_quantised_oracle_with_unit_scales_is_the_bf16_oracle(oracle):
         s = got["logits"]
         np.testing.assert_allclose(ea_quant.scores(s, ea_quant.e4m3_decode(vq), 0.02, mode),
                                    oracle.scores(s, to_bf16(vq), 0.02, group_mode=mode), rtol=1e-11)
+
+
+def test_fill_holes_is_a_permutation_of_the_kept_set_that_moves_only_the_tail(oracle):
+    """The unordered compaction map: same kept set, rows below n_kept that are kept do not move, exactly the
+    kept rows beyond n_kept move, and they fill the evicted positions in ascending order of both; checked
+    on every subset of a small cache by brute force."""
+    from itertools import combinations
+    from oracle.ea_stream import fill_holes
+    n, n_kept = 7, 4
+    for kept in combinations(range(n), n_kept):
+        where = fill_holes(np.array([kept], dtype=np.int32), n_kept)[0]
+        assert sorted(where) == list(kept)
+        for p in range(n_kept):
+            if p in kept:
+                assert where[p] == p
+        moved_to = [p for p in range(n_kept) if where[p] != p]
+        assert [where[p] for p in moved_to] == [i for i in kept if i >= n_kept]
+        assert moved_to == [p for p in range(n_kept) if p not in kept]
+    rng = np.random.default_rng(0)
+    sc = rng.random((2, 3, 50))
+    idx = oracle.select(sc, 20)
+    where = fill_holes(idx, 20)
+    assert np.array_equal(np.sort(where, axis=-1), idx)
+    ident = fill_holes(np.broadcast_to(np.arange(20, dtype=np.int32), (2, 3, 20)), 20)
+    assert np.array_equal(ident, np.broadcast_to(np.arange(20), (2, 3, 20)))

@@ -36,8 +36,8 @@ from paper_2510_00636_b200 import inputs  # noqa: E402
 # key-slots of that launch (one ncu --set full capture per shape on a few layers, clocks not locked),
 # keyed by (head_dim, query heads per KV head): the log-score write and the sharing of key tiles depend
 # on both.  NCU_CAPTURE_SOURCE is the fingerprint of the kernel source that was captured.
-NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.1018e9 / 2097152, (128, 4): 293.9e6 / 1048576}
-NCU_CAPTURE_SOURCE = "to-be-recorded"
+NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.10297e9 / 2097152, (128, 4): 294.13e6 / 1048576}
+NCU_CAPTURE_SOURCE = "202c9f43def85c26"
 # nominal figures of the part, reported beside the measured denominators
 NOMINAL_HBM_GBS, NOMINAL_TFLOPS = 8000.0, 2250.0
 
@@ -244,9 +244,11 @@ class DecodeWorkload:
     slowly turning query means; a step starts from 2048 valid rows of whatever the buffer holds (rows kept
     by the previous step: synthetic rows of the same distribution)."""
 
-    def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False):
+    def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False,
+                 unordered: bool = False):
         import dataclasses
         self.cfg, self.device, self.ea = cfg, device, ea
+        self.unordered = unordered          # ea_select_compact_inplace_unordered: only the tail's kept rows move
         self.use_graph, self.graphs = use_graph, {}
         self.events = inputs.decode_schedule()
         self.every = self.events[0][1] - 2048
@@ -299,7 +301,8 @@ class DecodeWorkload:
         ea.ea_window_push(ctx, shape, self.ring, self.pushed, self.new_q[ph])
         ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
         ea.ea_score(ctx, shape, self.k, self.v, self.mu, self.sigma, cfg.eps, scores)
-        ea.ea_select_compact_inplace(ctx, shape, scores, kept, self.k, self.v, idx)
+        compact = ea.ea_select_compact_inplace_unordered if self.unordered else ea.ea_select_compact_inplace
+        compact(ctx, shape, scores, kept, self.k, self.v, idx)
 
     def step(self, ctx, units_per_call):
         for e, (pos, n, kept) in enumerate(self.events):
@@ -454,7 +457,7 @@ def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_work
         gc.collect()
         torch.cuda.empty_cache()
     decode = cfg.cfg_id == 4
-    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph) if decode else Workload(cfg, device, ea, args.head_adaptive,
+    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph, unordered=args.unordered) if decode else Workload(cfg, device, ea, args.head_adaptive,
                                                                  args.hidden_stats, args.with_wo, args.kv_dtype == "fp8")
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
@@ -567,6 +570,9 @@ def main():
                     help="run the value-norm pass on this many SMs beside the log-score kernel (ea_set_side_sms)")
     ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
                     help="default run: skip the device-resident figures of the 32k and the decode workloads")
+    ap.add_argument("--unordered", action="store_true",
+                    help="decode config: compact with ea_select_compact_inplace_unordered (kept rows of the tail fill "
+                         "the evicted positions; the cache loses its temporal order, not its contents)")
     ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
                     help="prefill configs: cache held as FP8 E4M3 codes with scales (ea_score_q8, ea_select_compact_q8); "
                          "the device-resident line only, with the algorithmic bytes of that format")
@@ -625,7 +631,8 @@ def main():
         "clocks": m["clocks"],
     }
     if cfg.cfg_id == 4:
-        result["config"]["cache"] = "one carried buffer per sequence, compacted in place, 512 pairs appended per event"
+        result["config"]["cache"] = "one carried buffer per sequence, compacted in place (%s), 512 pairs appended per event" % (
+            "unordered: the tail's kept rows fill the evicted positions" if args.unordered else "temporal order kept")
 
     # end to end from host buffers through ea_compress_host (rank-local; max over ranks)
     if not args.skip_e2e:
@@ -645,6 +652,12 @@ def main():
                                  "kernel_frac": om["roofline"]["frac"], "kernel_ms": om["roofline"]["kernel_ms"],
                                  "kernel_mcycles": om["roofline"]["kernel_mcycles"], "sm_mhz": om["clocks"]["sm_mhz"],
                                  "gpu_launches": om["gpu_launches"]}
+        args.unordered = True
+        om = measure(args, inputs.CONFIGS[4], ea, device, world, local, peaks, max(5, args.steps // 2), 3, keep_workload=False)
+        args.unordered = False
+        others[inputs.CONFIGS[4].name]["unordered_compaction"] = {
+            "ms_per_step": om["ms"], "value": om["slots"] / (om["ms"] * 1e-3) / 1e9,
+            "path_roofline_frac": om["path_roofline"]["frac"]}
         result["other_configs"] = others
 
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:

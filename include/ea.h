@@ -334,6 +334,24 @@ ea_status ea_select_compact_inplace(ea_ctx* ctx, const ea_shape* shape, const fl
                                     void* cuda_stream);
 
 /*
+ * The same eviction without the temporal order (the paper has no counterpart:
+ * attention does not depend on the order of the cached pairs, and post-RoPE
+ * keys carry their positions).  Kept rows below n_kept stay where they are; the
+ * kept rows at or beyond n_kept move, in ascending order, into the evicted
+ * positions below n_kept, in ascending order.  In a stream that appends a few
+ * hundred pairs per event to a cache of thousands this moves only about as many
+ * rows as were appended, where the ordered compaction moves almost every row.
+ * kept_idx[u, g, j] is the position, before the call, of the row that sits at j
+ * afterwards: the same SET as ea_select_compact_inplace returns, in the new
+ * physical order (not ascending).  n_kept <= 25600 (EA_ERR_UNSUPPORTED beyond);
+ * needs the context's workspace (EA_ERR_WORKSPACE if smaller than
+ * ea_workspace_bytes(shape)).  Arguments as for ea_select_compact_inplace.
+ */
+ea_status ea_select_compact_inplace_unordered(ea_ctx* ctx, const ea_shape* shape,
+                                              const float* scores, int32_t n_kept, void* k, void* v,
+                                              int32_t* kept_idx, void* cuda_stream);
+
+/*
  * Streaming decode: one cache buffer and one window buffer carried through
  * consecutive compression events (the decoding set-up of the "Implementation
  * details" paragraph: a buffer of the most recent 128 states, compression

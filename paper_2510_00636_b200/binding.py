@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_select_compact_q8",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_select_compact_q8", "ea_select_compact_inplace_unordered",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.ea_n_floor.restype = i64
         L.ea_select_compact_inplace.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp]
         L.ea_select_compact_inplace.restype = ctypes.c_int
+        L.ea_select_compact_inplace_unordered.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp]
+        L.ea_select_compact_inplace_unordered.restype = ctypes.c_int
         L.ea_selftest_wait_timeout.argtypes = [vp, i32, vp]
         L.ea_selftest_wait_timeout.restype = ctypes.c_int
         L.ea_cache_append.argtypes = [vp, sp, vp, vp, vp, vp, i32, vp]
@@ -409,6 +411,21 @@ def ea_select_compact(ctx: Context, shape: Shape, scores, n_kept: int, k=None, v
                                    _ptr(v), _ptr(kept_idx), _ptr(k_out), _ptr(v_out),
                                    _stream(ctx.device)), "ea_select_compact")
     return kept_idx, k_out, v_out
+
+
+def ea_select_compact_inplace_unordered(ctx: Context, shape: Shape, scores, n_kept: int, k, v, kept_idx=None):
+    """Selection, then only the kept rows beyond ``n_kept`` move, into the evicted positions below it (in place).
+    Returns the position, before the call, of the row at each of the first ``n_kept`` positions afterwards."""
+    _dev_tensor(scores, torch.float32, "scores")
+    _dev_tensor(k, torch.bfloat16, "k")
+    _dev_tensor(v, torch.bfloat16, "v")
+    if kept_idx is None:
+        kept_idx = torch.empty((shape.n_units, shape.n_kv_heads, max(n_kept, 0)), dtype=torch.int32,
+                               device=scores.device)
+    _check(lib().ea_select_compact_inplace_unordered(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k),
+                                                     _ptr(v), _ptr(kept_idx), _stream(ctx.device)),
+           "ea_select_compact_inplace_unordered")
+    return kept_idx
 
 
 def ea_select_compact_inplace(ctx: Context, shape: Shape, scores, n_kept: int, k, v, kept_idx=None):

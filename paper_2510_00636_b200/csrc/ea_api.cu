@@ -427,6 +427,40 @@ ea_status ea_select_compact_inplace(ea_ctx* ctx, const ea_shape* shape, const fl
     return st;
 }
 
+ea_status ea_select_compact_inplace_unordered(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                                              int32_t n_kept, void* k, void* v, int32_t* kept_idx,
+                                              void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (n_kept < 0 || n_kept > shape->n_keys) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0 || n_kept == 0) return EA_OK;
+    if (!scores || !kept_idx || !k || !v) return EA_ERR_INVALID_ARG;
+    if (!aligned16(scores) || !aligned16(k) || !aligned16(v)) return EA_ERR_INVALID_ARG;
+    if (2 * (size_t)n_kept * sizeof(int32_t) > 200 * 1024) return EA_ERR_UNSUPPORTED;
+    {
+        const size_t bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) * shape->head_dim *
+                             sizeof(__nv_bfloat16);
+        const char* a = static_cast<const char*>(k);
+        const char* b = static_cast<const char*>(v);
+        if (a < b + bytes && b < a + bytes) return EA_ERR_INVALID_ARG;      // K and V are distinct buffers
+    }
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    if (ctx->workspace_bytes < plan.total) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // the ascending selection goes to the workspace (the log-score region: nothing of a compaction reads it)
+    int32_t* sel = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + plan.logits);
+    st = ea_launch_select(ctx, *shape, scores, n_kept, sel, stream);
+    if (st == EA_OK)
+        st = ea_launch_compact_fill(ctx, *shape, n_kept, sel, kept_idx, static_cast<__nv_bfloat16*>(k),
+                                    static_cast<__nv_bfloat16*>(v), stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
 ea_status ea_select_compact_adaptive(ea_ctx* ctx, const ea_shape* shape, const float* scores,
                                      int32_t n_kept, int32_t n_floor, const void* k, const void* v,
                                      int32_t* kept_idx, int32_t* head_offsets, void* k_out, void* v_out,

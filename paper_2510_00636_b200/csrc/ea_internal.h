@@ -180,6 +180,11 @@ ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* sc
 ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
                                     __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st);
 
+// Unordered variant: kept rows beyond n_kept fill the evicted positions below it; `sel` ascending kept positions
+// (scratch), `where` the original row at each position afterwards.
+ea_status ea_launch_compact_fill(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* sel,
+                                 int32_t* where, __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st);
+
 // Head-adaptive eviction: per-head counts and offsets from one radix search over the unit's scores,
 // then the per-head selection with those counts and a gather through the offsets.
 size_t ea_adaptive_ws_bytes(const ea_shape& s);

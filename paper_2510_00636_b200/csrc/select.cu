@@ -544,6 +544,61 @@ compact_inplace_kernel(const int32_t* __restrict__ kept_idx, int n, int n_kept, 
     }
 }
 
+// Unordered in-place compaction of one head of one tensor per CTA.  `sel` holds the head's kept positions
+// ascending.  Kept rows below n_kept stay; the kept rows at or beyond n_kept (the tail of `sel`) move, in
+// order, into the evicted positions below n_kept, in order.  Sources lie at or beyond n_kept and
+// destinations below it, so no move can disturb another.  where[j] = the original row now at j.
+constexpr int kFillThreads = 256;
+
+template <int D>
+__global__ void __launch_bounds__(kFillThreads)
+compact_fill_kernel(const int32_t* __restrict__ sel, int cap, int n_kept, int32_t* __restrict__ where, uint4* k,
+                    uint4* v) {
+    constexpr int LPR = D / 8;                         // 16-byte pieces per row
+    extern __shared__ int32_t fill_smem[];             // [n_kept] kept positions, then [n_kept] destinations of the movers
+    int32_t* a = fill_smem;
+    int32_t* dst_of = fill_smem + n_kept;
+    __shared__ int m_sh;
+    const long long head = blockIdx.x;
+    const int32_t* src_idx = sel + head * (long long)n_kept;
+    for (int j = threadIdx.x; j < n_kept; j += kFillThreads) a[j] = src_idx[j];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int lo = 0, hi = n_kept;                       // first j with a[j] >= n_kept: the rows before it stay
+        while (lo < hi) {
+            const int mid = (lo + hi) / 2;
+            if (a[mid] < n_kept) lo = mid + 1;
+            else hi = mid;
+        }
+        m_sh = lo;
+    }
+    __syncthreads();
+    const int m = m_sh;
+    for (int p = threadIdx.x; p < n_kept; p += kFillThreads) {
+        int lo = 0, hi = m;                            // kept positions below p
+        while (lo < hi) {
+            const int mid = (lo + hi) / 2;
+            if (a[mid] < p) lo = mid + 1;
+            else hi = mid;
+        }
+        const bool stays = lo < m && a[lo] == p;
+        int32_t w = p;
+        if (!stays) {
+            const int r = p - lo;                      // rank of this hole = rank of the mover that fills it
+            w = a[m + r];
+            dst_of[r] = p;
+        }
+        if (blockIdx.y == 0) where[head * (long long)n_kept + p] = w;
+    }
+    __syncthreads();
+    uint4* rows = (blockIdx.y == 0 ? k : v) + head * (long long)cap * LPR;
+    const int n_moves = n_kept - m;
+    for (int t = threadIdx.x; t < n_moves * LPR; t += kFillThreads) {
+        const int r = t / LPR, piece = t % LPR;
+        rows[(long long)dst_of[r] * LPR + piece] = rows[(long long)a[m + r] * LPR + piece];
+    }
+}
+
 }  // namespace
 
 static ea_status launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
@@ -694,5 +749,34 @@ ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_
         case 256: compact_inplace_kernel<256><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
         default: return EA_ERR_UNSUPPORTED;
     }
+    return EA_CHECK_LAUNCH();
+}
+
+ea_status ea_launch_compact_fill(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* sel,
+                                 int32_t* where, __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st) {
+    if (n_kept <= 0) return EA_OK;
+    const size_t smem = 2 * (size_t)n_kept * sizeof(int32_t);
+    if (smem > 200 * 1024) return EA_ERR_UNSUPPORTED;
+    const dim3 grid((unsigned)(s.n_units * s.n_kv_heads), 2);
+    uint4* k4 = reinterpret_cast<uint4*>(k);
+    uint4* v4 = reinterpret_cast<uint4*>(v);
+    const int cap = ea_kv_cap(s);
+    switch (s.head_dim) {
+        case 64:
+            EA_CUDA_TRY(cudaFuncSetAttribute(compact_fill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            compact_fill_kernel<64><<<grid, kFillThreads, smem, st>>>(sel, cap, n_kept, where, k4, v4);
+            break;
+        case 128:
+            EA_CUDA_TRY(cudaFuncSetAttribute(compact_fill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            compact_fill_kernel<128><<<grid, kFillThreads, smem, st>>>(sel, cap, n_kept, where, k4, v4);
+            break;
+        case 256:
+            EA_CUDA_TRY(cudaFuncSetAttribute(compact_fill_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            compact_fill_kernel<256><<<grid, kFillThreads, smem, st>>>(sel, cap, n_kept, where, k4, v4);
+            break;
+        default:
+            return EA_ERR_UNSUPPORTED;
+    }
+    ea_count_launches(ctx, 1);
     return EA_CHECK_LAUNCH();
 }

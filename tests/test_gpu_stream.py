@@ -251,3 +251,32 @@ def test_ring_statistics_partly_filled_and_wrapped(ea, oracle):
         assert (np.abs(sig - sig_r) / tot).max() < 1e-4, m
         np.testing.assert_allclose(mu.cpu().numpy(), mu_r, atol=2e-5 * (1 + np.abs(mu_r).max()))
         assert pushed.tolist() == [everything.shape[2]] * U
+
+
+@pytest.mark.parametrize("n,n_kept,d,cap", [(1, 1, 64, 0), (7, 3, 64, 9), (129, 129, 128, 0), (1000, 1, 128, 1000), (4608, 4096, 128, 4608),
+                                            (3001, 1500, 256, 3100), (30000, 25600, 64, 0)])
+def test_unordered_inplace_compaction_exact(ea, oracle, n, n_kept, d, cap):
+    """The unordered compaction against the oracle's index map: same kept set as the ordered selection, kept rows
+    below n_kept untouched, the others filled from the tail; rows at and beyond n_kept and everything outside
+    the heads' ranges are left alone."""
+    from oracle.ea_stream import fill_holes
+    torch.manual_seed(n)
+    U, Hkv = 2, 3
+    rows = cap or n
+    sc = torch.rand(U, Hkv, n, device="cuda")
+    sc[0, 0] = (sc[0, 0] * 4).floor() / 4               # many ties at the cut
+    sc[0, 1] = torch.arange(n, 0, -1, device="cuda")    # nothing moves
+    sc[1, 0] = torch.arange(n, device="cuda")           # everything kept sits in the tail
+    k = torch.randn(U, Hkv, rows, d, device="cuda").to(torch.bfloat16)
+    v = torch.randn(U, Hkv, rows, d, device="cuda").to(torch.bfloat16)
+    k0, v0 = inputs.bits(k), inputs.bits(v)
+    shape = ea.make_shape(U, Hkv, Hkv, d, n, 1, kv_capacity=cap)
+    ctx = ea.Context.for_shape(shape)
+    where = ea.ea_select_compact_inplace_unordered(ctx, shape, sc, n_kept, k, v)
+    ctx.sync_status()
+    want = fill_holes(oracle.select(sc.cpu().numpy().astype(np.float64), n_kept), n_kept)
+    assert np.array_equal(where.cpu().numpy(), want)
+    k1, v1 = inputs.bits(k), inputs.bits(v)
+    assert np.array_equal(k1[:, :, :n_kept], oracle.gather(k0[:, :, :n], want))
+    assert np.array_equal(v1[:, :, :n_kept], oracle.gather(v0[:, :, :n], want))
+    assert np.array_equal(k1[:, :, n_kept:], k0[:, :, n_kept:]) and np.array_equal(v1[:, :, n_kept:], v0[:, :, n_kept:])

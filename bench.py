@@ -245,9 +245,10 @@ class DecodeWorkload:
     by the previous step: synthetic rows of the same distribution)."""
 
     def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False,
-                 unordered: bool = False):
+                 unordered: bool = False, fused: bool = False):
         import dataclasses
         self.cfg, self.device, self.ea = cfg, device, ea
+        self.fused = fused                  # ea_set_fused_stats: no sigma_bar round trip, no image kernel
         self.unordered = unordered          # ea_select_compact_inplace_unordered: only the tail's kept rows move
         self.use_graph, self.graphs = use_graph, {}
         self.events = inputs.decode_schedule()
@@ -290,7 +291,9 @@ class DecodeWorkload:
                                   kv_capacity=self.cap)
 
     def make_ctx(self, units_per_call):
-        return self.ea.Context.for_shape(self._shape(self.cap), self.device.index)
+        ctx = self.ea.Context.for_shape(self._shape(self.cap), self.device.index)
+        ctx.set_fused_stats(self.fused)
+        return ctx
 
     def _event(self, ctx, n, kept, ph, pos):
         ea, cfg = self.ea, self.cfg
@@ -299,8 +302,13 @@ class DecodeWorkload:
         idx = self.idx.view(-1)[:self.n_units * cfg.n_kv_heads * kept].view(self.n_units, cfg.n_kv_heads, kept)
         ea.ea_cache_append(ctx, self._shape(n - self.every), self.k, self.v, self.new_k[ph], self.new_v[ph])
         ea.ea_window_push(ctx, shape, self.ring, self.pushed, self.new_q[ph])
-        ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
-        ea.ea_score(ctx, shape, self.k, self.v, self.mu, self.sigma, cfg.eps, scores)
+        if self.fused:
+            ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu,
+                                   want_sigma=False)
+            ea.ea_score(ctx, shape, self.k, self.v, None, None, cfg.eps, scores)
+        else:
+            ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
+            ea.ea_score(ctx, shape, self.k, self.v, self.mu, self.sigma, cfg.eps, scores)
         compact = ea.ea_select_compact_inplace_unordered if self.unordered else ea.ea_select_compact_inplace
         compact(ctx, shape, scores, kept, self.k, self.v, idx)
 
@@ -457,7 +465,7 @@ def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_work
         gc.collect()
         torch.cuda.empty_cache()
     decode = cfg.cfg_id == 4
-    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph, unordered=args.unordered) if decode else Workload(cfg, device, ea, args.head_adaptive,
+    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph, unordered=args.unordered, fused=args.fused_stats) if decode else Workload(cfg, device, ea, args.head_adaptive,
                                                                  args.hidden_stats, args.with_wo, args.kv_dtype == "fp8")
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
@@ -573,6 +581,9 @@ def main():
     ap.add_argument("--unordered", action="store_true",
                     help="decode config: compact with ea_select_compact_inplace_unordered (kept rows of the tail fill "
                          "the evicted positions; the cache loses its temporal order, not its contents)")
+    ap.add_argument("--fused-stats", action="store_true",
+                    help="decode config: the statistics kernel writes the log-score kernel's operand itself "
+                         "(ea_set_fused_stats): no sigma_bar round trip, no image kernel")
     ap.add_argument("--kv-dtype", default="bf16", choices=["bf16", "fp8"],
                     help="prefill configs: cache held as FP8 E4M3 codes with scales (ea_score_q8, ea_select_compact_q8); "
                          "the device-resident line only, with the algorithmic bytes of that format")
@@ -633,6 +644,7 @@ def main():
     if cfg.cfg_id == 4:
         result["config"]["cache"] = "one carried buffer per sequence, compacted in place (%s), 512 pairs appended per event" % (
             "unordered: the tail's kept rows fill the evicted positions" if args.unordered else "temporal order kept")
+        result["config"]["fused_statistics"] = bool(args.fused_stats)
 
     # end to end from host buffers through ea_compress_host (rank-local; max over ranks)
     if not args.skip_e2e:
@@ -652,10 +664,10 @@ def main():
                                  "kernel_frac": om["roofline"]["frac"], "kernel_ms": om["roofline"]["kernel_ms"],
                                  "kernel_mcycles": om["roofline"]["kernel_mcycles"], "sm_mhz": om["clocks"]["sm_mhz"],
                                  "gpu_launches": om["gpu_launches"]}
-        args.unordered = True
+        args.unordered = args.fused_stats = True
         om = measure(args, inputs.CONFIGS[4], ea, device, world, local, peaks, max(5, args.steps // 2), 3, keep_workload=False)
-        args.unordered = False
-        others[inputs.CONFIGS[4].name]["unordered_compaction"] = {
+        args.unordered = args.fused_stats = False
+        others[inputs.CONFIGS[4].name]["unordered_compaction_fused_statistics"] = {
             "ms_per_step": om["ms"], "value": om["slots"] / (om["ms"] * 1e-3) / 1e9,
             "path_roofline_frac": om["path_roofline"]["frac"]}
         result["other_configs"] = others

@@ -445,6 +445,26 @@ int64_t ea_n_floor(int64_t n_kept, double safeguard);
 ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms);
 
 /*
+ * Fused statistics (the paper has no counterpart; a shortcut for the streaming
+ * path, where a compression event scores a few thousand keys for thousands of
+ * query heads and preparing the tensor-core operand from sigma_bar is a
+ * noticeable part of it).  With on != 0, ea_query_stats and
+ * ea_query_stats_ring also write, straight from their accumulators, the bf16
+ * operand that ea_score's tensor-core kernel would otherwise build from
+ * mu_bar and sigma_bar, into the context's workspace; a following
+ *     ea_score(ctx, shape, k, v, NULL, NULL, ...)
+ * on the SAME context with the SAME shape (every field but `window`) uses it
+ * and needs neither array.  In this mode sigma_bar may be NULL in the statistics
+ * call (mu_bar is still written).  The scores are bit for bit those of the
+ * two-step path.  Conditions: head_dim 64 or 128, n_keys >= 128, group mode
+ * not EA_GROUP_MEAN_LOGIT, workspace of ea_workspace_bytes(shape); otherwise
+ * the statistics call behaves as without the flag (and then needs sigma_bar),
+ * and ea_score with NULL statistics returns EA_ERR_INVALID_ARG.  Any later
+ * statistics call of the context replaces the operand.
+ */
+ea_status ea_set_fused_stats(ea_ctx* ctx, int32_t on);
+
+/*
  * Runs the value-norm pass of ea_score (the ||v|| of Eq. 9, which does not
  * depend on the log-scores) on n_sms SMs of its own, beside the tensor-bound
  * log-score kernel instead of after it (the paper has no counterpart): a

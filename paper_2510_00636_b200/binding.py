@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_select_compact_q8", "ea_select_compact_inplace_unordered",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_select_compact_q8", "ea_select_compact_inplace_unordered",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.ea_score_q8.argtypes = [vp, sp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp]
         L.ea_select_compact_q8.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.ea_score_q8.restype = L.ea_select_compact_q8.restype = ctypes.c_int
+        L.ea_set_fused_stats.argtypes = [vp, i32]
+        L.ea_set_fused_stats.restype = ctypes.c_int
         L.ea_set_sm_budget.argtypes = [vp, i32]
         L.ea_set_side_sms.argtypes = [vp, i32]
         L.ea_set_side_sms.restype = ctypes.c_int
@@ -198,6 +200,11 @@ class Context:
         """Run the value-norm pass of ``ea_score`` on ``n_sms`` SMs beside the log-score kernel (0: off)."""
         _check(lib().ea_set_side_sms(self._h, int(n_sms)), "ea_set_side_sms")
 
+    def set_fused_stats(self, on: bool = True):
+        """Statistics calls also write the log-score kernel's operand; ``ea_score`` may then be called without
+        ``mu_bar`` / ``sigma_bar`` (see ``ea_set_fused_stats``)."""
+        _check(lib().ea_set_fused_stats(self._h, int(bool(on))), "ea_set_fused_stats")
+
     def profile_begin(self):
         _check(lib().ea_profile_begin(self._h), "ea_profile_begin")
 
@@ -210,14 +217,15 @@ class Context:
 
 
 def ea_query_stats(ctx: Context, shape: Shape, q_win, pos_next, n_future: int, rope_base: float,
-                   mu_bar=None, sigma_bar=None):
-    """q_win bf16 [U,Hq,W,d], pos_next int64 [U] (device) -> (mu_bar [U,Hq,d], sigma_bar [U,Hq,d,d])."""
+                   mu_bar=None, sigma_bar=None, want_sigma: bool = True):
+    """q_win bf16 [U,Hq,W,d], pos_next int64 [U] (device) -> (mu_bar [U,Hq,d], sigma_bar [U,Hq,d,d]).
+    ``want_sigma=False`` (fused statistics only) leaves sigma_bar out: returns (mu_bar, None)."""
     _dev_tensor(q_win, torch.bfloat16, "q_win")
     _dev_tensor(pos_next, torch.int64, "pos_next")
     U, Hq, d = shape.n_units, shape.n_q_heads, shape.head_dim
     if mu_bar is None:
         mu_bar = torch.empty((U, Hq, d), dtype=torch.float32, device=q_win.device)
-    if sigma_bar is None:
+    if sigma_bar is None and want_sigma:
         sigma_bar = torch.empty((U, Hq, d, d), dtype=torch.float32, device=q_win.device)
     _check(lib().ea_query_stats(ctx._h, ctypes.byref(shape), _ptr(q_win), _ptr(pos_next), int(n_future),
                                 float(rope_base), _ptr(mu_bar), _ptr(sigma_bar), _stream(ctx.device)),
@@ -244,7 +252,7 @@ def ea_window_push(ctx: Context, shape: Shape, q_ring, ring_pushed, q_new):
 
 
 def ea_query_stats_ring(ctx: Context, shape: Shape, q_ring, ring_pushed, pos_next, n_future: int, rope_base: float,
-                        mu_bar=None, sigma_bar=None):
+                        mu_bar=None, sigma_bar=None, want_sigma: bool = True):
     """``ea_query_stats`` over the rows a window ring holds -> (mu_bar, sigma_bar)."""
     _dev_tensor(q_ring, torch.bfloat16, "q_ring")
     _dev_tensor(ring_pushed, torch.int64, "ring_pushed")
@@ -252,7 +260,7 @@ def ea_query_stats_ring(ctx: Context, shape: Shape, q_ring, ring_pushed, pos_nex
     U, Hq, d = shape.n_units, shape.n_q_heads, shape.head_dim
     if mu_bar is None:
         mu_bar = torch.empty((U, Hq, d), dtype=torch.float32, device=q_ring.device)
-    if sigma_bar is None:
+    if sigma_bar is None and want_sigma:
         sigma_bar = torch.empty((U, Hq, d, d), dtype=torch.float32, device=q_ring.device)
     _check(lib().ea_query_stats_ring(ctx._h, ctypes.byref(shape), _ptr(q_ring), _ptr(ring_pushed), _ptr(pos_next),
                                      int(n_future), float(rope_base), _ptr(mu_bar), _ptr(sigma_bar),
@@ -306,8 +314,9 @@ def ea_score(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, epsilon: float
     """k, v bf16 [U,Hkv,n,d] -> scores fp32 [U,Hkv,n] (and the log-scores [U,Hq,n] if asked)."""
     _dev_tensor(k, torch.bfloat16, "k")
     _dev_tensor(v, torch.bfloat16, "v")
-    _dev_tensor(mu_bar, torch.float32, "mu_bar")
-    _dev_tensor(sigma_bar, torch.float32, "sigma_bar")
+    if sigma_bar is not None:                       # (None, None): the operand of a fused statistics call
+        _dev_tensor(mu_bar, torch.float32, "mu_bar")
+        _dev_tensor(sigma_bar, torch.float32, "sigma_bar")
     U, Hq, Hkv, n = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys
     if scores is None:
         scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=k.device)

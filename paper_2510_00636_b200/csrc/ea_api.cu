@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument validation, workspace planning, context
 // lifetime, and the order of kernel launches of each call.
 #include <stdio.h>
+#include <string.h>
 
 #include <new>
 
@@ -30,6 +31,22 @@ ea_status check_shape(const ea_shape* s) {
 thread_local char g_last_cuda_error[192] = "";
 
 }  // namespace
+
+// Fused statistics: where the images of `s` go, or nullptr when this call does not write them.
+bool ea_fused_image_target(ea_ctx* ctx, const ea_shape& s, void** image, float** vec) {
+    *image = nullptr;
+    *vec = nullptr;
+    ctx->image_ready = false;                          // whatever the workspace held is stale after a statistics call
+    if (!ctx->fused_stats) return true;
+    if (s.head_dim > 128 || !ea_mma_path_supported(s) || s.group_mode == EA_GROUP_MEAN_LOGIT) return true;
+    const ea_ws_plan plan = ea_plan_workspace(s);
+    if (ctx->workspace_bytes < plan.total) return false;
+    *image = static_cast<char*>(ctx->workspace) + plan.image;
+    *vec = reinterpret_cast<float*>(static_cast<char*>(ctx->workspace) + plan.vec);
+    ctx->image_ready = true;
+    ctx->image_shape = s;
+    return true;
+}
 
 void ea_note_cuda_error(cudaError_t err, const char* file, int line) {
     const char* base = file;
@@ -111,6 +128,8 @@ ea_status ea_create(ea_ctx** out_ctx, int device, size_t workspace_bytes) {
     ctx->sm_budget = ctx->sm_count;
     ctx->side_sms = 0;
     ctx->side_ready = false;
+    ctx->fused_stats = false;
+    ctx->image_ready = false;
     ctx->workspace = nullptr;
     ctx->workspace_bytes = workspace_bytes;
     ctx->status_host = nullptr;
@@ -184,19 +203,24 @@ ea_status ea_query_stats(ea_ctx* ctx, const ea_shape* shape, const void* q_win,
     ea_status st = check_shape(shape);
     if (st != EA_OK) return st;
     if (shape->n_units == 0) return EA_OK;
-    if (!q_win || !pos_next || !mu_bar || !sigma_bar) return EA_ERR_INVALID_ARG;
+    if (!q_win || !pos_next || !mu_bar) return EA_ERR_INVALID_ARG;
     if (!aligned16(q_win) || !aligned16(mu_bar) || !aligned16(sigma_bar)) return EA_ERR_INVALID_ARG;
     if (n_future < 1 || !(rope_base > 0.0)) return EA_ERR_INVALID_ARG;
     if (shape->window < 1 || (shape->cov_norm == EA_COV_SAMPLE && shape->window < 2))
         return EA_ERR_INVALID_ARG;
     const ea_ws_plan plan = ea_plan_workspace(*shape);
     if (ctx->workspace_bytes < plan.logits /* rope_coef region only */) return EA_ERR_WORKSPACE;
+    void* image = nullptr;
+    float* vec = nullptr;
+    if (!ea_fused_image_target(ctx, *shape, &image, &vec)) return EA_ERR_WORKSPACE;
+    if (!sigma_bar && !image) return EA_ERR_INVALID_ARG;       // sigma_bar may only be left out in fused mode
     int prev = 0;
     EA_CUDA_TRY(cudaGetDevice(&prev));
     if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
     float* coef = reinterpret_cast<float*>(static_cast<char*>(ctx->workspace) + plan.rope_coef);
     st = ea_launch_stats(ctx, *shape, static_cast<const __nv_bfloat16*>(q_win), pos_next, n_future,
-                         rope_base, coef, mu_bar, sigma_bar, static_cast<cudaStream_t>(cuda_stream));
+                         rope_base, coef, mu_bar, sigma_bar, static_cast<cudaStream_t>(cuda_stream), image, vec);
+    if (st != EA_OK) ctx->image_ready = false;
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }
@@ -242,7 +266,17 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     ea_status st = check_shape(shape);
     if (st != EA_OK) return st;
     if (shape->n_units == 0 || shape->n_keys == 0) return EA_OK;
-    if (!k || !v || !mu_bar || !sigma_bar || !scores) return EA_ERR_INVALID_ARG;
+    if (!k || !v || !scores) return EA_ERR_INVALID_ARG;
+    // sigma_bar == NULL: the images the last statistics call of this context wrote for this very shape
+    // (ea_set_fused_stats) stand in for mu_bar and sigma_bar
+    const bool from_image = sigma_bar == nullptr;
+    if (from_image) {
+        ea_shape a = *shape, b = ctx->image_shape;
+        a.window = b.window = 0;                                // the window length does not shape the images
+        if (!ctx->image_ready || memcmp(&a, &b, sizeof(ea_shape)) != 0) return EA_ERR_INVALID_ARG;
+    } else if (!mu_bar) {
+        return EA_ERR_INVALID_ARG;
+    }
     if (!aligned16(k) || !aligned16(v) || !aligned16(mu_bar) || !aligned16(sigma_bar) ||
         !aligned16(scores) || !aligned16(logits_opt))
         return EA_ERR_INVALID_ARG;
@@ -258,7 +292,7 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
     const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
-    const ea_quad_form eq7 = ea_eq7_form(*shape, mu_bar, sigma_bar);
+    const ea_quad_form eq7 = ea_eq7_form(*shape, from_image ? nullptr : mu_bar, sigma_bar);
     if (ea_mma_path_supported(*shape) && shape->group_mode != EA_GROUP_MEAN_LOGIT) {
         // tensor-core log-scores with the log-sum-exp partials from their epilogue
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
@@ -517,6 +551,13 @@ ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms) {
     if (n_sms == 0) n_sms = ctx->sm_count;
     if (n_sms < 2 || n_sms > ctx->sm_count) return EA_ERR_INVALID_ARG;
     ctx->sm_budget = n_sms;
+    return EA_OK;
+}
+
+ea_status ea_set_fused_stats(ea_ctx* ctx, int32_t on) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ctx->fused_stats = on != 0;
+    ctx->image_ready = false;
     return EA_OK;
 }
 

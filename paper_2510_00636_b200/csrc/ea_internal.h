@@ -14,6 +14,9 @@ struct ea_ctx {
     int device;
     int sm_count;        // SMs of the device
     int sm_budget;       // SMs the persistent kernels of this context may occupy (ea_set_sm_budget)
+    bool fused_stats;    // ea_set_fused_stats: the statistics calls also write the covariance images
+    bool image_ready;    // the workspace holds the images of `image_shape`, written by the last statistics call
+    ea_shape image_shape;
     int side_sms;        // SMs of the value-norm pass that runs beside the log-score kernel (0: no side pass)
     bool side_ready;     // side stream and events exist
     cudaStream_t st_side;
@@ -87,14 +90,22 @@ static inline size_t ea_align_up(size_t x, size_t a) { return (x + a - 1) / a * 
 static inline int ea_kv_cap(const ea_shape& s) { return s.kv_capacity > 0 ? s.kv_capacity : s.n_keys; }
 
 // ---- launchers (each returns EA_OK or EA_ERR_CUDA from cudaGetLastError) ----
+// image / vec != nullptr (head_dim <= 128 only): also write the log-score kernel's covariance images; sigma_bar
+// may then be nullptr.
 ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
                           const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
-                          float* mu_bar, float* sigma_bar, cudaStream_t st);
+                          float* mu_bar, float* sigma_bar, cudaStream_t st, void* image = nullptr,
+                          float* vec = nullptr);
 
 // The same statistics over a ring of window rows: pushed[u] rows written so far, at most s.window of them valid.
 ea_status ea_launch_stats_ring(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_ring,
                                const int64_t* pushed, const int64_t* pos_next, int n_future, double rope_base,
-                               float* rope_coef, float* mu_bar, float* sigma_bar, cudaStream_t st);
+                               float* rope_coef, float* mu_bar, float* sigma_bar, cudaStream_t st,
+                               void* image = nullptr, float* vec = nullptr);
+
+// Fused statistics (ea_set_fused_stats): the workspace addresses the images of `s` go to, or nullptr when this
+// statistics call does not write them; false if the workspace is too small for them.
+bool ea_fused_image_target(ea_ctx* ctx, const ea_shape& s, void** image, float** vec);
 
 // What the log-score kernels evaluate per (query head h, row x of the KV head it reads):
 //   lin_scale * lin_h . x + quad_scale * x^T quad_h x
@@ -135,6 +146,7 @@ bool ea_mma_path_supported(const ea_shape& s);
 size_t ea_mma_image_bytes(const ea_shape& s);
 size_t ea_mma_vec_bytes(const ea_shape& s);
 size_t ea_mma_lse_part_bytes(const ea_shape& s);
+// form.quad == nullptr: the images in `image` / `vec` are already there (fused statistics)
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                const ea_quad_form& form, void* image, float* vec,
                                float* logits, float* lse_part, int* n_chunks, cudaStream_t st);

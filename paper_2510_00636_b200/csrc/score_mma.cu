@@ -34,6 +34,7 @@
 #include <mutex>
 
 #include "ea_internal.h"
+#include "image_layout.cuh"
 #include "ptx_sm100.cuh"
 
 namespace {
@@ -47,11 +48,12 @@ constexpr int kChunkA = kTileKeys * 128;           // bytes of one 64-channel ch
 
 template <int D, bool PAIR>
 struct Geo {
-    static constexpr int HPC = 256 / D;                  // query heads per pass (1, 2 or 4)
-    static constexpr int KCH = D / 64;                   // 64-channel (128-byte) chunks per row
-    static constexpr int IMG_ROWS = HPC * D;             // rows of a whole image (accumulator columns)
-    static constexpr int CHUNK_B_FULL = IMG_ROWS * 128;  // bytes of one chunk of a whole image (global)
-    static constexpr int IMG_MAIN = KCH * CHUNK_B_FULL;  // bytes of the covariance part of a whole image (global)
+    using L = EaImage<D>;                                // the image's layout in global memory
+    static constexpr int HPC = L::HPC;
+    static constexpr int KCH = L::KCH;
+    static constexpr int IMG_ROWS = L::IMG_ROWS;
+    static constexpr int CHUNK_B_FULL = L::CHUNK_B_FULL;
+    static constexpr int IMG_MAIN = L::IMG_MAIN;
     static constexpr int ROWS_CTA = PAIR ? IMG_ROWS / 2 : IMG_ROWS;   // image rows one CTA keeps
     static constexpr int CHUNK_B = ROWS_CTA * 128;
     static constexpr int IMG_CTA = KCH * CHUNK_B;
@@ -65,22 +67,13 @@ struct Geo {
     // linear term: one extra K = 16 MMA step, a constant block of ones times (hi, lo) of mu' per column,
     // both as unswizzled K-major core matrices (8 rows x 16 bytes; 128 bytes on along K, 256 on along rows)
     static constexpr int ONES = kTileKeys * 32;
-    static constexpr int LIN_FULL = IMG_ROWS * 32;       // bytes of the mu' operand of a whole image (global)
+    static constexpr int LIN_FULL = L::LIN_FULL;
     static constexpr int LIN_CTA = ROWS_CTA * 32;
-    // At d <= 128 the epilogue is the limit, so the diagonal goes to the tensor cores as well: its bf16
-    // part sits on the image's diagonal, and the bf16 rounding of what that leaves is added by one
-    // M128 N16 K16 step per (head, 16 channels) against a 16 x 16 diagonal block (unswizzled core
-    // matrices, 512 bytes).  At d = 256 the diagonal stays in fp32 in the epilogue.
-    static constexpr bool DIAG_MMA = D <= 128;
-    static constexpr int DIAG_BLOCK = 16 * HPC * 32;                    // bytes: 16 HPC rows x 16 bf16
-    static constexpr int DIAG_FULL = DIAG_MMA ? (D / 16) * DIAG_BLOCK : 0;   // per whole image
-    // Accumulator column (= image row) of channel c of head j.  With the diagonal blocks the heads are
-    // interleaved in runs of 16 channels, so that the 16 channels of one MMA step are 16 HPC adjacent
-    // columns and every head's share of the diagonal is added by one instruction per step.
-    __host__ __device__ static constexpr int col(int j, int c) {
-        return DIAG_MMA ? (c / 16) * (16 * HPC) + j * 16 + c % 16 : j * D + c;
-    }
-    static constexpr int IMG_FULL = IMG_MAIN + LIN_FULL + DIAG_FULL;   // bytes of a whole image (global)
+    static constexpr bool DIAG_MMA = L::DIAG_MMA;
+    static constexpr int DIAG_BLOCK = L::DIAG_BLOCK;
+    static constexpr int DIAG_FULL = L::DIAG_FULL;
+    __host__ __device__ static constexpr int col(int j, int c) { return L::col(j, c); }
+    static constexpr int IMG_FULL = L::IMG_FULL;
     // partial sums of the column parts: [tile parity][part][head][key]
     static constexpr int PART = 2 * EPI_PARTS * HPC * kTileKeys * (int)sizeof(float);
     static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
@@ -719,7 +712,8 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     CUtensorMap k_map;
     if (!make_k_map(&k_map, k, D, s.n_keys, ea_kv_cap(s), (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
 
-    sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(form, s.n_q_heads, s.n_kv_heads, image, vec);
+    if (form.quad)
+        sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(form, s.n_q_heads, s.n_kv_heads, image, vec);
     auto kern = logits_mma_kernel<D, PAIR>;
     EA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
     const long long want = (long long)p.n_groups * p.n_subsets;
@@ -735,7 +729,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    ea_count_launches(ctx, 2);
+    ea_count_launches(ctx, form.quad ? 2 : 1);
     cudaEvent_t stop = ea_profile_mark_start(ctx, st);
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, k_map, p);
     ea_profile_mark_stop(ctx, stop, st);

@@ -9,6 +9,7 @@
 //   Sigma_bar = (1/N) sum_w x_w x_w^T,  x_w = R_bar (u_w - mu),
 // which equals R_bar Sigma R_bar^T.  Tensor cores on a bf16 (hi, lo) pair of x, fp32 accumulation.
 #include "ea_internal.h"
+#include "image_layout.cuh"
 
 namespace {
 
@@ -51,6 +52,17 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Fused mode (ea_set_fused_stats): the statistics kernel also writes, from its accumulators, the bf16
+// covariance image that the log-score kernel loads (what sigma_image_kernel would build from sigma_bar),
+// so that ea_score needs neither that kernel nor sigma_bar.  image == nullptr: off.
+struct StatsImage {
+    uint8_t* image;      // images of the call, one per (unit, KV head, head subset)
+    float* vec;          // fp32 [units * Hq, d] diagonals
+    int Hkv;
+    float lin_scale;     // 1 / sqrt(d)
+    float quad_scale;    // 1 / (2 d)
+};
+
 template <int D, typename QT>
 constexpr int stats_smem_bytes() {
     constexpr int BM = D < 128 ? D : 128;
@@ -65,7 +77,7 @@ template <int D, typename QT>
 __global__ void __launch_bounds__(256)
 stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
                  int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar,
-                 int w_cap, const long long* __restrict__ pushed, int cov_sample) {
+                 int w_cap, const long long* __restrict__ pushed, int cov_sample, const StatsImage img) {
     constexpr int HALF = D / 2;
     constexpr int BM = D < 128 ? D : 128;          // block edge
     constexpr int NB1 = D / BM;                    // blocks per edge (1 or 2)
@@ -96,19 +108,10 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
     if (pushed) {
         const long long p = pushed[u];
         W = p < (long long)w_cap ? (int)p : w_cap;
-        if (W < 1 + cov_sample) {
-            // nothing to estimate from: zero statistics (uniform expected attention)
-            if (blockIdx.y == 0)
-                for (int c = tid; c < D; c += 256) mu_bar[(size_t)uh * D + c] = 0.f;
-            const int r0 = NB1 == 1 ? 0 : (blockIdx.y == 2 ? BM : 0), c0 = NB1 == 1 ? 0 : (blockIdx.y == 0 ? 0 : BM);
-            for (int e = tid; e < BM * BM; e += 256) {
-                const int a = r0 + e / BM, c = c0 + e % BM;
-                sigma_bar[(size_t)uh * D * D + (size_t)a * D + c] = 0.f;
-                sigma_bar[(size_t)uh * D * D + (size_t)c * D + a] = 0.f;
-            }
-            return;
-        }
-        inv_norm = 1.0f / (float)(W - cov_sample);
+        // nothing to estimate from: zero statistics (uniform expected attention); the loops below then run
+        // over no rows and every output is written as zero
+        if (W < 1 + cov_sample) { W = 0; inv_norm = 0.f; }
+        else         inv_norm = 1.0f / (float)(W - cov_sample);
     }
     const QT* q = q_win + (size_t)uh * w_cap * D;
 
@@ -144,7 +147,7 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
             float acc = 0.f;
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg) acc += red[gg * D + c];      // fixed order
-            mu_s[c] = acc / (float)W;
+            mu_s[c] = W > 0 ? acc / (float)W : 0.f;
         }
     }
     __syncthreads();
@@ -153,8 +156,11 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
             const int a = layout == EA_ROPE_INTERLEAVED ? 2 * m : m;
             const int b = layout == EA_ROPE_INTERLEAVED ? 2 * m + 1 : m + HALF;
             const float ma = mu_s[a], mb = mu_s[b];
-            mu_bar[(size_t)uh * D + a] = c_s[m] * ma - s_s[m] * mb;
-            mu_bar[(size_t)uh * D + b] = s_s[m] * ma + c_s[m] * mb;
+            const float ra = c_s[m] * ma - s_s[m] * mb, rb = s_s[m] * ma + c_s[m] * mb;
+            mu_bar[(size_t)uh * D + a] = ra;
+            mu_bar[(size_t)uh * D + b] = rb;
+            red[a] = ra;                       // (the mean's partial sums are no longer needed) for the fused image
+            red[b] = rb;
         }
     }
 
@@ -245,21 +251,92 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
     }
 
     // upper triangle from the accumulators, lower triangle as its mirror
-    float* out = sigma_bar + (size_t)uh * D * D;
+    if (sigma_bar) {
+        float* out = sigma_bar + (size_t)uh * D * D;
 #pragma unroll
-    for (int i = 0; i < TM; ++i)
+        for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < TN; ++j)
+            for (int j = 0; j < TN; ++j)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int a = bi * BM + wm * WM + i * 16 + lane / 4 + 8 * (e / 2);
-                const int c = bj * BM + wn * WN + j * 8 + 2 * (lane % 4) + (e % 2);
-                if (a <= c) {
-                    const float v = acc[i][j][e] * inv_norm;
-                    out[(size_t)a * D + c] = v;
-                    out[(size_t)c * D + a] = v;
+                for (int e = 0; e < 4; ++e) {
+                    const int a = bi * BM + wm * WM + i * 16 + lane / 4 + 8 * (e / 2);
+                    const int c = bj * BM + wn * WN + j * 8 + 2 * (lane % 4) + (e % 2);
+                    if (a <= c) {
+                        const float v = acc[i][j][e] * inv_norm;
+                        out[(size_t)a * D + c] = v;
+                        out[(size_t)c * D + a] = v;
+                    }
                 }
+    }
+    if constexpr (NB1 == 1) {
+        if (img.image) {
+            // ---- the covariance image of this head, bit for bit what sigma_image_kernel builds from sigma_bar
+            using L = EaImage<D>;
+            const int h = uh % Hq, Gq = Hq / img.Hkv;
+            const int g = h / Gq, hg = h % Gq;
+            const int n_subsets = (Gq + L::HPC - 1) / L::HPC;
+            const int hs = hg / L::HPC, jh = hg % L::HPC;
+            uint8_t* gimg = img.image + ((size_t)(u * img.Hkv + g) * n_subsets + hs) * L::IMG_FULL;
+            __syncthreads();                              // the staging buffers of the main loop are dead
+            // tile[kc][c][128 bytes]: this head's rows in channel order, swizzled as in the image (the image
+            // row of channel c has the same low three bits as c)
+            uint8_t* tile = stats_smem;
+            float* dg_s = red + D;                         // [D] diagonal of Sigma_bar / (2 d)
+            auto at = [&](int r, int k) {
+                return reinterpret_cast<__nv_bfloat16*>(tile + (k / 64) * (D * 128) + r * 128 +
+                                                        ((((k % 64) / 8) ^ (r & 7)) << 4) + (k % 8) * 2);
+            };
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int a = wm * WM + i * 16 + lane / 4 + 8 * (e / 2);
+                        const int c = wn * WN + j * 8 + 2 * (lane % 4) + (e % 2);
+                        const float v = acc[i][j][e] * inv_norm;
+                        if (a < c) {
+                            // the two mirrored entries together carry (S_ca + S_ac) / (2 d), split into a bf16
+                            // and the bf16 rounding of its remainder
+                            const float x = (v + v) * img.quad_scale;
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                            *at(c, a) = hi;
+                            *at(a, c) = __float2bfloat16_rn(x - __bfloat162float(hi));
+                        } else if (a == c) {
+                            const float dg = v * img.quad_scale;
+                            *at(c, c) = __float2bfloat16_rn(dg);     // its bf16 part; the rest in the diagonal blocks
+                            dg_s[c] = dg;
+                        }
+                    }
+            __syncthreads();
+            for (int e = tid; e < L::KCH * D * 8; e += 256) {
+                const int piece = e % 8, c = (e / 8) % D, kc = e / (8 * D);
+                const uint4 x = *reinterpret_cast<const uint4*>(tile + kc * (D * 128) + c * 128 + piece * 16);
+                *reinterpret_cast<uint4*>(gimg + (size_t)kc * L::CHUNK_B_FULL + (size_t)L::col(jh, c) * 128 + piece * 16) = x;
             }
+            // linear-term operand, diagonal vector and diagonal blocks (as sigma_image_kernel writes them)
+            for (int c = tid; c < D; c += 256) {
+                const float m = red[c] * img.lin_scale;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(m);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(m - __bfloat162float(hi));
+                const int row = L::col(jh, c);
+                uint8_t* dst = gimg + L::IMG_MAIN + (size_t)(row / 8) * 256 + (row % 8) * 16;
+                *reinterpret_cast<uint4*>(dst) =
+                    make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
+                const float dg = dg_s[c];
+                img.vec[(size_t)uh * D + c] = dg;
+                const __nv_bfloat16 dlo = __float2bfloat16_rn(dg - __bfloat162float(__float2bfloat16_rn(dg)));
+                const int kk = c % 16, n = 16 * jh + kk;
+                uint8_t* blk = gimg + L::IMG_MAIN + L::LIN_FULL + (size_t)(c / 16) * L::DIAG_BLOCK + (n / 8) * 256 + (n % 8) * 16;
+                uint32_t w4[4] = {0u, 0u, 0u, 0u};
+                w4[(kk % 8) / 2] = (uint32_t)__bfloat16_as_ushort(dlo) << (16 * (kk % 2));
+                const uint4 mine = make_uint4(w4[0], w4[1], w4[2], w4[3]), zero = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(blk) = kk < 8 ? mine : zero;
+                *reinterpret_cast<uint4*>(blk + 128) = kk < 8 ? zero : mine;
+            }
+        }
+    }
 }
 
 }  // namespace
@@ -267,7 +344,8 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
 template <typename QT>
 static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_win, const int64_t* pos_next,
                               int n_future, double rope_base, float* rope_coef, float* mu_bar, float* sigma_bar,
-                              cudaStream_t st, const int64_t* pushed = nullptr) {
+                              cudaStream_t st, const int64_t* pushed = nullptr, void* image = nullptr,
+                              float* vec = nullptr) {
     const int d = s.head_dim, half = d / 2;
     const int n_coef = s.n_units * half;
     rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, st>>>(pos_next, s.n_units, half, d, n_future,
@@ -275,6 +353,7 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
     const float inv_norm =
         1.0f / (float)(s.cov_norm == EA_COV_SAMPLE ? s.window - 1 : s.window);
     const unsigned heads = (unsigned)(s.n_units * s.n_q_heads);
+    const StatsImage img = {static_cast<uint8_t*>(image), vec, s.n_kv_heads, 1.0f / sqrtf((float)d), 0.5f / (float)d};
     auto launch = [&](auto kern, int smem, unsigned blocks_y) {
         if (smem > 48 * 1024 &&
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
@@ -282,7 +361,7 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
         kern<<<dim3(heads, blocks_y), 256, smem, st>>>(q_win, rope_coef, s.n_q_heads, s.window, s.rope_layout,
                                                        inv_norm, mu_bar, sigma_bar, s.window,
                                                        reinterpret_cast<const long long*>(pushed),
-                                                       s.cov_norm == EA_COV_SAMPLE ? 1 : 0);
+                                                       s.cov_norm == EA_COV_SAMPLE ? 1 : 0, img);
         return true;
     };
     bool ok;
@@ -299,14 +378,17 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
 
 ea_status ea_launch_stats(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_win,
                           const int64_t* pos_next, int n_future, double rope_base, float* rope_coef,
-                          float* mu_bar, float* sigma_bar, cudaStream_t st) {
-    return launch_stats(ctx, s, q_win, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st);
+                          float* mu_bar, float* sigma_bar, cudaStream_t st, void* image, float* vec) {
+    return launch_stats(ctx, s, q_win, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st, nullptr, image,
+                        vec);
 }
 
 ea_status ea_launch_stats_ring(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* q_ring,
                                const int64_t* pushed, const int64_t* pos_next, int n_future, double rope_base,
-                               float* rope_coef, float* mu_bar, float* sigma_bar, cudaStream_t st) {
-    return launch_stats(ctx, s, q_ring, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st, pushed);
+                               float* rope_coef, float* mu_bar, float* sigma_bar, cudaStream_t st, void* image,
+                               float* vec) {
+    return launch_stats(ctx, s, q_ring, pos_next, n_future, rope_base, rope_coef, mu_bar, sigma_bar, st, pushed, image,
+                        vec);
 }
 
 ea_status ea_launch_stats_f32(const ea_ctx* ctx, const ea_shape& s, const float* q_win, const int64_t* pos_next,
@@ -384,21 +466,21 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
     switch (d) {
         case 64:
             stats_mma_kernel<64, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<64, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                    s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0);
+                                                                    s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0, StatsImage{nullptr, nullptr, 1, 0.f, 0.f});
             break;
         case 128:
             if (cudaFuncSetAttribute(stats_mma_kernel<128, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      stats_smem_bytes<128, __nv_bfloat16>()) != cudaSuccess)
                 return EA_ERR_CUDA;
             stats_mma_kernel<128, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<128, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0);
+                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0, StatsImage{nullptr, nullptr, 1, 0.f, 0.f});
             break;
         default:
             if (cudaFuncSetAttribute(stats_mma_kernel<256, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      stats_smem_bytes<256, __nv_bfloat16>()) != cudaSuccess)
                 return EA_ERR_CUDA;
             stats_mma_kernel<256, __nv_bfloat16><<<dim3(heads, 3), 256, stats_smem_bytes<256, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0);
+                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0, StatsImage{nullptr, nullptr, 1, 0.f, 0.f});
             break;
     }
     return EA_CHECK_LAUNCH();

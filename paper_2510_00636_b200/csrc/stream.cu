@@ -128,17 +128,22 @@ ea_status ea_query_stats_ring(ea_ctx* ctx, const ea_shape* shape, const void* q_
         return EA_ERR_INVALID_ARG;
     if (shape->cov_norm != EA_COV_POPULATION && shape->cov_norm != EA_COV_SAMPLE) return EA_ERR_INVALID_ARG;
     if (shape->n_units == 0) return EA_OK;
-    if (!q_ring || !ring_pushed || !pos_next || !mu_bar || !sigma_bar) return EA_ERR_INVALID_ARG;
+    if (!q_ring || !ring_pushed || !pos_next || !mu_bar) return EA_ERR_INVALID_ARG;
     if (!aligned16(q_ring) || !aligned16(mu_bar) || !aligned16(sigma_bar)) return EA_ERR_INVALID_ARG;
     if (n_future < 1 || !(rope_base > 0.0) || shape->window < 1) return EA_ERR_INVALID_ARG;
     const ea_ws_plan plan = ea_plan_workspace(*shape);
     if (ctx->workspace_bytes < plan.logits /* rope_coef region only */) return EA_ERR_WORKSPACE;
+    void* image = nullptr;
+    float* vec = nullptr;
+    if (!ea_fused_image_target(ctx, *shape, &image, &vec)) return EA_ERR_WORKSPACE;
+    if (!sigma_bar && !image) return EA_ERR_INVALID_ARG;       // sigma_bar may only be left out in fused mode
     int prev = 0;
     EA_CUDA_TRY(cudaGetDevice(&prev));
     if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
     float* coef = reinterpret_cast<float*>(static_cast<char*>(ctx->workspace) + plan.rope_coef);
     st = ea_launch_stats_ring(ctx, *shape, static_cast<const __nv_bfloat16*>(q_ring), ring_pushed, pos_next, n_future,
-                              rope_base, coef, mu_bar, sigma_bar, static_cast<cudaStream_t>(cuda_stream));
+                              rope_base, coef, mu_bar, sigma_bar, static_cast<cudaStream_t>(cuda_stream), image, vec);
+    if (st != EA_OK) ctx->image_ready = false;
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

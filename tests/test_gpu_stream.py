@@ -280,3 +280,56 @@ def test_unordered_inplace_compaction_exact(ea, oracle, n, n_kept, d, cap):
     assert np.array_equal(k1[:, :, :n_kept], oracle.gather(k0[:, :, :n], want))
     assert np.array_equal(v1[:, :, :n_kept], oracle.gather(v0[:, :, :n], want))
     assert np.array_equal(k1[:, :, n_kept:], k0[:, :, n_kept:]) and np.array_equal(v1[:, :, n_kept:], v0[:, :, n_kept:])
+
+
+@pytest.mark.parametrize("d,Hq,Hkv,n,ring", [(128, 28, 4, 1408, True), (128, 8, 2, 640, False), (64, 10, 2, 300, False),
+                                             (64, 4, 2, 512, True)])
+def test_fused_statistics_give_the_same_scores_bit_for_bit(ea, d, Hq, Hkv, n, ring):
+    """ea_set_fused_stats: the operand written by the statistics kernel must be, bit for bit, the one
+    ea_score builds from mu_bar and sigma_bar - so the log-scores and the scores of
+    ea_score(NULL, NULL) equal those of the two-step path exactly, with and without sigma_bar
+    written, for a plain window and for a ring (partly filled and wrapped, and empty)."""
+    import dataclasses
+    cfg = dataclasses.replace(inputs.CONFIGS[4].tempered(2.0), n_layers=1, batch=3, n_q_heads=Hq, n_kv_heads=Hkv,
+                              head_dim=d, n_keys=n, window=48)
+    q, k, v, pos = inputs.generate_layer(cfg, layer=1, device="cuda")
+    U, W = cfg.batch, cfg.window
+    shape = ea.make_shape(U, Hq, Hkv, d, n, W)
+    ctx = ea.Context.for_shape(shape)
+    pos = pos.cuda()
+    ringbuf = torch.zeros_like(q)
+    pushed = torch.zeros((U,), dtype=torch.int64, device="cuda")
+
+    def stats(**kw):
+        if ring:
+            return ea.ea_query_stats_ring(ctx, shape, ringbuf, pushed, pos, cfg.n_future, cfg.rope_base, **kw)
+        return ea.ea_query_stats(ctx, shape, q, pos, cfg.n_future, cfg.rope_base, **kw)
+
+    for fill in ([0, 20, 70] if ring else [None]):
+        if fill:
+            ea.ea_window_push(ctx, shape, ringbuf, pushed, q[:, :, :fill - int(pushed[0]) if fill <= W else W].contiguous())
+        ctx.set_fused_stats(False)
+        mu, sig = stats()
+        sc0, lg0 = ea.ea_score(ctx, shape, k, v, mu, sig, cfg.eps, want_logits=True)
+        sc0, lg0 = sc0.clone(), lg0.clone()
+        ctx.set_fused_stats(True)
+        mu1, sig1 = stats()
+        assert torch.equal(mu1, mu) and torch.equal(sig1, sig)
+        sc1, lg1 = ea.ea_score(ctx, shape, k, v, None, None, cfg.eps, want_logits=True)
+        assert torch.equal(lg1, lg0) and torch.equal(sc1, sc0)
+        mu2, none = stats(want_sigma=False)
+        assert none is None and torch.equal(mu2, mu)
+        sc2, lg2 = ea.ea_score(ctx, shape, k, v, None, None, cfg.eps, want_logits=True)
+        ctx.sync_status()
+        assert torch.equal(lg2, lg0) and torch.equal(sc2, sc0)
+    # without a matching operand the call is refused
+    other = ea.make_shape(U, Hq, Hkv, d, n - 1 if n > 129 else n + 1, W)
+    big = ea.Context.for_shape(ea.make_shape(U, Hq, Hkv, d, n + 1, W))
+    with pytest.raises(ea.EAError) as e:
+        ea.ea_score(big, other, k[:, :, :other.n_keys].contiguous(), v[:, :, :other.n_keys].contiguous(), None, None, cfg.eps)
+    assert e.value.status == 1
+    ctx.set_fused_stats(False)
+    with pytest.raises(ea.EAError):
+        stats(want_sigma=False)
+    with pytest.raises(ea.EAError):
+        ea.ea_score(ctx, shape, k, v, None, None, cfg.eps)

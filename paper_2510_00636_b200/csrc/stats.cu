@@ -372,7 +372,7 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
         default: return EA_ERR_UNSUPPORTED;
     }
     if (!ok) return EA_ERR_CUDA;
-    ea_count_launches(ctx, 2);
+    if (ctx) ea_count_launches(ctx, 2);
     return EA_CHECK_LAUNCH();
 }
 
@@ -455,33 +455,8 @@ extern "C" ea_status ea_query_stats_static(const ea_shape* s, const void* q_win,
     ea_status st = static_coef_address(&coef);
     if (st != EA_OK) return st;
 
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(q_win);
-    const int n_coef = s->n_units * half;
-    // every coefficient this call reads is written first, so stale contents of earlier calls are harmless
-    rope_coef_kernel<<<(n_coef + 127) / 128, 128, 0, stream>>>(pos_next, s->n_units, half, d, n_future,
-                                                               rope_base, coef);
-    const float inv_norm = 1.0f / (float)(s->cov_norm == EA_COV_SAMPLE ? s->window - 1 : s->window);
-    const unsigned heads = (unsigned)(s->n_units * s->n_q_heads);
-    switch (d) {
-        case 64:
-            stats_mma_kernel<64, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<64, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                    s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0, StatsImage{nullptr, nullptr, 1, 0.f, 0.f});
-            break;
-        case 128:
-            if (cudaFuncSetAttribute(stats_mma_kernel<128, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     stats_smem_bytes<128, __nv_bfloat16>()) != cudaSuccess)
-                return EA_ERR_CUDA;
-            stats_mma_kernel<128, __nv_bfloat16><<<dim3(heads, 1), 256, stats_smem_bytes<128, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0, StatsImage{nullptr, nullptr, 1, 0.f, 0.f});
-            break;
-        default:
-            if (cudaFuncSetAttribute(stats_mma_kernel<256, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     stats_smem_bytes<256, __nv_bfloat16>()) != cudaSuccess)
-                return EA_ERR_CUDA;
-            stats_mma_kernel<256, __nv_bfloat16><<<dim3(heads, 3), 256, stats_smem_bytes<256, __nv_bfloat16>(), stream>>>(q, coef, s->n_q_heads, s->window,
-                                                                     s->rope_layout, inv_norm, mu_bar, sigma_bar, s->window, nullptr, 0, StatsImage{nullptr, nullptr, 1, 0.f, 0.f});
-            break;
-    }
-    return EA_CHECK_LAUNCH();
+    // the same launches as ea_query_stats, without a context (nothing to count the launches in); every
+    // coefficient this call reads is written first, so stale contents of earlier calls are harmless
+    return launch_stats(nullptr, *s, static_cast<const __nv_bfloat16*>(q_win), pos_next, n_future, rope_base, coef,
+                        mu_bar, sigma_bar, static_cast<cudaStream_t>(cuda_stream));
 }

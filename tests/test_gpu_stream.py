@@ -333,3 +333,39 @@ def test_fused_statistics_give_the_same_scores_bit_for_bit(ea, d, Hq, Hkv, n, ri
         stats(want_sigma=False)
     with pytest.raises(ea.EAError):
         ea.ea_score(ctx, shape, k, v, None, None, cfg.eps)
+
+
+def test_streaming_calls_validate_their_arguments(ea):
+    U, Hq, Hkv, d, W, cap = 1, 4, 2, 64, 8, 40
+    k = torch.zeros((U, Hkv, cap, d), dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    new = torch.ones((U, Hkv, 16, d), dtype=torch.bfloat16, device="cuda")
+    ring = torch.zeros((U, Hq, W, d), dtype=torch.bfloat16, device="cuda")
+    pushed = torch.zeros((U,), dtype=torch.int64, device="cuda")
+    ctx = ea.Context.for_shape(ea.make_shape(U, Hq, Hkv, d, cap, W, kv_capacity=cap))
+
+    def status(fn):
+        with pytest.raises(ea.EAError) as e:
+            fn()
+        return e.value.status
+
+    # appending beyond the capacity, and a capacity below the cache length
+    assert status(lambda: ea.ea_cache_append(ctx, ea.make_shape(U, Hq, Hkv, d, 30, W, kv_capacity=cap), k, v, new, new)) == 1
+    assert status(lambda: ea.ea_cache_append(ctx, ea.make_shape(U, Hq, Hkv, d, 30, W, kv_capacity=20), k, v, new, new)) == 1
+    # exactly to the brim is fine, and lands where it should
+    ea.ea_cache_append(ctx, ea.make_shape(U, Hq, Hkv, d, 24, W, kv_capacity=cap), k, v, new, new)
+    ctx.sync_status()
+    assert float(k[:, :, :24].abs().max()) == 0.0 and float(k[:, :, 24:].min()) == 1.0
+    # a ring without rows, a missing counter
+    assert status(lambda: ea.ea_window_push(ctx, ea.make_shape(U, Hq, Hkv, d, 0, 0), ring, pushed, new[:, :, :4].repeat(1, 2, 1, 1))) == 1
+    shape = ea.make_shape(U, Hq, Hkv, d, 0, W)
+    import ctypes
+    L = ea.lib()
+    assert L.ea_window_push(ctx._h, ctypes.byref(shape), ctypes.c_void_p(ring.data_ptr()), None,
+                            ctypes.c_void_p(ring.data_ptr()), 2, None) == 1
+    assert L.ea_query_stats_ring(ctx._h, ctypes.byref(shape), ctypes.c_void_p(ring.data_ptr()), None, None, 4, 1e4, None,
+                                 None, None) == 1
+    # empty pushes and appends are no-ops
+    ea.ea_window_push(ctx, shape, ring, pushed, ring[:, :, :0].contiguous())
+    ctx.sync_status()
+    assert int(pushed[0]) == 0

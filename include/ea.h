@@ -439,7 +439,7 @@ int64_t ea_n_floor(int64_t n_kept, double safeguard);
  * so that work launched beside it - another context's memory-bound passes, a
  * decode step of the serving engine - finds the other SMs free instead of
  * queueing behind it (the paper has no counterpart).  n_sms = 0 restores the
- * default, every SM of the device.  2 <= n_sms <= SM count, else
+ * default, every SM of the device.  32 <= n_sms <= SM count, else
  * EA_ERR_INVALID_ARG.  Takes effect from the next ea_score / ea_score_wo.
  */
 ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms);
@@ -471,7 +471,7 @@ ea_status ea_set_fused_stats(ea_ctx* ctx, int32_t on);
  * persistent kernel of n_sms CTAs streams V through bulk copies on a stream the
  * context owns, the log-score kernel takes the other SMs, and a light weighting
  * pass joins the two.  The scores are those of the default path up to the
- * rounding of one fp32 square root.  n_sms even, 0 <= n_sms <= SM count - 2
+ * rounding of one fp32 square root.  n_sms even, 0 <= n_sms <= SM count - 32
  * (EA_ERR_INVALID_ARG otherwise); 0 (the default) switches the side pass off.
  * The first call with n_sms > 0 creates the stream and two events: make it
  * outside a stream capture.  Applies to ea_score with the tensor-core path

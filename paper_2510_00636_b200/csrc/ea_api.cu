@@ -549,7 +549,7 @@ int64_t ea_n_floor(int64_t n_kept, double safeguard) {
 ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms) {
     if (!ctx) return EA_ERR_INVALID_ARG;
     if (n_sms == 0) n_sms = ctx->sm_count;
-    if (n_sms < 2 || n_sms > ctx->sm_count) return EA_ERR_INVALID_ARG;
+    if (n_sms < 32 || n_sms > ctx->sm_count) return EA_ERR_INVALID_ARG;
     ctx->sm_budget = n_sms;
     return EA_OK;
 }
@@ -563,7 +563,7 @@ ea_status ea_set_fused_stats(ea_ctx* ctx, int32_t on) {
 
 ea_status ea_set_side_sms(ea_ctx* ctx, int32_t n_sms) {
     if (!ctx) return EA_ERR_INVALID_ARG;
-    if (n_sms < 0 || n_sms % 2 != 0 || n_sms > ctx->sm_count - 2) return EA_ERR_INVALID_ARG;
+    if (n_sms < 0 || n_sms % 2 != 0 || n_sms > ctx->sm_count - 32) return EA_ERR_INVALID_ARG;
     if (n_sms > 0 && !ctx->side_ready) {
         int prev = 0;
         EA_CUDA_TRY(cudaGetDevice(&prev));

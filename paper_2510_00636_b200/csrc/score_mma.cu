@@ -770,6 +770,10 @@ bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint
 }
 
 bool ea_mma_path_supported(const ea_shape& s) {
+    // one worker (CTA or CTA pair) per head subset of a KV head must exist even on the smallest SM budget
+    // (ea_set_sm_budget admits 32 SMs = 16 pairs); wider groups take the CUDA-core kernel
+    const int subsets = (s.n_q_heads / s.n_kv_heads + 256 / s.head_dim - 1) / (256 / s.head_dim);
+    if (subsets > 16) return false;
     if (s.head_dim == 256) return s.n_keys >= 2 * kTileKeys;
     return (s.head_dim == 64 || s.head_dim == 128) && s.n_keys >= kTileKeys;
 }

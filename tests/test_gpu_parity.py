@@ -215,7 +215,7 @@ def test_score_ragged_sizes(ea, oracle, n):
 
 
 @pytest.mark.parametrize("n", [129, 300, 1000])
-@pytest.mark.parametrize("d,Hq,Hkv", [(128, 6, 2), (64, 10, 2)])
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 6, 2), (64, 10, 2), (64, 68, 1)])   # the last: more head subsets than the tensor-core kernel takes
 def test_score_ragged_sizes_odd_groups(ea, oracle, n, d, Hq, Hkv):
     """Ragged caches with a group size that leaves the last pass of the tensor-core kernel partly
     empty (three query heads per KV head at two heads per pass; five at four per pass)."""
@@ -386,4 +386,4 @@ def test_side_pass_and_sm_budget_leave_the_result_unchanged(ea, cfg_id, side, bu
         with pytest.raises(ea.EAError):
             ctx.set_side_sms(bad)
     with pytest.raises(ea.EAError):
-        ctx.set_sm_budget(1)
+        ctx.set_sm_budget(16)

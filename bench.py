@@ -141,7 +141,8 @@ class Workload:
         if fp8:
             self.k_scale = torch.empty((U, Hkv, d), dtype=f32, device=device)
             self.v_scale = torch.empty((U, Hkv, n), dtype=f32, device=device)
-            self.k_scratch = torch.empty((U, Hkv, n, d), dtype=bf, device=device)
+            # scratch for the widened key codes: only head_dim 256 needs it (the kernel widens them itself below)
+            self.k_scratch = torch.empty((U, Hkv, n, d), dtype=bf, device=device) if d == 256 else None
         for layer in range(L):
             q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device=device)
             sl = slice(layer * B, (layer + 1) * B)
@@ -209,7 +210,8 @@ class Workload:
                                   self.mu[u0:u1], self.sigma[u0:u1])
             if self.fp8:
                 ea.ea_score_q8(ctx, shape, self.k[u0:u1], self.k_scale[u0:u1], self.v[u0:u1], self.v_scale[u0:u1],
-                               self.mu[u0:u1], self.sigma[u0:u1], cfg.eps, self.k_scratch[u0:u1], self.scores[u0:u1])
+                               self.mu[u0:u1], self.sigma[u0:u1], cfg.eps,
+                               None if self.k_scratch is None else self.k_scratch[u0:u1], self.scores[u0:u1])
                 ea.ea_select_compact_q8(ctx, shape, self.scores[u0:u1], cfg.n_kept, self.k[u0:u1], self.v[u0:u1],
                                         self.v_scale[u0:u1], out=(self.idx[u0:u1], self.k_out[u0:u1],
                                                                   self.v_out[u0:u1], self.v_scale_out[u0:u1]))

@@ -276,8 +276,10 @@ ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const v
  * k_q8, v_q8  uint8 [n_units, Hkv, n, d] E4M3 codes, 16-byte aligned, dense
  *             (kv_capacity must be 0 or n_keys: EA_ERR_UNSUPPORTED otherwise)
  * k_scale     fp32 [n_units, Hkv, d];   v_scale  fp32 [n_units, Hkv, n]
- * k_scratch   bf16 [n_units, Hkv, n, d]  caller-owned scratch; holds the
- *             widened key codes on return
+ * k_scratch   bf16 [n_units, Hkv, n, d]  caller-owned scratch for the widened key
+ *             codes.  Needed, and written, only where the tensor-core kernel
+ *             does not widen the codes itself: head_dim 256, or fewer keys than
+ *             one tile; may be NULL otherwise (head_dim 64 and 128)
  * the other arguments as for ea_score.
  */
 ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, const float* k_scale,

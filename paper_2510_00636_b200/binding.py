@@ -337,7 +337,8 @@ def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar
     _dev_tensor(v_scale, torch.float32, "v_scale")
     U, Hq, Hkv, n, d = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys, shape.head_dim
     dev = k_q8.device
-    if k_scratch is None:
+    if k_scratch is None and (d == 256 or n < 128):
+        # only where the tensor-core kernel does not widen the codes itself
         k_scratch = torch.empty((U, Hkv, n, d), dtype=torch.bfloat16, device=dev)
     if scores is None:
         scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=dev)

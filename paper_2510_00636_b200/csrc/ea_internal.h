@@ -130,7 +130,7 @@ ea_status ea_launch_logits_simt(const ea_ctx* ctx, const ea_shape& s, const __nv
 
 // bf16 rank-3 TMA tensor map, box (box0 x box1 x 1), 128-byte swizzle, zero fill outside.
 bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint64_t n1, uint64_t n2,
-                           uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1);
+                           uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1, bool bytes_plain = false);
 
 // Window queries from hidden states, Q[u,h,w,:] = W_Q^h H[u,w,:] in fp32 (tcgen05 GEMM).
 bool ea_project_supported(const ea_shape& s, int d_model);
@@ -150,6 +150,11 @@ size_t ea_mma_lse_part_bytes(const ea_shape& s);
 ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k,
                                const ea_quad_form& form, void* image, float* vec,
                                float* logits, float* lse_part, int* n_chunks, cudaStream_t st);
+// The same kernel on FP8 E4M3 key codes, widened to bf16 inside it (head_dim <= 128); form.ch_scale carries the scales.
+bool ea_mma_q8_supported(const ea_shape& s);
+ea_status ea_launch_logits_mma_q8(const ea_ctx* ctx, const ea_shape& s, const uint8_t* k_q8,
+                                  const ea_quad_form& form, void* image, float* vec, float* logits,
+                                  float* lse_part, int* n_chunks, cudaStream_t st);
 // log-sum-exp per softmax row from the per-work-unit partials of the tensor-core kernel
 ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const float* lse_part, int n_chunks,
                                 float* lse, cudaStream_t st);

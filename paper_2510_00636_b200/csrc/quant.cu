@@ -182,8 +182,8 @@ ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, cons
     if (st != EA_OK) return st;
     if (shape->kv_capacity != 0 && shape->kv_capacity != shape->n_keys) return EA_ERR_UNSUPPORTED;
     if (shape->n_units == 0 || shape->n_keys == 0) return EA_OK;
-    if (!k_q8 || !k_scale || !v_q8 || !v_scale || !mu_bar || !sigma_bar || !k_scratch || !scores)
-        return EA_ERR_INVALID_ARG;
+    if (!k_q8 || !k_scale || !v_q8 || !v_scale || !mu_bar || !sigma_bar || !scores) return EA_ERR_INVALID_ARG;
+    if (!k_scratch && !ea_mma_q8_supported(*shape)) return EA_ERR_INVALID_ARG;
     if (!aligned16(k_q8) || !aligned16(v_q8) || !aligned16(k_scratch) || !aligned16(mu_bar) || !aligned16(sigma_bar) ||
         !aligned16(scores) || !aligned16(logits_opt))
         return EA_ERR_INVALID_ARG;
@@ -200,9 +200,22 @@ ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, cons
     __nv_bfloat16* codes = static_cast<__nv_bfloat16*>(k_scratch);
     ea_quad_form eq7 = ea_eq7_form(*shape, mu_bar, sigma_bar);
     eq7.ch_scale = k_scale;
-    st = ea_launch_dequant_k(ctx, *shape, static_cast<const uint8_t*>(k_q8), codes, stream);
     bool lse_ready = false;
-    if (st == EA_OK) {
+    if (ea_mma_q8_supported(*shape)) {
+        // head_dim <= 128: the tensor-core kernel takes the codes as they are and widens them itself
+        float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
+        int n_chunks = 0;
+        st = ea_launch_logits_mma_q8(ctx, *shape, static_cast<const uint8_t*>(k_q8), eq7, ws + plan.image,
+                                     reinterpret_cast<float*>(ws + plan.vec), logits, lse_part, &n_chunks, stream);
+        if (st == EA_OK && shape->group_mode != EA_GROUP_MEAN_LOGIT) {
+            st = ea_launch_lse_combine(ctx, *shape, lse_part, n_chunks, lse, stream);
+            lse_ready = true;
+        }
+    } else {
+        // otherwise a pass of its own widens the codes into the caller's scratch first
+        st = ea_launch_dequant_k(ctx, *shape, static_cast<const uint8_t*>(k_q8), codes, stream);
+    }
+    if (st == EA_OK && !ea_mma_q8_supported(*shape)) {
         if (ea_mma_path_supported(*shape)) {
             float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
             int n_chunks = 0;

@@ -31,6 +31,9 @@
 // head_dim 256, four at head_dim <= 128.  The epilogue reads the key rows from the slots as it works
 // through the accumulator and hands each slot back as soon as its warps are done with it.
 // Every wait is bounded; a wait that gives up raises the context's status word.
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+
 #include <mutex>
 
 #include "ea_internal.h"
@@ -45,8 +48,13 @@ constexpr int kTileKeys = 128;                     // keys per CTA per step
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;                      // columns of one accumulator stage
 constexpr int kChunkA = kTileKeys * 128;           // bytes of one 64-channel chunk of a key tile
+constexpr int kChunkQ = kTileKeys * 64;            // the same chunk as FP8 codes
 
-template <int D, bool PAIR>
+// Q8: the keys arrive as FP8 E4M3 codes.  The copy engine lands a chunk of codes in a small staging slot,
+// four more warps widen it to bf16 (exact) straight into the chunk's slot of the operand ring, in the
+// swizzled layout the MMA reads; everything downstream is unchanged.  head_dim <= 128 only: the staging
+// slots and one tile less of ring fit there, at head_dim 256 nothing is left.
+template <int D, bool PAIR, bool Q8 = false>
 struct Geo {
     using L = EaImage<D>;                                // the image's layout in global memory
     static constexpr int HPC = L::HPC;
@@ -60,9 +68,11 @@ struct Geo {
     // Epilogue: EPI_PARTS warps per tensor-memory lane quarter, each with CPP columns of every head.
     static constexpr int EPI_PARTS = 2;
     static constexpr int EPI_WARPS = 4 * EPI_PARTS;
-    static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+    static constexpr int CONV_WARPS = Q8 ? 4 : 0;          // warps 2 + EPI_WARPS ..: code -> bf16
+    static constexpr int THREADS = 32 * (2 + EPI_WARPS + CONV_WARPS);
     static constexpr int CPP = D / EPI_PARTS;
-    static constexpr int NSLOT = (D == 256 ? 2 : 4) * KCH;   // ring of 16 KiB chunk slots: 2 or 4 key tiles
+    static constexpr int NSLOT = (D == 256 ? 2 : (Q8 ? 3 : 4)) * KCH;   // ring of 16 KiB chunk slots: 2, 3 or 4 key tiles
+    static constexpr int NQ = Q8 ? 4 : 0;                  // staging slots of 8 KiB for chunks of codes
     static constexpr int VEC = HPC * D * (int)sizeof(float);       // diagonal vectors of the resident heads
     // linear term: one extra K = 16 MMA step, a constant block of ones times (hi, lo) of mu' per column,
     // both as unswizzled K-major core matrices (8 rows x 16 bytes; 128 bytes on along K, 256 on along rows)
@@ -77,12 +87,13 @@ struct Geo {
     // partial sums of the column parts: [tile parity][part][head][key]
     static constexpr int PART = 2 * EPI_PARTS * HPC * kTileKeys * (int)sizeof(float);
     static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
-    static constexpr int NBAR = 2 * NSLOT + 6;
+    static constexpr int NBAR = 2 * NSLOT + 6 + 2 * NQ;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
+    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + NQ * kChunkQ + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
     // epilogue warps that read a chunk slot and hand it back to the producer
     static constexpr int SLOT_READERS = D == 64 ? EPI_WARPS : 4;
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
+    static_assert(!Q8 || (!PAIR && D <= 128), "codes are widened in the kernel at head_dim <= 128 only");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
@@ -224,6 +235,12 @@ __device__ __forceinline__ Item decode_item(long long w, int hs, const MmaParams
     return it;
 }
 
+// two E4M3 codes -> two floats (exact)
+__device__ __forceinline__ float2 e4m3x2_to_float2(uint16_t two) {
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(two), __NV_E4M3);
+    return __half22float2(*reinterpret_cast<const __half2*>(&h));
+}
+
 // AND of `ok` over all NT epilogue threads (named barrier 1): keeps their control flow identical.
 template <int NT>
 __device__ __forceinline__ bool epi_all(bool ok) {
@@ -239,10 +256,10 @@ __device__ __forceinline__ bool epi_all(bool ok) {
     return r != 0;
 }
 
-template <int D, bool PAIR>
-__global__ void __launch_bounds__(Geo<D, PAIR>::THREADS, 1)
+template <int D, bool PAIR, bool Q8>
+__global__ void __launch_bounds__(Geo<D, PAIR, Q8>::THREADS, 1)
 logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) {
-    using G = Geo<D, PAIR>;
+    using G = Geo<D, PAIR, Q8>;
     static_assert(!(G::DIAG_MMA && PAIR), "the diagonal blocks are laid out for a single CTA");
     extern __shared__ uint8_t smem_raw[];
     // carve shared memory: 1024-byte aligned operand tiles first
@@ -250,7 +267,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_img = base;
     const uint32_t s_k = s_img + G::IMG_CTA;
-    constexpr int kOffOnes = G::IMG_CTA + G::NSLOT * kChunkA;
+    const uint32_t s_q = s_k + G::NSLOT * kChunkA;                 // staging slots for chunks of codes (Q8)
+    constexpr int kOffOnes = G::IMG_CTA + G::NSLOT * kChunkA + G::NQ * kChunkQ;
     const uint32_t s_ones = base + kOffOnes;
     const uint32_t s_lin = s_ones + G::ONES;
     constexpr int kOffVec = kOffOnes + G::ONES + G::LIN_CTA;
@@ -268,6 +286,8 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     auto tmem_empty = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + 2 + a); };
     const uint32_t img_full = s_bar + 8u * (2 * G::NSLOT + 4);
     const uint32_t img_peer = s_bar + 8u * (2 * G::NSLOT + 5);
+    auto q_full = [&](int s) { return s_bar + 8u * (2 * G::NSLOT + 6 + s); };           // codes have landed
+    auto q_empty = [&](int s) { return s_bar + 8u * (2 * G::NSLOT + 6 + G::NQ + s); };  // codes have been widened
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * G::NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * G::NBAR + 4);
 
@@ -277,8 +297,12 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < G::NSLOT; ++s) {
-            mbar_init(full_k(s), 1);
+            mbar_init(full_k(s), Q8 ? G::CONV_WARPS : 1);          // Q8: the widening warps fill the slot
             mbar_init(empty_k(s), G::SLOT_READERS);
+        }
+        for (int s = 0; s < G::NQ; ++s) {
+            mbar_init(q_full(s), 1);
+            mbar_init(q_empty(s), G::CONV_WARPS);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
@@ -363,6 +387,16 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     for (int kc = 0; ok && kc < G::KCH; ++kc) {
                         const long long c = tile_no * G::KCH + kc;
                         const int slot = slot_of(c);
+                        if constexpr (Q8) {
+                            // codes go to a staging slot; the widening warps take it from there to ring slot `slot`
+                            const int qs = (int)(c % G::NQ);
+                            ok = mbar_wait(q_empty(qs), ((uint32_t)(c / G::NQ) & 1) ^ 1, abort_flag);
+                            if (!ok) break;
+                            mbar_arrive_expect_tx(q_full(qs), kChunkQ);
+                            tma_load_3d(s_q + qs * kChunkQ, &k_map, q_full(qs), kc * 64, key0, it.ug);
+                            issued = c + 1;
+                            continue;
+                        }
                         ok = mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
                         if (!ok) break;
                         if (PAIR) {
@@ -378,7 +412,12 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     }
                 }
             }
-            if (!ok && leader) {
+            if (!ok && Q8) {
+                for (int back = 1; back <= G::NQ && back <= issued; ++back) {
+                    const long long c = issued - back;
+                    mbar_drain(q_full((int)(c % G::NQ)), (uint32_t)(c / G::NQ) & 1);
+                }
+            } else if (!ok && leader) {
                 // Let the copies already in flight land before the shared memory goes away.  In a pair the
                 // leader's barriers count both CTAs' bytes, and the peer stays until the teardown's cluster
                 // barrier, which the leader reaches only after this.  Bounded by time: a copy the peer
@@ -472,6 +511,51 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             }
         }
         __syncwarp();
+    } else if (warp >= 2 + G::EPI_WARPS) {
+        // ------------------------------------------------------------------ code -> bf16 (Q8)
+        // 128 threads, 512 pieces of 16 codes per chunk: thread t takes pieces t, t + 128, ... (a warp reads
+        // 512 contiguous bytes); piece (row, u) becomes the 16-byte units 2u and 2u + 1 of the row's 128
+        // bytes in the ring slot, at the swizzled places the MMA and the epilogue expect.
+        const int ct = threadIdx.x - 32 * (2 + G::EPI_WARPS);
+        long long tile_no = 0;
+        bool ok = true;
+        for (long long item = first; ok && item < last; ++item) {
+            const Item it = decode_item(item, my_hs, p, G::HPC);
+            for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
+                for (int kc = 0; ok && kc < G::KCH; ++kc) {
+                    const long long c = tile_no * G::KCH + kc;
+                    const int slot = slot_of(c), qs = (int)(c % (G::NQ > 0 ? G::NQ : 1));
+                    ok = mbar_wait(q_full(qs), (uint32_t)(c / (G::NQ > 0 ? G::NQ : 1)) & 1, abort_flag);
+                    ok = ok && mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    const uint32_t src = s_q + qs * kChunkQ, dst = s_k + slot * kChunkA;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int piece = ct + 128 * i, r = piece / 4, u = piece % 4;
+                        const uint4 x = lds128(src + piece * 16);
+                        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                        uint32_t o[8];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float2 lo = e4m3x2_to_float2((uint16_t)(w[q] & 0xffffu));
+                            const float2 hi = e4m3x2_to_float2((uint16_t)(w[q] >> 16));
+                            // exact: the floats' low 16 bits are zero
+                            o[2 * q] = (__float_as_uint(lo.x) >> 16) | (__float_as_uint(lo.y) & 0xffff0000u);
+                            o[2 * q + 1] = (__float_as_uint(hi.x) >> 16) | (__float_as_uint(hi.y) & 0xffff0000u);
+                        }
+                        sts128(dst + r * 128 + (((2 * u) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
+                        sts128(dst + r * 128 + (((2 * u + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
+                    }
+                    fence_proxy_async_smem();          // the MMA reads these bytes through the async proxy
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(full_k(slot));
+                        mbar_arrive(q_empty(qs));
+                    }
+                }
+            }
+        }
     } else {
         // ------------------------------------------------------------------ epilogue
         // Warp (quarter, part): accumulator lanes 32*quarter.. (thread <-> lane <-> key) and columns
@@ -670,16 +754,17 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 // ------------------------------------------------------------------------------------------
 // K as a rank-3 tensor (d, n, unit*kv_head); one box is 64 channels x 128 keys, 128-byte swizzle.
 // Rows past n read as zero; heads are kv_capacity rows apart.
-bool make_k_map(CUtensorMap* map, const __nv_bfloat16* k, int d, int n, int cap, long long heads) {
-    return ea_tensor_map_bf16_3d(map, k, (uint64_t)d, (uint64_t)n, (uint64_t)heads, (uint64_t)d * 2,
-                                 (uint64_t)cap * d * 2, 64, kTileKeys);
+bool make_k_map(CUtensorMap* map, const void* k, int d, int n, int cap, long long heads, bool codes) {
+    const uint64_t es = codes ? 1 : 2;                 // bytes per element: FP8 codes or bf16
+    return ea_tensor_map_bf16_3d(map, k, (uint64_t)d, (uint64_t)n, (uint64_t)heads, (uint64_t)d * es,
+                                 (uint64_t)cap * d * es, 64, kTileKeys, codes);
 }
 
-template <int D, bool PAIR>
-ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* k, const ea_quad_form& form,
+template <int D, bool PAIR, bool Q8>
+ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const void* k, const ea_quad_form& form,
                      uint8_t* image, float* vec, float* logits, float* lse_part, int* n_chunks_out,
                      cudaStream_t st) {
-    using G = Geo<D, PAIR>;
+    using G = Geo<D, PAIR, Q8>;
     const int Gq = s.n_q_heads / s.n_kv_heads;
     constexpr int keys_per_step = PAIR ? 2 * kTileKeys : kTileKeys;
     // CTAs or CTA pairs, one per SM; the SMs of a side pass (ea_set_side_sms) are left to it
@@ -710,11 +795,11 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
     *n_chunks_out = p.n_chunks * (PAIR ? 2 : 1);
 
     CUtensorMap k_map;
-    if (!make_k_map(&k_map, k, D, s.n_keys, ea_kv_cap(s), (long long)s.n_units * s.n_kv_heads)) return EA_ERR_CUDA;
+    if (!make_k_map(&k_map, k, D, s.n_keys, ea_kv_cap(s), (long long)s.n_units * s.n_kv_heads, Q8)) return EA_ERR_CUDA;
 
     if (form.quad)
         sigma_image_kernel<D><<<s.n_units * s.n_q_heads, 256, 0, st>>>(form, s.n_q_heads, s.n_kv_heads, image, vec);
-    auto kern = logits_mma_kernel<D, PAIR>;
+    auto kern = logits_mma_kernel<D, PAIR, Q8>;
     EA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
     const long long want = (long long)p.n_groups * p.n_subsets;
     cudaLaunchConfig_t cfg = {};
@@ -742,7 +827,7 @@ ea_status launch_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* 
 // bf16 rank-3 tensor map (innermost extent first) with a (box0 x box1 x 1) box, 128-byte swizzle,
 // zero fill outside the tensor.  Strides in bytes, multiples of 16; base 16-byte aligned.
 bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint64_t n1, uint64_t n2,
-                           uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1) {
+                           uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1, bool bytes_plain) {
     typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -764,8 +849,10 @@ bool ea_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t n0, uint
     const cuuint64_t strides[2] = {stride1, stride2};
     const cuuint32_t box[3] = {box0, box1, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    // bytes_plain: 8-bit elements, rows of the box stored one after the other without swizzle
+    return fn(map, bytes_plain ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              bytes_plain ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -802,11 +889,27 @@ ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_
     uint8_t* img = static_cast<uint8_t*>(image);
     switch (s.head_dim) {
         case 64:
-            return launch_mma<64, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
+            return launch_mma<64, false, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
         case 128:
-            return launch_mma<128, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
+            return launch_mma<128, false, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
         case 256:
-            return launch_mma<256, true>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
+            return launch_mma<256, true, false>(ctx, s, k, form, img, vec, logits, lse_part, n_chunks, st);
+        default:
+            return EA_ERR_UNSUPPORTED;
+    }
+}
+
+bool ea_mma_q8_supported(const ea_shape& s) { return ea_mma_path_supported(s) && s.head_dim <= 128; }
+
+ea_status ea_launch_logits_mma_q8(const ea_ctx* ctx, const ea_shape& s, const uint8_t* k_q8,
+                                  const ea_quad_form& form, void* image, float* vec, float* logits,
+                                  float* lse_part, int* n_chunks, cudaStream_t st) {
+    uint8_t* img = static_cast<uint8_t*>(image);
+    switch (s.head_dim) {
+        case 64:
+            return launch_mma<64, false, true>(ctx, s, k_q8, form, img, vec, logits, lse_part, n_chunks, st);
+        case 128:
+            return launch_mma<128, false, true>(ctx, s, k_q8, form, img, vec, logits, lse_part, n_chunks, st);
         default:
             return EA_ERR_UNSUPPORTED;
     }

@@ -26,7 +26,8 @@ def _np(t):
 
 @pytest.mark.parametrize("cfg_id,scale,eps,n,mode", [(0, 2.0, 0.02, None, 0), (1, 2.0, 0.02, None, 0), (1, 3.0, 0.0, None, 0),
                                                      (1, 20.0, 0.02, None, 0), (0, 2.0, 0.02, 100, 0), (3, 2.0, 0.02, 3000, 0),
-                                                     (0, 2.0, 0.02, None, 1), (0, 2.0, 0.02, None, 2)])
+                                                     (0, 2.0, 0.02, None, 1), (0, 2.0, 0.02, None, 2),
+                                                     (2, 2.0, 0.02, 32768, 0), (4, 3.0, 0.0, 4608, 0)])   # full-size layers, codes widened in the kernel
 def test_quantised_whole_path(ea, oracle, cfg_id, scale, eps, n, mode):
     """Window statistics, scores of the quantised cache and compaction of code rows with their value scales,
     against the fp64 oracle on the same codes and scales: log-scores and scores within the tolerance protocol

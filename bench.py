@@ -141,8 +141,9 @@ class Workload:
         if fp8:
             self.k_scale = torch.empty((U, Hkv, d), dtype=f32, device=device)
             self.v_scale = torch.empty((U, Hkv, n), dtype=f32, device=device)
-            # scratch for the widened key codes: only head_dim 256 needs it (the kernel widens them itself below)
-            self.k_scratch = torch.empty((U, Hkv, n, d), dtype=bf, device=device) if d == 256 else None
+            # scratch for widened key codes: none at the bench shapes (the log-score kernel widens them itself)
+            scratch = ea.score_q8_scratch_bytes(ea.make_shape(U, Hq, Hkv, d, n, W))
+            self.k_scratch = torch.empty((U, Hkv, n, d), dtype=bf, device=device) if scratch > 0 else None
         for layer in range(L):
             q, k, v, pos = inputs.generate_layer(cfg, layer=layer, device=device)
             sl = slice(layer * B, (layer + 1) * B)

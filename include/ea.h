@@ -277,15 +277,19 @@ ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const v
  *             (kv_capacity must be 0 or n_keys: EA_ERR_UNSUPPORTED otherwise)
  * k_scale     fp32 [n_units, Hkv, d];   v_scale  fp32 [n_units, Hkv, n]
  * k_scratch   bf16 [n_units, Hkv, n, d]  caller-owned scratch for the widened key
- *             codes.  Needed, and written, only where the tensor-core kernel
- *             does not widen the codes itself: head_dim 256, or fewer keys than
- *             one tile; may be NULL otherwise (head_dim 64 and 128)
+ *             codes.  Needed, and written, only where the tensor-core kernel,
+ *             which widens the codes itself, does not take the shape (fewer
+ *             keys than one tile: 128, or 256 at head_dim 256; query groups of
+ *             more than 16 head subsets); ea_score_q8_scratch_bytes says how
+ *             many bytes that is, 0 meaning that k_scratch may be NULL
  * the other arguments as for ea_score.
  */
 ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, const float* k_scale,
                       const void* v_q8, const float* v_scale, const float* mu_bar,
                       const float* sigma_bar, float epsilon, void* k_scratch, float* scores,
                       float* logits_opt, void* cuda_stream);
+/* Host only: bytes of k_scratch that ea_score_q8 needs for this shape (0: none). */
+ea_status ea_score_q8_scratch_bytes(const ea_shape* shape, size_t* bytes);
 /*
  * ea_select_compact on a quantised cache: the same selection, then the kept
  * code rows and the value scales of their tokens are gathered (the key scales

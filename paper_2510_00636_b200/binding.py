@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_select_compact_q8", "ea_select_compact_inplace_unordered",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_select_compact_inplace_unordered",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.ea_score_q8.argtypes = [vp, sp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp]
         L.ea_select_compact_q8.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.ea_score_q8.restype = L.ea_select_compact_q8.restype = ctypes.c_int
+        L.ea_score_q8_scratch_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+        L.ea_score_q8_scratch_bytes.restype = ctypes.c_int
         L.ea_set_fused_stats.argtypes = [vp, i32]
         L.ea_set_fused_stats.restype = ctypes.c_int
         L.ea_set_sm_budget.argtypes = [vp, i32]
@@ -327,6 +329,13 @@ def ea_score(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, epsilon: float
     return (scores, logits) if (want_logits or logits is not None) else scores
 
 
+def score_q8_scratch_bytes(shape: Shape) -> int:
+    """Bytes of k_scratch ea_score_q8 needs for this shape (0: none)."""
+    out = ctypes.c_size_t(0)
+    _check(lib().ea_score_q8_scratch_bytes(ctypes.byref(shape), ctypes.byref(out)), "ea_score_q8_scratch_bytes")
+    return int(out.value)
+
+
 def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar, sigma_bar, epsilon: float,
                 k_scratch=None, scores=None, logits=None, want_logits: bool = False):
     """Scores of a quantised cache: k_q8, v_q8 uint8 [U,Hkv,n,d] (E4M3 codes), k_scale fp32 [U,Hkv,d],
@@ -337,7 +346,7 @@ def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar
     _dev_tensor(v_scale, torch.float32, "v_scale")
     U, Hq, Hkv, n, d = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys, shape.head_dim
     dev = k_q8.device
-    if k_scratch is None and (d == 256 or n < 128):
+    if k_scratch is None and score_q8_scratch_bytes(shape) > 0:
         # only where the tensor-core kernel does not widen the codes itself
         k_scratch = torch.empty((U, Hkv, n, d), dtype=torch.bfloat16, device=dev)
     if scores is None:

@@ -173,6 +173,17 @@ ea_status ea_launch_gather_q8(const ea_ctx* ctx, const ea_shape& s, int n_kept, 
 
 extern "C" {
 
+ea_status ea_score_q8_scratch_bytes(const ea_shape* shape, size_t* bytes) {
+    if (!shape || !bytes) return EA_ERR_INVALID_ARG;
+    size_t need = 0;
+    const ea_status st = ea_workspace_bytes(shape, &need);    // validates the shape
+    if (st != EA_OK) return st;
+    *bytes = ea_mma_q8_supported(*shape)
+                 ? 0
+                 : (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys * shape->head_dim * sizeof(__nv_bfloat16);
+    return EA_OK;
+}
+
 ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, const float* k_scale, const void* v_q8,
                       const float* v_scale, const float* mu_bar, const float* sigma_bar, float epsilon,
                       void* k_scratch, float* scores, float* logits_opt, void* cuda_stream) {
@@ -202,7 +213,7 @@ ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, cons
     eq7.ch_scale = k_scale;
     bool lse_ready = false;
     if (ea_mma_q8_supported(*shape)) {
-        // head_dim <= 128: the tensor-core kernel takes the codes as they are and widens them itself
+        // the tensor-core kernel takes the codes as they are and widens them itself
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
         int n_chunks = 0;
         st = ea_launch_logits_mma_q8(ctx, *shape, static_cast<const uint8_t*>(k_q8), eq7, ws + plan.image,

@@ -50,10 +50,10 @@ constexpr int kAccCols = 256;                      // columns of one accumulator
 constexpr int kChunkA = kTileKeys * 128;           // bytes of one 64-channel chunk of a key tile
 constexpr int kChunkQ = kTileKeys * 64;            // the same chunk as FP8 codes
 
-// Q8: the keys arrive as FP8 E4M3 codes.  The copy engine lands a chunk of codes in a small staging slot,
-// four more warps widen it to bf16 (exact) straight into the chunk's slot of the operand ring, in the
-// swizzled layout the MMA reads; everything downstream is unchanged.  head_dim <= 128 only: the staging
-// slots and one tile less of ring fit there, at head_dim 256 nothing is left.
+// Q8: the keys arrive as FP8 E4M3 codes.  The copy engine lands a chunk of codes (8 KiB) in the upper half
+// of the chunk's 16 KiB slot of the operand ring; four more warps read them all, meet at a named barrier and
+// write the bf16 values (exact) over the whole slot in the swizzled layout the MMA reads.  Everything
+// downstream is unchanged.  Each CTA of a pair widens its own keys and reports them on the leader's barrier.
 template <int D, bool PAIR, bool Q8 = false>
 struct Geo {
     using L = EaImage<D>;                                // the image's layout in global memory
@@ -71,8 +71,10 @@ struct Geo {
     static constexpr int CONV_WARPS = Q8 ? 4 : 0;          // warps 2 + EPI_WARPS ..: code -> bf16
     static constexpr int THREADS = 32 * (2 + EPI_WARPS + CONV_WARPS);
     static constexpr int CPP = D / EPI_PARTS;
-    static constexpr int NSLOT = (D == 256 ? 2 : (Q8 ? 3 : 4)) * KCH;   // ring of 16 KiB chunk slots: 2, 3 or 4 key tiles
-    static constexpr int NQ = Q8 ? 4 : 0;                  // staging slots of 8 KiB for chunks of codes
+    static constexpr int NSLOT = (D == 256 ? 2 : 4) * KCH;   // ring of 16 KiB chunk slots: 2 or 4 key tiles
+    static constexpr int NQ = Q8 ? NSLOT : 0;              // "codes have landed" barriers, one per slot
+    // arrivals that complete a ring slot: the copy engine's, or every widening warp's (of both CTAs of a pair)
+    static constexpr int FILLERS = Q8 ? (PAIR ? 2 : 1) * CONV_WARPS : 1;
     static constexpr int VEC = HPC * D * (int)sizeof(float);       // diagonal vectors of the resident heads
     // linear term: one extra K = 16 MMA step, a constant block of ones times (hi, lo) of mu' per column,
     // both as unswizzled K-major core matrices (8 rows x 16 bytes; 128 bytes on along K, 256 on along rows)
@@ -87,13 +89,12 @@ struct Geo {
     // partial sums of the column parts: [tile parity][part][head][key]
     static constexpr int PART = 2 * EPI_PARTS * HPC * kTileKeys * (int)sizeof(float);
     static constexpr int RED = HPC * 4 * 2 * (int)sizeof(float);   // per-warp (max, sum) of a work unit
-    static constexpr int NBAR = 2 * NSLOT + 6 + 2 * NQ;
+    static constexpr int NBAR = 2 * NSLOT + 6 + NQ;
     static constexpr int CTRL = ((NBAR * 8 + 16) + 127) / 128 * 128;
-    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + NQ * kChunkQ + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
+    static constexpr int SMEM = IMG_CTA + NSLOT * kChunkA + ONES + LIN_CTA + VEC + DIAG_FULL + PART + RED + CTRL + 1024;
     // epilogue warps that read a chunk slot and hand it back to the producer
     static constexpr int SLOT_READERS = D == 64 ? EPI_WARPS : 4;
     static_assert(!(D == 256) || PAIR, "head_dim 256 needs the paired form to fit in shared memory");
-    static_assert(!Q8 || (!PAIR && D <= 128), "codes are widened in the kernel at head_dim <= 128 only");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
@@ -235,26 +236,39 @@ __device__ __forceinline__ Item decode_item(long long w, int hs, const MmaParams
     return it;
 }
 
-// two E4M3 codes -> two floats (exact)
-__device__ __forceinline__ float2 e4m3x2_to_float2(uint16_t two) {
-    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(two), __NV_E4M3);
-    return __half22float2(*reinterpret_cast<const __half2*>(&h));
+// Four E4M3 codes (one per byte of w, lowest channel in the lowest byte) -> four bf16, exact.  A code
+// s eeee mmm is laid out as the bf16 pattern s 0000eeee mmm0000, which reads (-1)^s 2^(e-127) (1 + m/8) or,
+// for e = 0, the bf16 subnormal (-1)^s 2^-126 m/8; times 2^120 that is the E4M3 value in either case
+// (bias 7, subnormals m 2^-9).  The byte permute also spreads the sign over the byte above each code, so
+// one shift and one mask place all three fields.  The NaN codes 0x7f and 0xff have no place in a cache and
+// read as +-480 here.
+__device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+    uint32_t a, b;
+    asm("prmt.b32 %0, %1, 0, 0x9180;" : "=r"(a) : "r"(w));       // (sign(b1), b1, sign(b0), b0)
+    asm("prmt.b32 %0, %1, 0, 0xb3a2;" : "=r"(b) : "r"(w));       // (sign(b3), b3, sign(b2), b2)
+    a = (a << 4) & 0x87f087f0u;
+    b = (b << 4) & 0x87f087f0u;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(lo) : "r"(a), "r"(0x7b807b80u));   // x 2^120
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(b), "r"(0x7b807b80u));
 }
 
-// AND of `ok` over all NT epilogue threads (named barrier 1): keeps their control flow identical.
-template <int NT>
-__device__ __forceinline__ bool epi_all(bool ok) {
+// AND of `ok` over the NT threads that meet at named barrier ID: keeps their control flow identical.
+template <int ID, int NT>
+__device__ __forceinline__ bool named_all(bool ok) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, %2, q;\n\t"
+        "bar.red.and.pred p, %2, %3, q;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(r)
-        : "r"((uint32_t)ok), "n"(NT)
+        : "r"((uint32_t)ok), "n"(ID), "n"(NT)
         : "memory");
     return r != 0;
 }
+// the epilogue threads' barrier
+template <int NT>
+__device__ __forceinline__ bool epi_all(bool ok) { return named_all<1, NT>(ok); }
 
 template <int D, bool PAIR, bool Q8>
 __global__ void __launch_bounds__(Geo<D, PAIR, Q8>::THREADS, 1)
@@ -267,8 +281,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t s_img = base;
     const uint32_t s_k = s_img + G::IMG_CTA;
-    const uint32_t s_q = s_k + G::NSLOT * kChunkA;                 // staging slots for chunks of codes (Q8)
-    constexpr int kOffOnes = G::IMG_CTA + G::NSLOT * kChunkA + G::NQ * kChunkQ;
+    constexpr int kOffOnes = G::IMG_CTA + G::NSLOT * kChunkA;
     const uint32_t s_ones = base + kOffOnes;
     const uint32_t s_lin = s_ones + G::ONES;
     constexpr int kOffVec = kOffOnes + G::ONES + G::LIN_CTA;
@@ -286,8 +299,7 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
     auto tmem_empty = [&](int a) { return s_bar + 8u * (2 * G::NSLOT + 2 + a); };
     const uint32_t img_full = s_bar + 8u * (2 * G::NSLOT + 4);
     const uint32_t img_peer = s_bar + 8u * (2 * G::NSLOT + 5);
-    auto q_full = [&](int s) { return s_bar + 8u * (2 * G::NSLOT + 6 + s); };           // codes have landed
-    auto q_empty = [&](int s) { return s_bar + 8u * (2 * G::NSLOT + 6 + G::NQ + s); };  // codes have been widened
+    auto q_full = [&](int slot) { return s_bar + 8u * (2 * G::NSLOT + 6 + slot); };     // Q8: the slot's codes have landed
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * G::NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * G::NBAR + 4);
 
@@ -297,13 +309,10 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < G::NSLOT; ++s) {
-            mbar_init(full_k(s), Q8 ? G::CONV_WARPS : 1);          // Q8: the widening warps fill the slot
+            mbar_init(full_k(s), G::FILLERS);                      // Q8: the widening warps fill the slot
             mbar_init(empty_k(s), G::SLOT_READERS);
         }
-        for (int s = 0; s < G::NQ; ++s) {
-            mbar_init(q_full(s), 1);
-            mbar_init(q_empty(s), G::CONV_WARPS);
-        }
+        for (int s = 0; s < G::NQ; ++s) mbar_init(q_full(s), 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(tmem_full(a), 1);
             mbar_init(tmem_empty(a), PAIR ? 2 * G::EPI_WARPS : G::EPI_WARPS);
@@ -387,18 +396,15 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                     for (int kc = 0; ok && kc < G::KCH; ++kc) {
                         const long long c = tile_no * G::KCH + kc;
                         const int slot = slot_of(c);
+                        ok = mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
+                        if (!ok) break;
                         if constexpr (Q8) {
-                            // codes go to a staging slot; the widening warps take it from there to ring slot `slot`
-                            const int qs = (int)(c % G::NQ);
-                            ok = mbar_wait(q_empty(qs), ((uint32_t)(c / G::NQ) & 1) ^ 1, abort_flag);
-                            if (!ok) break;
-                            mbar_arrive_expect_tx(q_full(qs), kChunkQ);
-                            tma_load_3d(s_q + qs * kChunkQ, &k_map, q_full(qs), kc * 64, key0, it.ug);
+                            // codes go to the upper half of the slot; the widening warps spread them over it
+                            mbar_arrive_expect_tx(q_full(slot), kChunkQ);
+                            tma_load_3d(s_k + slot * kChunkA + kChunkQ, &k_map, q_full(slot), kc * 64, key0, it.ug);
                             issued = c + 1;
                             continue;
                         }
-                        ok = mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
-                        if (!ok) break;
                         if (PAIR) {
                             // both CTAs' copies are counted on the leader's barrier, which the MMA issuer watches
                             if (leader) mbar_arrive_expect_tx(full_k(slot), 2 * kChunkA);
@@ -413,9 +419,9 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
                 }
             }
             if (!ok && Q8) {
-                for (int back = 1; back <= G::NQ && back <= issued; ++back) {
+                for (int back = 1; back <= G::NSLOT && back <= issued; ++back) {
                     const long long c = issued - back;
-                    mbar_drain(q_full((int)(c % G::NQ)), (uint32_t)(c / G::NQ) & 1);
+                    mbar_drain(q_full(slot_of(c)), use_of(c) & 1);
                 }
             } else if (!ok && leader) {
                 // Let the copies already in flight land before the shared memory goes away.  In a pair the
@@ -513,10 +519,13 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         __syncwarp();
     } else if (warp >= 2 + G::EPI_WARPS) {
         // ------------------------------------------------------------------ code -> bf16 (Q8)
-        // 128 threads, 512 pieces of 16 codes per chunk: thread t takes pieces t, t + 128, ... (a warp reads
+        // 512 pieces of 16 codes per chunk: thread t takes pieces t, t + 128, ... (a warp reads
         // 512 contiguous bytes); piece (row, u) becomes the 16-byte units 2u and 2u + 1 of the row's 128
-        // bytes in the ring slot, at the swizzled places the MMA and the epilogue expect.
+        // bytes in the slot, at the swizzled places the MMA and the epilogue expect.  The bf16 rows cover the
+        // codes they came from, so every thread holds its codes in registers before any thread writes.
         const int ct = threadIdx.x - 32 * (2 + G::EPI_WARPS);
+        constexpr int kConvThreads = 32 * (G::CONV_WARPS > 0 ? G::CONV_WARPS : 1);
+        constexpr int kPieces = kChunkQ / 16 / kConvThreads;          // 16-code pieces per thread and chunk
         long long tile_no = 0;
         bool ok = true;
         for (long long item = first; ok && item < last; ++item) {
@@ -524,34 +533,39 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
             for (int t = it.tile0; ok && t < it.tile1; ++t, ++tile_no) {
                 for (int kc = 0; ok && kc < G::KCH; ++kc) {
                     const long long c = tile_no * G::KCH + kc;
-                    const int slot = slot_of(c), qs = (int)(c % (G::NQ > 0 ? G::NQ : 1));
-                    ok = mbar_wait(q_full(qs), (uint32_t)(c / (G::NQ > 0 ? G::NQ : 1)) & 1, abort_flag);
-                    ok = ok && mbar_wait(empty_k(slot), (use_of(c) & 1) ^ 1, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    const uint32_t src = s_q + qs * kChunkQ, dst = s_k + slot * kChunkA;
+                    const int slot = slot_of(c);
+                    bool my_ok = mbar_wait(q_full(slot), use_of(c) & 1, abort_flag);
+                    const uint32_t dst = s_k + slot * kChunkA, src = dst + kChunkQ;
+                    uint4 x[kPieces];
+                    if (my_ok) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int piece = ct + 128 * i, r = piece / 4, u = piece % 4;
-                        const uint4 x = lds128(src + piece * 16);
-                        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                        for (int i = 0; i < kPieces; ++i) x[i] = lds128(src + (ct + kConvThreads * i) * 16);
+                    }
+                    // named barrier 2: all codes are in registers (and a wait that gave up stops all four warps)
+                    if (!named_all<2, kConvThreads>(my_ok)) {
+                        ok = false;
+                        break;
+                    }
+#pragma unroll
+                    for (int i = 0; i < kPieces; ++i) {
+                        const int piece = ct + kConvThreads * i, r = piece / 4, u = piece % 4;
                         uint32_t o[8];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float2 lo = e4m3x2_to_float2((uint16_t)(w[q] & 0xffffu));
-                            const float2 hi = e4m3x2_to_float2((uint16_t)(w[q] >> 16));
-                            // exact: the floats' low 16 bits are zero
-                            o[2 * q] = (__float_as_uint(lo.x) >> 16) | (__float_as_uint(lo.y) & 0xffff0000u);
-                            o[2 * q + 1] = (__float_as_uint(hi.x) >> 16) | (__float_as_uint(hi.y) & 0xffff0000u);
-                        }
+                        e4m3x4_to_bf16x4(x[i].x, o[0], o[1]);
+                        e4m3x4_to_bf16x4(x[i].y, o[2], o[3]);
+                        e4m3x4_to_bf16x4(x[i].z, o[4], o[5]);
+                        e4m3x4_to_bf16x4(x[i].w, o[6], o[7]);
                         sts128(dst + r * 128 + (((2 * u) ^ (r & 7)) << 4), make_uint4(o[0], o[1], o[2], o[3]));
                         sts128(dst + r * 128 + (((2 * u + 1) ^ (r & 7)) << 4), make_uint4(o[4], o[5], o[6], o[7]));
                     }
                     fence_proxy_async_smem();          // the MMA reads these bytes through the async proxy
                     __syncwarp();
                     if (lane == 0) {
-                        mbar_arrive(full_k(slot));
-                        mbar_arrive(q_empty(qs));
+                        // In a pair the leader's barrier counts both CTAs' widening warps.  The bytes stay on
+                        // this SM (its own tensor core reads them) and the proxy fence above has completed the
+                        // stores, so the plain remote arrival is enough; a cluster-wide release here stalls the
+                        // warp for about a microsecond per chunk and doubled the kernel's time.
+                        if (PAIR) mbar_arrive_cluster(mapa(full_k(slot), 0));
+                        else mbar_arrive(full_k(slot));
                     }
                 }
             }
@@ -566,7 +580,9 @@ logits_mma_kernel(const __grid_constant__ CUtensorMap k_map, const MmaParams p) 
         const int cp = ew / 4;                     // column part
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        constexpr int BW = D == 256 ? 32 : 16;                      // accumulator columns per tensor-memory load
+        // accumulator columns per tensor-memory load; the widening warps cap the kernel at 128 registers, which
+        // the 32-column form of head_dim 256 does not fit
+        constexpr int BW = (D == 256 && !Q8) ? 32 : 16;
         constexpr int NBW = (G::CPP / BW) * G::HPC;                 // loads per tile for this warp
         constexpr int kEpiThreads = 32 * G::EPI_WARPS;
         const uint32_t empty_remote = PAIR ? mapa(tmem_empty(0), 0) : 0u;
@@ -899,7 +915,7 @@ ea_status ea_launch_logits_mma(const ea_ctx* ctx, const ea_shape& s, const __nv_
     }
 }
 
-bool ea_mma_q8_supported(const ea_shape& s) { return ea_mma_path_supported(s) && s.head_dim <= 128; }
+bool ea_mma_q8_supported(const ea_shape& s) { return ea_mma_path_supported(s); }
 
 ea_status ea_launch_logits_mma_q8(const ea_ctx* ctx, const ea_shape& s, const uint8_t* k_q8,
                                   const ea_quad_form& form, void* image, float* vec, float* logits,
@@ -910,6 +926,8 @@ ea_status ea_launch_logits_mma_q8(const ea_ctx* ctx, const ea_shape& s, const ui
             return launch_mma<64, false, true>(ctx, s, k_q8, form, img, vec, logits, lse_part, n_chunks, st);
         case 128:
             return launch_mma<128, false, true>(ctx, s, k_q8, form, img, vec, logits, lse_part, n_chunks, st);
+        case 256:
+            return launch_mma<256, true, true>(ctx, s, k_q8, form, img, vec, logits, lse_part, n_chunks, st);
         default:
             return EA_ERR_UNSUPPORTED;
     }

@@ -27,7 +27,8 @@ def _np(t):
 @pytest.mark.parametrize("cfg_id,scale,eps,n,mode", [(0, 2.0, 0.02, None, 0), (1, 2.0, 0.02, None, 0), (1, 3.0, 0.0, None, 0),
                                                      (1, 20.0, 0.02, None, 0), (0, 2.0, 0.02, 100, 0), (3, 2.0, 0.02, 3000, 0),
                                                      (0, 2.0, 0.02, None, 1), (0, 2.0, 0.02, None, 2),
-                                                     (2, 2.0, 0.02, 32768, 0), (4, 3.0, 0.0, 4608, 0)])   # full-size layers, codes widened in the kernel
+                                                     (2, 2.0, 0.02, 32768, 0), (4, 3.0, 0.0, 4608, 0),   # full-size layers, codes widened in the kernel
+                                                     (3, 3.0, 0.0, 3000 + 256, 0), (3, 2.0, 0.02, 131072, 0)])
 def test_quantised_whole_path(ea, oracle, cfg_id, scale, eps, n, mode):
     """Window statistics, scores of the quantised cache and compaction of code rows with their value scales,
     against the fp64 oracle on the same codes and scales: log-scores and scores within the tolerance protocol
@@ -72,10 +73,14 @@ def test_quantised_whole_path(ea, oracle, cfg_id, scale, eps, n, mode):
                score_worst_rel=float((np.abs(_np(sc) - ref["scores"]) / np.maximum(ref["scores"], 1e-300)).max())))
 
 
-def test_unit_scales_reproduce_the_bf16_path_bitwise(ea):
+@pytest.mark.parametrize("cfg_id,n", [(0, None), (1, None), (3, 5000), (3, 131072)])
+def test_unit_scales_reproduce_the_bf16_path_bitwise(ea, cfg_id, n):
     """With all scales one the quantised entry points see the same numbers as the bf16 ones: same log-scores
-    bit for bit (the codes are widened without rounding, the folded scales are ones)."""
-    cfg = inputs.CONFIGS[1].tempered(2.0)
+    bit for bit (the codes are widened without rounding, the folded scales are ones), at every head_dim the
+    tensor-core kernel has a form for."""
+    cfg = inputs.CONFIGS[cfg_id].tempered(2.0)
+    if n is not None:
+        cfg = dataclasses.replace(cfg, n_layers=1, n_keys=n, n_kept=n // 2)
     q, k, v, pos = inputs.generate_layer(cfg, device="cuda")
     kq, ks, vq, vs = inputs.quantize_e4m3(k, v)
     ks.fill_(1.0), vs.fill_(1.0)

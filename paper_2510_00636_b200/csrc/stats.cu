@@ -36,13 +36,31 @@ __global__ void rope_coef_kernel(const int64_t* __restrict__ pos_next, int n_uni
 // mma.sync.m16n8k16 (bf16 x bf16 -> fp32).  X is kept as a bf16 pair (hi, lo) and three products
 // (hi.hi + hi.lo + lo.hi) are accumulated, so every product carries 16 significant bits of each
 // factor; the lower triangle is a copy of the upper one, which makes the result bitwise symmetric.
+// X is staged as it lies, [window row][channel]: both MMA operands want the window index as their
+// contraction index, which ldmatrix.trans delivers from that layout, so nothing is transposed on the way.
 constexpr int kKC = 32;            // window rows per shared-memory chunk
-constexpr int kXtPitch = 40;       // bf16 per row of the transposed chunk: 80 bytes, conflict-free for ldmatrix
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+// four 8x8 bf16 matrices, each stored as 8 rows (contraction index) of 8 contiguous elements, transposed
+// into the fragment layout of mma.m16n8k16
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
+}
+// eight consecutive channels of a window row
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -63,34 +81,63 @@ struct StatsImage {
     float quad_scale;    // 1 / (2 d)
 };
 
-template <int D, typename QT>
-constexpr int stats_smem_bytes() {
-    constexpr int BM = D < 128 ? D : 128;
-    return 2 * 2 * BM * kXtPitch * 2 + kKC * D * (int)sizeof(QT) + (D + D) * 4 + (256 / (D / 2)) * D * 4;
-}
+// Shared memory: the staged chunk (hi and lo, kKC rows of the block's channels, padded by 16 bytes so that
+// the eight rows of an 8x8 matrix fall into different banks), which the fused image's tile reuses; then
+// the mean, the averaged rotation and the partial sums of the mean.
+template <int D>
+struct StatsGeo {
+    static constexpr int BM = D < 128 ? D : 128;          // block edge
+    static constexpr int NB1 = D / BM;                    // blocks per edge (1 or 2)
+    static constexpr int PITCH = (NB1 == 1 ? BM : 2 * BM) + 8;       // bf16 per staged window row
+    static constexpr int STAGE = 2 * kKC * PITCH * 2;
+    static constexpr int TILE = NB1 == 1 ? EaImage<D>::KCH * D * 128 : 0;
+    static constexpr int REGION = STAGE > TILE ? STAGE : TILE;
+    static constexpr int SMEM = REGION + (D + D) * 4 + (256 / (D / 2)) * D * 4;
+};
 
-__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
-__device__ __forceinline__ float to_f32(float x) { return x; }
+// packed fp32 pair arithmetic (two lanes per instruction)
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)), "l"(reinterpret_cast<uint64_t&>(c)));
+    return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+    float2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;"
+        : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
+    return d;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
+    float2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;"
+        : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
+    return d;
+}
+// eight consecutive floats from shared memory, 16-byte aligned
+__device__ __forceinline__ void lds8(const float* p, float (&v)[8]) {
+    const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
 
 // QT: the window queries as bf16 (what a model's query projection emits) or fp32 (from project_kernel).
 template <int D, typename QT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
                  int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar,
                  int w_cap, const long long* __restrict__ pushed, int cov_sample, const StatsImage img) {
+    using SG = StatsGeo<D>;
     constexpr int HALF = D / 2;
-    constexpr int BM = D < 128 ? D : 128;          // block edge
-    constexpr int NB1 = D / BM;                    // blocks per edge (1 or 2)
+    constexpr int BM = SG::BM, NB1 = SG::NB1, P = SG::PITCH;
     constexpr int WM = BM / 2, WN = BM / 4;        // warp tile: 2 x 4 warps
     constexpr int TM = WM / 16, TN = WN / 8;       // mma tiles per warp
-    // dynamic shared memory: the transposed (hi, lo) chunk, the raw window chunk, the mean, R_bar
     extern __shared__ __align__(16) unsigned char stats_smem[];
-    // [hi / lo][row: BM channels of the block's rows, then BM channels of its columns][w in chunk]
-    typedef __nv_bfloat16 (*xt_t)[2 * BM][kXtPitch];
-    xt_t xt = reinterpret_cast<xt_t>(stats_smem);
-    constexpr int kXtBytes = 2 * 2 * BM * kXtPitch * 2;
-    QT* raw = reinterpret_cast<QT*>(stats_smem + kXtBytes);                                // [kKC][D]
-    float* mu_s = reinterpret_cast<float*>(stats_smem + kXtBytes + kKC * D * sizeof(QT));  // [D]
+    // [hi / lo][w in chunk][channel: BM channels of the block's rows, then (off the diagonal) of its columns]
+    float* mu_s = reinterpret_cast<float*>(stats_smem + SG::REGION);                        // [D]
     float* c_s = mu_s + D;                                                                  // [HALF]
     float* s_s = c_s + HALF;                                                                // [HALF]
     float* red = s_s + HALF;                                                                // [256 / (D/2)][D]
@@ -173,51 +220,68 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
             for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
 
     const int wm = warp / 4, wn = warp % 4;        // warp position in the block
-    const int n_rows = diag ? BM : 2 * BM;         // channel rows staged per chunk
-    const uint32_t xt_hi = static_cast<uint32_t>(__cvta_generic_to_shared(&xt[0][0][0]));
-    const uint32_t xt_lo = static_cast<uint32_t>(__cvta_generic_to_shared(&xt[1][0][0]));
-    const uint4* q4 = reinterpret_cast<const uint4*>(q);
-    uint4* raw4 = reinterpret_cast<uint4*>(raw);
+    const int n_ch = diag ? BM : 2 * BM;           // channels staged per chunk
+    const uint32_t xs_hi = static_cast<uint32_t>(__cvta_generic_to_shared(stats_smem));
+    const uint32_t xs_lo = xs_hi + kKC * P * 2;
 
-    // this thread's channel of the staged rows (the block's rows, then its columns), its rotation partner
-    // and the two coefficients of x = (R_bar (u - mu))[ch] = t_c (u_ch - mu_ch) + t_s (u_partner - mu_partner)
-    const int t_r = tid % n_rows, t_w = tid / n_rows, t_wstep = 256 / n_rows;
-    const int t_ch = (t_r < BM ? bi * BM : bj * BM - BM) + t_r;
-    int t_m, t_partner;
-    bool t_first;                                                   // t_ch is the first channel of its rotation pair
-    if (layout == EA_ROPE_INTERLEAVED) { t_m = t_ch >> 1; t_first = (t_ch & 1) == 0; t_partner = t_ch ^ 1; }
-    else { t_m = t_ch < HALF ? t_ch : t_ch - HALF; t_first = t_ch < HALF; t_partner = t_first ? t_ch + HALF : t_ch - HALF; }
-    const float t_mu = mu_s[t_ch], t_mu_partner = mu_s[t_partner];
-    const float t_c = c_s[t_m], t_s = t_first ? -s_s[t_m] : s_s[t_m];
+    // This thread's eight staged channels (one 16-byte piece of a row; the same for the whole kernel), the
+    // channels they rotate with, and where the averaged rotation's coefficients of the pairs start:
+    //   x[ch] = c_m (u_ch - mu_ch) -/+ s_m (u_partner - mu_partner),  minus for the first channel of a pair.
+    const int pieces = n_ch / 8, t_p = tid % pieces, t_w = tid / pieces, t_wstep = 256 / pieces;
+    const int sc0 = 8 * t_p;
+    const int ch0 = (sc0 < BM ? bi * BM : bj * BM - BM) + sc0;
+    const bool interleaved = layout == EA_ROPE_INTERLEAVED;
+    const bool first_side = ch0 < HALF;                      // (half-split layout) the piece holds first channels
+    const int pch0 = interleaved ? ch0 : (first_side ? ch0 + HALF : ch0 - HALF);
+    const int m0 = interleaved ? ch0 / 2 : (first_side ? ch0 : ch0 - HALF);
 
     for (int w0 = 0; w0 < W; w0 += kKC) {
         __syncthreads();
-        // the raw chunk with 128-bit loads (rows past the window read as zero) ...
-        constexpr int kRowPieces = D * (int)sizeof(QT) / 16;      // 16-byte pieces per window row
-        for (int e = tid; e < kKC * kRowPieces; e += 256) {
-            const int w = e / kRowPieces;
-            raw4[e] = w0 + w < W ? __ldg(q4 + (size_t)w0 * kRowPieces + e) : make_uint4(0u, 0u, 0u, 0u);
-        }
-        __syncthreads();
-        // ... then x[w][ch] = (R_bar (u_w - mu))[ch] transposed, as bf16 hi and lo
-        // (a thread keeps one channel for the whole kernel: n_rows divides the block size)
-        // two neighbouring window rows per step: one 32-bit store per (hi, lo)
-        for (int w = 2 * t_w; w < kKC; w += 2 * t_wstep) {
-            __nv_bfloat162 hi2, lo2;
+        for (int w = t_w; w < kKC; w += t_wstep) {
+            uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
+            if (w0 + w < W) {
+                float uo[8], up[8];
+                load8(q + (size_t)(w0 + w) * D + ch0, uo);
+                if (interleaved) {
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                float x = 0.f;
-                if (w0 + w + k < W) {
-                    const float xa = to_f32(raw[(w + k) * D + t_ch]) - t_mu;
-                    const float xb = to_f32(raw[(w + k) * D + t_partner]) - t_mu_partner;
-                    x = t_c * xa + t_s * xb;
+                    for (int i = 0; i < 8; ++i) up[i] = uo[i ^ 1];
+                } else {
+                    load8(q + (size_t)(w0 + w) * D + pch0, up);
                 }
-                const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
-                if (k == 0) { hi2.x = hi; lo2.x = lo; } else { hi2.y = hi; lo2.y = lo; }
+                float mo[8], mp[8], cm[8], sm[8];
+                lds8(mu_s + ch0, mo);
+                // (interleaved pairs: four coefficient pairs serve the piece; the second half of these loads is
+                // not used and may run four entries into the array that follows in shared memory)
+                lds8(mu_s + pch0, mp);
+                lds8(c_s + m0, cm);
+                lds8(s_s + m0, sm);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // two channels at a time with packed fp32 arithmetic and packed conversions
+                    float2 tc, ts, mpp;
+                    if (interleaved) {
+                        tc = make_float2(cm[i], cm[i]);
+                        ts = make_float2(-sm[i], sm[i]);
+                        mpp = make_float2(mp[2 * i + 1], mp[2 * i]);
+                    } else {
+                        tc = make_float2(cm[2 * i], cm[2 * i + 1]);
+                        ts = first_side ? make_float2(-sm[2 * i], -sm[2 * i + 1]) : make_float2(sm[2 * i], sm[2 * i + 1]);
+                        mpp = make_float2(mp[2 * i], mp[2 * i + 1]);
+                    }
+                    const float2 xa = sub2(make_float2(uo[2 * i], uo[2 * i + 1]), make_float2(mo[2 * i], mo[2 * i + 1]));
+                    const float2 xb = sub2(make_float2(up[2 * i], up[2 * i + 1]), mpp);
+                    const float2 x = fma2(tc, xa, mul2(ts, xb));
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(x.x, x.y);
+                    const uint32_t hb = *reinterpret_cast<const uint32_t*>(&h);
+                    const float2 r = sub2(x, make_float2(__uint_as_float(hb << 16), __uint_as_float(hb & 0xffff0000u)));
+                    const __nv_bfloat162 l = __floats2bfloat162_rn(r.x, r.y);
+                    hi[i] = hb;
+                    lo[i] = *reinterpret_cast<const uint32_t*>(&l);
+                }
             }
-            *reinterpret_cast<__nv_bfloat162*>(&xt[0][t_r][w]) = hi2;
-            *reinterpret_cast<__nv_bfloat162*>(&xt[1][t_r][w]) = lo2;
+            // rows past the window are zero
+            *reinterpret_cast<uint4*>(stats_smem + (w * P + sc0) * 2) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(stats_smem + ((kKC + w) * P + sc0) * 2) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
         __syncthreads();
 #pragma unroll
@@ -225,19 +289,22 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
             uint32_t a_hi[TM][4], a_lo[TM][4];
 #pragma unroll
             for (int i = 0; i < TM; ++i) {
-                const int row = wm * WM + i * 16 + (lane % 8) + 8 * ((lane / 8) % 2);
-                const uint32_t off = (uint32_t)((row * kXtPitch + k0 + 8 * (lane / 16)) * 2);
-                ldmatrix_x4(xt_hi + off, a_hi[i]);
-                ldmatrix_x4(xt_lo + off, a_lo[i]);
+                // matrices: (channels +0, w +0), (channels +8, w +0), (channels +0, w +8), (channels +8, w +8)
+                const int kr = k0 + (lane % 8) + 8 * (lane / 16);
+                const int mc = wm * WM + i * 16 + 8 * ((lane / 8) % 2);
+                const uint32_t off = (uint32_t)((kr * P + mc) * 2);
+                ldmatrix_x4_trans(xs_hi + off, a_hi[i]);
+                ldmatrix_x4_trans(xs_lo + off, a_lo[i]);
             }
 #pragma unroll
             for (int j2 = 0; j2 < TN; j2 += 2) {
-                // two 8-channel column tiles per ldmatrix.x4
+                // two 8-channel column tiles per load: (tile 0, w +0), (tile 0, w +8), (tile 1, w +0), (tile 1, w +8)
                 uint32_t b_hi[4], b_lo[4];
-                const int row = (diag ? 0 : BM) + wn * WN + j2 * 8 + (lane % 8) + 8 * (lane / 16);
-                const uint32_t off = (uint32_t)((row * kXtPitch + k0 + 8 * ((lane / 8) % 2)) * 2);
-                ldmatrix_x4(xt_hi + off, b_hi);
-                ldmatrix_x4(xt_lo + off, b_lo);
+                const int kr = k0 + (lane % 8) + 8 * ((lane / 8) % 2);
+                const int nc = (diag ? 0 : BM) + wn * WN + j2 * 8 + 8 * (lane / 16);
+                const uint32_t off = (uint32_t)((kr * P + nc) * 2);
+                ldmatrix_x4_trans(xs_hi + off, b_hi);
+                ldmatrix_x4_trans(xs_lo + off, b_lo);
 #pragma unroll
                 for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -366,9 +433,9 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
     };
     bool ok;
     switch (d) {
-        case 64: ok = launch(stats_mma_kernel<64, QT>, stats_smem_bytes<64, QT>(), 1); break;
-        case 128: ok = launch(stats_mma_kernel<128, QT>, stats_smem_bytes<128, QT>(), 1); break;
-        case 256: ok = launch(stats_mma_kernel<256, QT>, stats_smem_bytes<256, QT>(), 3); break;
+        case 64: ok = launch(stats_mma_kernel<64, QT>, StatsGeo<64>::SMEM, 1); break;
+        case 128: ok = launch(stats_mma_kernel<128, QT>, StatsGeo<128>::SMEM, 1); break;
+        case 256: ok = launch(stats_mma_kernel<256, QT>, StatsGeo<256>::SMEM, 3); break;
         default: return EA_ERR_UNSUPPORTED;
     }
     if (!ok) return EA_ERR_CUDA;

@@ -34,10 +34,12 @@ from paper_2510_00636_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the log-score kernel divided by the
 # key-slots of that launch (one ncu --set full capture per shape on a few layers, clocks not locked),
-# keyed by (head_dim, query heads per KV head): the log-score write and the sharing of key tiles depend
-# on both.  NCU_CAPTURE_SOURCE is the fingerprint of the kernel source that was captured.
-NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2): 1.10309e9 / 2097152, (128, 4): 293.78e6 / 1048576}
-NCU_CAPTURE_SOURCE = "d9ac1f115e3f6ed1"
+# keyed by (head_dim, query heads per KV head, cache format): the log-score write, the sharing of key
+# tiles and the bytes of a key depend on them.  NCU_CAPTURE_SOURCE is the fingerprint of the kernel
+# source that was captured.
+NCU_DRAM_BYTES_PER_KEY_SLOT = {(256, 2, "bf16"): 1.101994e9 / 2097152, (128, 4, "bf16"): 293.660e6 / 1048576,
+                               (256, 2, "fp8"): 563.424e6 / 2097152}
+NCU_CAPTURE_SOURCE = "e185e5558dd2cd61"
 # nominal figures of the part, reported beside the measured denominators
 NOMINAL_HBM_GBS, NOMINAL_TFLOPS = 8000.0, 2250.0
 
@@ -530,7 +532,7 @@ def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_work
     # DRAM bytes per launch from an ncu capture of this kernel on a few layers of the same shapes, scaled by
     # the key-slots of a launch (traffic is proportional to them); null when the kernel's source is no
     # longer the one that was captured
-    captured = NCU_DRAM_BYTES_PER_KEY_SLOT.get((cfg.head_dim, cfg.group))
+    captured = NCU_DRAM_BYTES_PER_KEY_SLOT.get((cfg.head_dim, cfg.group, args.kv_dtype))
     fresh = captured is not None and NCU_CAPTURE_SOURCE == source_fingerprint()
     traffic = captured * slots / n_calls if fresh else None
     sm_mhz = clocks.get("sm_mhz")
@@ -673,6 +675,17 @@ def main():
         others[inputs.CONFIGS[4].name]["unordered_compaction_fused_statistics"] = {
             "ms_per_step": om["ms"], "value": om["slots"] / (om["ms"] * 1e-3) / 1e9,
             "path_roofline_frac": om["path_roofline"]["frac"]}
+        # the headline shapes with the cache held as FP8 E4M3 codes (its own algorithmic bytes)
+        args.kv_dtype = "fp8"
+        om = measure(args, cfg, ea, device, world, local, peaks, max(5, args.steps // 2), 3, keep_workload=False)
+        args.kv_dtype = "bf16"
+        others[cfg.name + ", FP8 E4M3 cache"] = {
+            "ms_per_step": om["ms"], "value": om["slots"] / (om["ms"] * 1e-3) / 1e9, "unit": UNIT,
+            "path_roofline_frac": om["path_roofline"]["frac"],
+            "path_roofline_frac_nominal": om["path_roofline"]["frac_nominal"],
+            "kernel_frac": om["roofline"]["frac"], "kernel_ms": om["roofline"]["kernel_ms"],
+            "kernel_mcycles": om["roofline"]["kernel_mcycles"], "traffic": om["roofline"]["traffic"],
+            "sm_mhz": om["clocks"]["sm_mhz"], "gpu_launches": om["gpu_launches"]}
         result["other_configs"] = others
 
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:

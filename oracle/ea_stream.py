@@ -11,12 +11,15 @@ eviction rule).  Nothing here is arithmetic of its own: appending is concatenati
 Parity status: plumbing around pinned functions; pinned itself (``tests/test_oracle_pins.py``) by a
 one-event stream reproducing ``compress`` on the concatenated inputs, by the window equalling the
 tail of everything pushed, and by the kept rows of consecutive events composing as index maps.
+``QuantStreamOracle`` is the same driver on a quantised cache (``ea_quant``): pinned by a one-event
+stream reproducing ``ea_quant.compress`` on the concatenated codes and scales, and by a stream with
+unit scales walking through the same kept indices as ``StreamOracle`` on the decoded values.
 """
 from __future__ import annotations
 
 import numpy as np
 
-from oracle import ea_oracle
+from oracle import ea_oracle, ea_quant
 
 
 def fill_holes(kept_idx, n_kept: int):
@@ -74,3 +77,45 @@ class StreamOracle:
         idx = np.asarray(kept_idx)
         self.k = ea_oracle.gather(self.k, idx)
         self.v = ea_oracle.gather(self.v, idx)
+
+
+class QuantStreamOracle:
+    """The same driver on a quantised cache: codes ``k_q8, v_q8`` uint8 [U, Hkv, n, d], one key scale per
+    channel ``k_scale`` [U, Hkv, d] that stays with the cache, one value scale per token ``v_scale`` [U, Hkv, n]
+    that travels with its row.  New pairs arrive as codes against the cache's key scales."""
+
+    def __init__(self, k_q8, k_scale, v_q8, v_scale, window: int, budget: int):
+        self.k = np.ascontiguousarray(k_q8)
+        self.v = np.ascontiguousarray(v_q8)
+        self.k_scale = np.ascontiguousarray(k_scale)
+        self.v_scale = np.ascontiguousarray(v_scale)
+        self.window, self.budget = int(window), int(budget)
+        self.q = None
+
+    @property
+    def n_keys(self) -> int:
+        return self.k.shape[2]
+
+    def append(self, k_new_q8, v_new_q8, v_scale_new):
+        self.k = np.concatenate([self.k, k_new_q8], axis=2)
+        self.v = np.concatenate([self.v, v_new_q8], axis=2)
+        self.v_scale = np.concatenate([self.v_scale, v_scale_new], axis=2)
+
+    def push_queries(self, q_new_bits):
+        q = q_new_bits if self.q is None else np.concatenate([self.q, q_new_bits], axis=2)
+        self.q = np.ascontiguousarray(q[:, :, -self.window:])
+
+    def compress(self, pos_next, n_future, rope_base, eps, group_mode=ea_oracle.GROUP_MEAN_PROB):
+        """One event on what the buffers hold: ``ea_quant.compress``'s dict; the cache is NOT replaced."""
+        n_kept = min(self.n_keys, self.budget)
+        return ea_quant.compress(self.q, self.k, self.k_scale, self.v, self.v_scale,
+                                 np.asarray(pos_next, dtype=np.int64), n_future, rope_base, eps, n_kept,
+                                 group_mode=group_mode)
+
+    def keep(self, kept_idx):
+        """Replace every head's cache by its rows ``kept_idx`` [U, Hkv, n_kept], in that order; the value
+        scales follow their rows, the key scales stay."""
+        i64 = np.asarray(kept_idx).astype(np.int64)
+        self.k = np.take_along_axis(self.k, i64[..., None], axis=2)
+        self.v = np.take_along_axis(self.v, i64[..., None], axis=2)
+        self.v_scale = np.take_along_axis(self.v_scale, i64, axis=2)

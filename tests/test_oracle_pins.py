@@ -681,3 +681,48 @@ def test_fill_holes_is_a_permutation_of_the_kept_set_that_moves_only_the_tail(or
     assert np.array_equal(np.sort(where, axis=-1), idx)
     ident = fill_holes(np.broadcast_to(np.arange(20, dtype=np.int32), (2, 3, 20)), 20)
     assert np.array_equal(ident, np.broadcast_to(np.arange(20), (2, 3, 20)))
+
+
+# ------------------------------------------------------------------------------------------
+# Streaming on a quantised cache (oracle/ea_stream.py, QuantStreamOracle)
+def test_quantised_stream_single_event_is_quantised_compress_on_the_concatenated_inputs(oracle):
+    from oracle import ea_quant
+    from oracle.ea_stream import QuantStreamOracle
+    q, kq, ks, vq, vs = _quant_case(21, U=1, n=96, W=16)
+    st = QuantStreamOracle(kq[:, :, :60], ks, vq[:, :, :60], vs[:, :, :60], window=16, budget=50)
+    st.append(kq[:, :, 60:], vq[:, :, 60:], vs[:, :, 60:])
+    st.push_queries(q)
+    got = st.compress([96], 8, 1e4, 0.02)
+    want = ea_quant.compress(q, kq, ks, vq, vs, np.array([96]), 8, 1e4, 0.02, 50)
+    assert np.array_equal(got["kept_idx"], want["kept_idx"]) and np.array_equal(got["scores"], want["scores"])
+    st.keep(got["kept_idx"])
+    assert st.n_keys == 50
+    assert np.array_equal(st.k, want["k_out"]) and np.array_equal(st.v, want["v_out"])
+    assert np.array_equal(st.v_scale, want["v_scale_out"]) and np.array_equal(st.k_scale, ks)
+
+
+def test_quantised_stream_with_unit_scales_walks_with_the_bf16_stream(oracle):
+    """E4M3 values are bf16 values: with all scales one, three events of the quantised driver keep the same rows
+    as the bf16 driver on the decoded values, and the caches stay decodings of one another."""
+    from oracle import ea_quant
+    from oracle.ea_stream import QuantStreamOracle, StreamOracle
+    to_bf16 = lambda codes: (ea_quant.e4m3_decode(codes).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    q, kq, ks, vq, vs = _quant_case(22, U=1, n=160, W=12)
+    ks[:], vs[:] = 1.0, 1.0
+    qs = QuantStreamOracle(kq[:, :, :40], ks, vq[:, :, :40], vs[:, :, :40], window=12, budget=48)
+    bs = StreamOracle(to_bf16(kq[:, :, :40]), to_bf16(vq[:, :, :40]), window=12, budget=48)
+    rng = np.random.default_rng(5)
+    for e in range(3):
+        lo, hi = 40 + 40 * e, 80 + 40 * e
+        qs.append(kq[:, :, lo:hi], vq[:, :, lo:hi], vs[:, :, lo:hi])
+        bs.append(to_bf16(kq[:, :, lo:hi]), to_bf16(vq[:, :, lo:hi]))
+        qn = (rng.normal(size=(1, 4, 7, 64)).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+        qs.push_queries(qn)
+        bs.push_queries(qn)
+        a, b = qs.compress([hi], 8, 1e4, 0.02), bs.compress([hi], 8, 1e4, 0.02)
+        np.testing.assert_allclose(a["scores"], b["scores"], rtol=1e-12, atol=0)
+        assert np.array_equal(a["kept_idx"], b["kept_idx"])
+        qs.keep(a["kept_idx"])
+        bs.keep(b["kept_idx"])
+        assert np.array_equal(to_bf16(qs.k), bs.k) and np.array_equal(to_bf16(qs.v), bs.v)
+        assert (qs.v_scale == 1.0).all() and qs.v_scale.shape == (1, 2, qs.n_keys)

@@ -250,9 +250,12 @@ class DecodeWorkload:
     by the previous step: synthetic rows of the same distribution)."""
 
     def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False,
-                 unordered: bool = False, fused: bool = False):
+                 unordered: bool = False, fused: bool = False, fp8: bool = False):
         import dataclasses
         self.cfg, self.device, self.ea = cfg, device, ea
+        self.fp8 = fp8                      # the carried cache holds FP8 E4M3 codes with scales (the _q8 calls)
+        if fp8 and fused:
+            raise SystemExit("--fused-stats builds the image without key scales: not with --kv-dtype fp8")
         self.fused = fused                  # ea_set_fused_stats: no sigma_bar round trip, no image kernel
         self.unordered = unordered          # ea_select_compact_inplace_unordered: only the tail's kept rows move
         self.use_graph, self.graphs = use_graph, {}
@@ -263,16 +266,25 @@ class DecodeWorkload:
         U, Hq, Hkv, d, W = L * B, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
         bf, f32 = torch.bfloat16, torch.float32
         self.n_units = U
-        self.k = torch.empty((U, Hkv, self.cap, d), dtype=bf, device=device)
-        self.v = torch.empty((U, Hkv, self.cap, d), dtype=bf, device=device)
+        kv_dtype = torch.uint8 if fp8 else bf
+        self.k = torch.empty((U, Hkv, self.cap, d), dtype=kv_dtype, device=device)
+        self.v = torch.empty((U, Hkv, self.cap, d), dtype=kv_dtype, device=device)
+        if fp8:
+            self.k_scale = torch.empty((U, Hkv, d), dtype=f32, device=device)
+            self.v_scale = torch.empty((U, Hkv, self.cap), dtype=f32, device=device)
         for layer in range(L):
             _, kk, vv, _ = inputs.generate_layer(dataclasses.replace(cfg, window=1), layer=layer, device=device,
                                                  n_keys=self.cap, draw=1)
-            self.k[layer * B:(layer + 1) * B], self.v[layer * B:(layer + 1) * B] = kk, vv
-        self.new_k, self.new_v, self.new_q = [], [], []
+            sl = slice(layer * B, (layer + 1) * B)
+            if fp8:
+                self.k[sl], self.k_scale[sl], self.v[sl], self.v_scale[sl] = inputs.quantize_e4m3(kk, vv)
+            else:
+                self.k[sl], self.v[sl] = kk, vv
+        self.new_k, self.new_v, self.new_q, self.new_vs = [], [], [], []
         for ph in range(n_phases):
-            nk = torch.empty((U, Hkv, self.every, d), dtype=bf, device=device)
+            nk = torch.empty((U, Hkv, self.every, d), dtype=kv_dtype, device=device)
             nv = torch.empty_like(nk)
+            nvs = torch.empty((U, Hkv, self.every), dtype=f32, device=device) if fp8 else None
             nq = torch.empty((U, Hq, W, d), dtype=bf, device=device)
             pos = 2048 + ph * self.every
             for layer in range(L):
@@ -280,8 +292,12 @@ class DecodeWorkload:
                                                       key_positions=torch.arange(pos, pos + self.every),
                                                       q_phase=2 * 3.141592653589793 / 64 * ph)
                 sl = slice(layer * B, (layer + 1) * B)
-                nk[sl], nv[sl], nq[sl] = kk, vv, qq
-            self.new_k.append(nk), self.new_v.append(nv), self.new_q.append(nq)
+                if fp8:         # new pairs arrive coded against the cache's key scales
+                    nk[sl], _, nv[sl], nvs[sl] = inputs.quantize_e4m3(kk, vv, k_scale=self.k_scale[sl])
+                    nq[sl] = qq
+                else:
+                    nk[sl], nv[sl], nq[sl] = kk, vv, qq
+            self.new_k.append(nk), self.new_v.append(nv), self.new_q.append(nq), self.new_vs.append(nvs)
         self.ring = torch.zeros((U, Hq, W, d), dtype=bf, device=device)
         self.pushed = torch.zeros((U,), dtype=torch.int64, device=device)
         self.pos = [torch.full((U,), pos, dtype=torch.int64, device=device) for pos, _, _ in self.events]
@@ -305,6 +321,16 @@ class DecodeWorkload:
         shape = self._shape(n)
         scores = self.scores.view(-1)[:self.n_units * cfg.n_kv_heads * n].view(self.n_units, cfg.n_kv_heads, n)
         idx = self.idx.view(-1)[:self.n_units * cfg.n_kv_heads * kept].view(self.n_units, cfg.n_kv_heads, kept)
+        if self.fp8:
+            ea.ea_cache_append_q8(ctx, self._shape(n - self.every), self.k, self.v, self.v_scale, self.new_k[ph],
+                                  self.new_v[ph], self.new_vs[ph])
+            ea.ea_window_push(ctx, shape, self.ring, self.pushed, self.new_q[ph])
+            ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
+            ea.ea_score_q8(ctx, shape, self.k, self.k_scale, self.v, self.v_scale, self.mu, self.sigma, cfg.eps,
+                           scores=scores)
+            ea.ea_select_compact_inplace_q8(ctx, shape, scores, kept, self.k, self.v, self.v_scale, idx,
+                                            unordered=self.unordered)
+            return
         ea.ea_cache_append(ctx, self._shape(n - self.every), self.k, self.v, self.new_k[ph], self.new_v[ph])
         ea.ea_window_push(ctx, shape, self.ring, self.pushed, self.new_q[ph])
         if self.fused:
@@ -349,7 +375,8 @@ class DecodeWorkload:
         cfg = self.cfg
         per_head = self.n_units * cfg.n_kv_heads
         slots = sum(per_head * n for _, n, _ in self.events)
-        bytes_ = slots * 4 * cfg.head_dim + sum(per_head * kept for _, _, kept in self.events) * 4 * cfg.head_dim
+        row = (2 if self.fp8 else 4) * cfg.head_dim          # bytes of a K row plus a V row
+        bytes_ = slots * row + sum(per_head * kept for _, _, kept in self.events) * row
         return slots, bytes_, slots * 2 * cfg.head_dim ** 2 * cfg.group
 
 
@@ -470,7 +497,8 @@ def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_work
         gc.collect()
         torch.cuda.empty_cache()
     decode = cfg.cfg_id == 4
-    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph, unordered=args.unordered, fused=args.fused_stats) if decode else Workload(cfg, device, ea, args.head_adaptive,
+    wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph, unordered=args.unordered, fused=args.fused_stats,
+                        fp8=args.kv_dtype == "fp8") if decode else Workload(cfg, device, ea, args.head_adaptive,
                                                                  args.hidden_stats, args.with_wo, args.kv_dtype == "fp8")
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
@@ -616,7 +644,7 @@ def main():
     ea.lib()
 
     variant = args.head_adaptive is not None or args.hidden_stats or args.with_wo or args.kv_dtype == "fp8"
-    if variant and cfg.cfg_id == 4:
+    if (args.head_adaptive is not None or args.hidden_stats or args.with_wo) and cfg.cfg_id == 4:
         raise SystemExit("--head-adaptive, --hidden-stats and --with-wo apply to the prefill configs")
     if variant or cfg.cfg_id == 4:
         args.skip_e2e = True           # the host-buffer entry point runs the three basic calls on a prefill cache

@@ -273,10 +273,10 @@ ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const v
  * core kernel runs on the codes, widened to bf16 without rounding; the value
  * norm is v_scale_i ||x_i||.
  *
- * k_q8, v_q8  uint8 [n_units, Hkv, n, d] E4M3 codes, 16-byte aligned, dense
- *             (kv_capacity must be 0 or n_keys: EA_ERR_UNSUPPORTED otherwise)
- * k_scale     fp32 [n_units, Hkv, d];   v_scale  fp32 [n_units, Hkv, n]
- * k_scratch   bf16 [n_units, Hkv, n, d]  caller-owned scratch for the widened key
+ * k_q8, v_q8  uint8 [n_units, Hkv, cap, d] E4M3 codes, 16-byte aligned; cap = kv_capacity
+ *             (n_keys when that is 0): the first n_keys rows of a head's range are its cache
+ * k_scale     fp32 [n_units, Hkv, d];   v_scale  fp32 [n_units, Hkv, cap]
+ * k_scratch   bf16 [n_units, Hkv, cap, d]  caller-owned scratch for the widened key
  *             codes.  Needed, and written, only where the tensor-core kernel,
  *             which widens the codes itself, does not take the shape (fewer
  *             keys than one tile: 128, or 256 at head_dim 256; query groups of
@@ -293,13 +293,41 @@ ea_status ea_score_q8_scratch_bytes(const ea_shape* shape, size_t* bytes);
 /*
  * ea_select_compact on a quantised cache: the same selection, then the kept
  * code rows and the value scales of their tokens are gathered (the key scales
- * belong to the channels and stay as they are).
+ * belong to the channels and stay as they are).  The source may sit in a
+ * larger buffer (kv_capacity); the outputs are dense.
  * k_out, v_out  uint8 [n_units, Hkv, n_kept, d];  v_scale_out fp32 [n_units, Hkv, n_kept]
  */
 ea_status ea_select_compact_q8(ea_ctx* ctx, const ea_shape* shape, const float* scores,
                                int32_t n_kept, const void* k_q8, const void* v_q8,
                                const float* v_scale, int32_t* kept_idx, void* k_out, void* v_out,
                                float* v_scale_out, void* cuda_stream);
+/*
+ * Streaming decode on a quantised cache (the decoding set-up of Sec. 4 with
+ * the format above): the two calls that let one buffer of codes live through
+ * consecutive compression events, beside ea_window_push / ea_query_stats_ring
+ * and ea_score_q8 with kv_capacity.
+ *
+ * ea_cache_append_q8: n_new code rows per head, k_new / v_new uint8
+ * [n_units, Hkv, n_new, d] with their value scales v_scale_new fp32
+ * [n_units, Hkv, n_new], go behind the shape->n_keys rows each head holds;
+ * the new key codes are codes against the cache's own key scales.
+ * n_keys + n_new > capacity: EA_ERR_INVALID_ARG.  Device pointers, 16-byte
+ * aligned codes; asynchronous on cuda_stream.
+ *
+ * ea_select_compact_inplace_q8: ea_select_compact_inplace (unordered == 0:
+ * kept rows move to the front of the head's range in ascending order of
+ * position, kept_idx ascending) or ea_select_compact_inplace_unordered
+ * (unordered != 0: kept rows beyond n_kept fill the evicted positions below
+ * it; kept_idx[j] = the original row now at position j; needs the context's
+ * workspace and 2 * n_kept * 4 bytes <= 200 KiB) on code rows; the value
+ * scales move with their rows.  k_q8 and v_q8 must not overlap.
+ */
+ea_status ea_cache_append_q8(ea_ctx* ctx, const ea_shape* shape, void* k_q8, void* v_q8, float* v_scale,
+                             const void* k_new, const void* v_new, const float* v_scale_new,
+                             int32_t n_new, void* cuda_stream);
+ea_status ea_select_compact_inplace_q8(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                                       int32_t n_kept, void* k_q8, void* v_q8, float* v_scale,
+                                       int32_t* kept_idx, int32_t unordered, void* cuda_stream);
 
 /*
  * Eviction and compaction: per (unit, KV head) keep the n_kept pairs with the

@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_select_compact_inplace_unordered",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_cache_append_q8", "ea_select_compact_inplace_q8", "ea_select_compact_inplace_unordered",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -96,6 +96,9 @@ def lib() -> ctypes.CDLL:
         L.ea_select_compact_q8.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.ea_score_q8.restype = L.ea_select_compact_q8.restype = ctypes.c_int
         L.ea_score_q8_scratch_bytes.argtypes = [sp, ctypes.POINTER(ctypes.c_size_t)]
+        L.ea_cache_append_q8.argtypes = [vp, sp, vp, vp, vp, vp, vp, vp, i32, vp]
+        L.ea_select_compact_inplace_q8.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, i32, vp]
+        L.ea_cache_append_q8.restype = L.ea_select_compact_inplace_q8.restype = ctypes.c_int
         L.ea_score_q8_scratch_bytes.restype = ctypes.c_int
         L.ea_set_fused_stats.argtypes = [vp, i32]
         L.ea_set_fused_stats.restype = ctypes.c_int
@@ -244,6 +247,18 @@ def ea_cache_append(ctx: Context, shape: Shape, k, v, k_new, v_new):
                                  int(k_new.shape[2]), _stream(ctx.device)), "ea_cache_append")
 
 
+def ea_cache_append_q8(ctx: Context, shape: Shape, k_q8, v_q8, v_scale, k_new, v_new, v_scale_new):
+    """Append code rows ``k_new, v_new`` uint8 [U,Hkv,n_new,d] and their value scales [U,Hkv,n_new] behind the
+    ``shape.n_keys`` rows each head holds in ``k_q8, v_q8`` [U,Hkv,kv_capacity,d] and ``v_scale`` (in place)."""
+    for t, name in ((k_q8, "k_q8"), (v_q8, "v_q8"), (k_new, "k_new"), (v_new, "v_new")):
+        _dev_tensor(t, torch.uint8, name)
+    _dev_tensor(v_scale, torch.float32, "v_scale")
+    _dev_tensor(v_scale_new, torch.float32, "v_scale_new")
+    _check(lib().ea_cache_append_q8(ctx._h, ctypes.byref(shape), _ptr(k_q8), _ptr(v_q8), _ptr(v_scale), _ptr(k_new),
+                                    _ptr(v_new), _ptr(v_scale_new), int(k_new.shape[2]), _stream(ctx.device)),
+           "ea_cache_append_q8")
+
+
 def ea_window_push(ctx: Context, shape: Shape, q_ring, ring_pushed, q_new):
     """Push ``q_new`` [U,Hq,n_new,d] into the ring ``q_ring`` [U,Hq,W,d]; ``ring_pushed`` int64 [U] (device) counts."""
     _dev_tensor(q_ring, torch.bfloat16, "q_ring")
@@ -338,8 +353,8 @@ def score_q8_scratch_bytes(shape: Shape) -> int:
 
 def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar, sigma_bar, epsilon: float,
                 k_scratch=None, scores=None, logits=None, want_logits: bool = False):
-    """Scores of a quantised cache: k_q8, v_q8 uint8 [U,Hkv,n,d] (E4M3 codes), k_scale fp32 [U,Hkv,d],
-    v_scale fp32 [U,Hkv,n] -> scores fp32 [U,Hkv,n] (and the log-scores if asked)."""
+    """Scores of a quantised cache: k_q8, v_q8 uint8 [U,Hkv,cap,d] (E4M3 codes), k_scale fp32 [U,Hkv,d],
+    v_scale fp32 [U,Hkv,cap] (cap = kv_capacity, or n) -> scores fp32 [U,Hkv,n] (and the log-scores if asked)."""
     _dev_tensor(k_q8, torch.uint8, "k_q8")
     _dev_tensor(v_q8, torch.uint8, "v_q8")
     _dev_tensor(k_scale, torch.float32, "k_scale")
@@ -348,7 +363,7 @@ def ea_score_q8(ctx: Context, shape: Shape, k_q8, k_scale, v_q8, v_scale, mu_bar
     dev = k_q8.device
     if k_scratch is None and score_q8_scratch_bytes(shape) > 0:
         # only where the tensor-core kernel does not widen the codes itself
-        k_scratch = torch.empty((U, Hkv, n, d), dtype=torch.bfloat16, device=dev)
+        k_scratch = torch.empty((U, Hkv, shape.kv_capacity or n, d), dtype=torch.bfloat16, device=dev)
     if scores is None:
         scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=dev)
     if logits is None and want_logits:
@@ -444,6 +459,23 @@ def ea_select_compact_inplace_unordered(ctx: Context, shape: Shape, scores, n_ke
     _check(lib().ea_select_compact_inplace_unordered(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k),
                                                      _ptr(v), _ptr(kept_idx), _stream(ctx.device)),
            "ea_select_compact_inplace_unordered")
+    return kept_idx
+
+
+def ea_select_compact_inplace_q8(ctx: Context, shape: Shape, scores, n_kept: int, k_q8, v_q8, v_scale, kept_idx=None,
+                                 unordered: bool = False):
+    """In-place compaction of a quantised cache (code rows and the value scales of their tokens); ordered as
+    ``ea_select_compact_inplace`` or, with ``unordered``, as ``ea_select_compact_inplace_unordered``."""
+    _dev_tensor(scores, torch.float32, "scores")
+    _dev_tensor(k_q8, torch.uint8, "k_q8")
+    _dev_tensor(v_q8, torch.uint8, "v_q8")
+    _dev_tensor(v_scale, torch.float32, "v_scale")
+    if kept_idx is None:
+        kept_idx = torch.empty((shape.n_units, shape.n_kv_heads, max(n_kept, 0)), dtype=torch.int32,
+                               device=scores.device)
+    _check(lib().ea_select_compact_inplace_q8(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), _ptr(k_q8),
+                                              _ptr(v_q8), _ptr(v_scale), _ptr(kept_idx), int(bool(unordered)),
+                                              _stream(ctx.device)), "ea_select_compact_inplace_q8")
     return kept_idx
 
 

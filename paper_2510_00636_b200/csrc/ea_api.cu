@@ -455,8 +455,7 @@ ea_status ea_select_compact_inplace(ea_ctx* ctx, const ea_shape* shape, const fl
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     st = ea_launch_select(ctx, *shape, scores, n_kept, kept_idx, stream);
     if (st == EA_OK)
-        st = ea_launch_compact_inplace(ctx, *shape, n_kept, kept_idx, static_cast<__nv_bfloat16*>(k),
-                                       static_cast<__nv_bfloat16*>(v), stream);
+        st = ea_launch_compact_inplace(ctx, *shape, n_kept, kept_idx, k, v, stream);
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }
@@ -489,8 +488,7 @@ ea_status ea_select_compact_inplace_unordered(ea_ctx* ctx, const ea_shape* shape
     int32_t* sel = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + plan.logits);
     st = ea_launch_select(ctx, *shape, scores, n_kept, sel, stream);
     if (st == EA_OK)
-        st = ea_launch_compact_fill(ctx, *shape, n_kept, sel, kept_idx, static_cast<__nv_bfloat16*>(k),
-                                    static_cast<__nv_bfloat16*>(v), stream);
+        st = ea_launch_compact_fill(ctx, *shape, n_kept, sel, kept_idx, k, v, stream);
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

@@ -194,13 +194,14 @@ ea_status ea_launch_select(const ea_ctx* ctx, const ea_shape& s, const float* sc
                            int32_t* kept_idx, cudaStream_t st);
 
 // Compaction inside the cache buffers: the kept rows of every head move to the front of its range.
+// (codes: rows of head_dim one-byte codes instead of bf16)
 ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
-                                    __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st);
+                                    void* k, void* v, cudaStream_t st, bool codes = false);
 
 // Unordered variant: kept rows beyond n_kept fill the evicted positions below it; `sel` ascending kept positions
 // (scratch), `where` the original row at each position afterwards.
 ea_status ea_launch_compact_fill(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* sel,
-                                 int32_t* where, __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st);
+                                 int32_t* where, void* k, void* v, cudaStream_t st, bool codes = false);
 
 // Head-adaptive eviction: per-head counts and offsets from one radix search over the unit's scores,
 // then the per-head selection with those counts and a gather through the offsets.

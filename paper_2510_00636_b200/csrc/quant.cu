@@ -45,7 +45,7 @@ constexpr int kFq8Threads = 256;
 template <int D>
 __global__ void __launch_bounds__(kFq8Threads)
 finalize_q8_kernel(const float* __restrict__ logits, const float* __restrict__ lse, const uint8_t* __restrict__ v_q8,
-                   const float* __restrict__ v_scale, int Hq, int Hkv, int n, int group_mode, float epsilon,
+                   const float* __restrict__ v_scale, int Hq, int Hkv, int n, int cap, int group_mode, float epsilon,
                    float* __restrict__ scores) {
     constexpr int LPR = D / 16;         // lanes per value row (one uint4 = 16 codes each)
     constexpr int RPS = 32 / LPR;       // rows per load step
@@ -56,7 +56,7 @@ finalize_q8_kernel(const float* __restrict__ logits, const float* __restrict__ l
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int key0 = (blockIdx.x * (kFq8Threads / 32) + warp) * 32;
     if (key0 >= n) return;
-    const uint4* vrow = reinterpret_cast<const uint4*>(v_q8 + ((size_t)ug * n + key0) * D);
+    const uint4* vrow = reinterpret_cast<const uint4*>(v_q8 + ((size_t)ug * cap + key0) * D);      // heads are cap rows apart
     float my_sumsq = 0.f;
 #pragma unroll 4
     for (int t = 0; t < STEPS; ++t) {
@@ -96,11 +96,11 @@ finalize_q8_kernel(const float* __restrict__ logits, const float* __restrict__ l
         }
         if (group_mode == EA_GROUP_MEAN_PROB) a *= 1.0f / (float)G;
     }
-    scores[(size_t)ug * n + key] = (a + epsilon) * (v_scale[(size_t)ug * n + key] * sqrtf(my_sumsq));
+    scores[(size_t)ug * n + key] = (a + epsilon) * (v_scale[(size_t)ug * cap + key] * sqrtf(my_sumsq));
 }
 
 // rows of D codes = D / 16 pieces of 16 bytes; the value scale of a token follows its row
-__global__ void gather_q8_kernel(const int32_t* __restrict__ kept_idx, long long n_rows_out, int n, int n_kept, int lpr,
+__global__ void gather_q8_kernel(const int32_t* __restrict__ kept_idx, long long n_rows_out, int cap, int n_kept, int lpr,
                                  const uint4* __restrict__ k, const uint4* __restrict__ v,
                                  const float* __restrict__ v_scale, uint4* __restrict__ k_out,
                                  uint4* __restrict__ v_out, float* __restrict__ v_scale_out) {
@@ -110,10 +110,39 @@ __global__ void gather_q8_kernel(const int32_t* __restrict__ kept_idx, long long
         const long long row = t / lpr;
         const int piece = (int)(t % lpr);
         const long long head = row / n_kept;
-        const long long src = head * n + kept_idx[row];
+        const long long src = head * cap + kept_idx[row];          // heads are cap rows apart in the cache
         k_out[t] = __ldg(k + src * lpr + piece);
         v_out[t] = __ldg(v + src * lpr + piece);
         if (piece == 0) v_scale_out[row] = v_scale[src];
+    }
+}
+
+// The value scales of a head follow their rows through an in-place compaction.  Ordered form: position j
+// receives the scale of row idx[j] >= j; one CTA per head walks the kept rows in chunks, a chunk's sources
+// in registers before its destinations are written; a later chunk reads at or behind its own first
+// destination, which earlier chunks never write.
+constexpr int kScaleThreads = 256;
+__global__ void __launch_bounds__(kScaleThreads)
+scale_inplace_kernel(const int32_t* __restrict__ kept_idx, int cap, int n_kept, float* v_scale) {
+    const long long head = blockIdx.x;
+    float* vs = v_scale + head * (long long)cap;
+    const int32_t* idx = kept_idx + head * (long long)n_kept;
+    for (int j0 = 0; j0 < n_kept; j0 += kScaleThreads) {
+        const int j = j0 + threadIdx.x;
+        const int src = j < n_kept ? idx[j] : -1;
+        const float x = src >= 0 ? vs[src] : 0.f;
+        __syncthreads();
+        if (src >= 0) vs[j] = x;
+    }
+}
+// Unordered form: where[p] is the original row now at p; the movers come from at or beyond n_kept and
+// land below it, so no move can disturb another.
+__global__ void scale_fill_kernel(const int32_t* __restrict__ where, long long total, int cap, int n_kept, float* v_scale) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
+        const long long head = t / n_kept;
+        const int p = (int)(t % n_kept), w = where[t];
+        if (w != p) v_scale[head * cap + p] = v_scale[head * cap + w];
     }
 }
 
@@ -123,7 +152,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 ea_status ea_launch_dequant_k(const ea_ctx* ctx, const ea_shape& s, const uint8_t* k_q8, __nv_bfloat16* k_codes,
                               cudaStream_t st) {
-    const long long pieces = (long long)s.n_units * s.n_kv_heads * s.n_keys * (s.head_dim / 16);
+    // every row of the buffers, so that the scratch has the cache's own strides
+    const long long pieces = (long long)s.n_units * s.n_kv_heads * ea_kv_cap(s) * (s.head_dim / 16);
     long long want = (pieces + 255) / 256;
     const long long cap = (long long)ctx->sm_count * 16;
     dequant_k_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(reinterpret_cast<const uint4*>(k_q8), pieces,
@@ -139,15 +169,15 @@ ea_status ea_launch_finalize_q8(const ea_ctx* ctx, const ea_shape& s, const floa
     switch (s.head_dim) {
         case 64:
             finalize_q8_kernel<64><<<grid, kFq8Threads, 0, st>>>(logits, lse, v_q8, v_scale, s.n_q_heads, s.n_kv_heads,
-                                                                 s.n_keys, s.group_mode, epsilon, scores);
+                                                                 s.n_keys, ea_kv_cap(s), s.group_mode, epsilon, scores);
             break;
         case 128:
             finalize_q8_kernel<128><<<grid, kFq8Threads, 0, st>>>(logits, lse, v_q8, v_scale, s.n_q_heads, s.n_kv_heads,
-                                                                  s.n_keys, s.group_mode, epsilon, scores);
+                                                                  s.n_keys, ea_kv_cap(s), s.group_mode, epsilon, scores);
             break;
         case 256:
             finalize_q8_kernel<256><<<grid, kFq8Threads, 0, st>>>(logits, lse, v_q8, v_scale, s.n_q_heads, s.n_kv_heads,
-                                                                  s.n_keys, s.group_mode, epsilon, scores);
+                                                                  s.n_keys, ea_kv_cap(s), s.group_mode, epsilon, scores);
             break;
         default:
             return EA_ERR_UNSUPPORTED;
@@ -165,7 +195,7 @@ ea_status ea_launch_gather_q8(const ea_ctx* ctx, const ea_shape& s, int n_kept, 
     long long want = (rows * lpr + 255) / 256;
     const long long cap = (long long)ctx->sm_count * 16;
     gather_q8_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(
-        kept_idx, rows, s.n_keys, n_kept, lpr, reinterpret_cast<const uint4*>(k_q8), reinterpret_cast<const uint4*>(v_q8),
+        kept_idx, rows, ea_kv_cap(s), n_kept, lpr, reinterpret_cast<const uint4*>(k_q8), reinterpret_cast<const uint4*>(v_q8),
         v_scale, reinterpret_cast<uint4*>(k_out), reinterpret_cast<uint4*>(v_out), v_scale_out);
     ea_count_launches(ctx, 1);
     return EA_CHECK_LAUNCH();
@@ -180,7 +210,7 @@ ea_status ea_score_q8_scratch_bytes(const ea_shape* shape, size_t* bytes) {
     if (st != EA_OK) return st;
     *bytes = ea_mma_q8_supported(*shape)
                  ? 0
-                 : (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys * shape->head_dim * sizeof(__nv_bfloat16);
+                 : (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) * shape->head_dim * sizeof(__nv_bfloat16);
     return EA_OK;
 }
 
@@ -191,7 +221,6 @@ ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, cons
     size_t need = 0;
     ea_status st = ea_workspace_bytes(shape, &need);          // validates the shape
     if (st != EA_OK) return st;
-    if (shape->kv_capacity != 0 && shape->kv_capacity != shape->n_keys) return EA_ERR_UNSUPPORTED;
     if (shape->n_units == 0 || shape->n_keys == 0) return EA_OK;
     if (!k_q8 || !k_scale || !v_q8 || !v_scale || !mu_bar || !sigma_bar || !scores) return EA_ERR_INVALID_ARG;
     if (!k_scratch && !ea_mma_q8_supported(*shape)) return EA_ERR_INVALID_ARG;
@@ -259,14 +288,13 @@ ea_status ea_select_compact_q8(ea_ctx* ctx, const ea_shape* shape, const float* 
     size_t need = 0;
     ea_status st = ea_workspace_bytes(shape, &need);
     if (st != EA_OK) return st;
-    if (shape->kv_capacity != 0 && shape->kv_capacity != shape->n_keys) return EA_ERR_UNSUPPORTED;
     if (n_kept < 0 || n_kept > shape->n_keys) return EA_ERR_INVALID_ARG;
     if (shape->n_units == 0 || n_kept == 0) return EA_OK;
     if (!scores || !kept_idx || !k_q8 || !v_q8 || !v_scale || !k_out || !v_out || !v_scale_out) return EA_ERR_INVALID_ARG;
     if (!aligned16(scores) || !aligned16(k_q8) || !aligned16(v_q8) || !aligned16(k_out) || !aligned16(v_out))
         return EA_ERR_INVALID_ARG;
     {
-        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * shape->n_keys * shape->head_dim;
+        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) * shape->head_dim;
         const size_t out_bytes = (size_t)shape->n_units * shape->n_kv_heads * n_kept * shape->head_dim;
         const char* ins[2] = {static_cast<const char*>(k_q8), static_cast<const char*>(v_q8)};
         const char* outs[2] = {static_cast<const char*>(k_out), static_cast<const char*>(v_out)};
@@ -283,6 +311,56 @@ ea_status ea_select_compact_q8(ea_ctx* ctx, const ea_shape* shape, const float* 
         st = ea_launch_gather_q8(ctx, *shape, n_kept, kept_idx, static_cast<const uint8_t*>(k_q8),
                                  static_cast<const uint8_t*>(v_q8), v_scale, static_cast<uint8_t*>(k_out),
                                  static_cast<uint8_t*>(v_out), v_scale_out, stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_select_compact_inplace_q8(ea_ctx* ctx, const ea_shape* shape, const float* scores, int32_t n_kept,
+                                       void* k_q8, void* v_q8, float* v_scale, int32_t* kept_idx, int32_t unordered,
+                                       void* cuda_stream) {
+    if (!ctx || !shape) return EA_ERR_INVALID_ARG;
+    size_t need = 0;
+    ea_status st = ea_workspace_bytes(shape, &need);
+    if (st != EA_OK) return st;
+    if (n_kept < 0 || n_kept > shape->n_keys) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0 || n_kept == 0) return EA_OK;
+    if (!scores || !kept_idx || !k_q8 || !v_q8 || !v_scale) return EA_ERR_INVALID_ARG;
+    if (!aligned16(scores) || !aligned16(k_q8) || !aligned16(v_q8)) return EA_ERR_INVALID_ARG;
+    if (unordered && 2 * (size_t)n_kept * sizeof(int32_t) > 200 * 1024) return EA_ERR_UNSUPPORTED;
+    {
+        const size_t bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) * shape->head_dim;
+        const char* a = static_cast<const char*>(k_q8);
+        const char* b = static_cast<const char*>(v_q8);
+        if (a < b + bytes && b < a + bytes) return EA_ERR_INVALID_ARG;      // K and V are distinct buffers
+    }
+    if (unordered && ctx->workspace_bytes < need) return EA_ERR_WORKSPACE;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int cap = ea_kv_cap(*shape);
+    const long long heads = (long long)shape->n_units * shape->n_kv_heads;
+    if (unordered) {
+        // the ascending selection goes to the workspace (the log-score region: nothing of a compaction reads it)
+        const ea_ws_plan plan = ea_plan_workspace(*shape);
+        int32_t* sel = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + plan.logits);
+        st = ea_launch_select(ctx, *shape, scores, n_kept, sel, stream);
+        if (st == EA_OK) st = ea_launch_compact_fill(ctx, *shape, n_kept, sel, kept_idx, k_q8, v_q8, stream, true);
+        if (st == EA_OK) {
+            const long long total = heads * n_kept, want = (total + 255) / 256, lim = (long long)ctx->sm_count * 16;
+            scale_fill_kernel<<<(unsigned)(want < lim ? want : lim), 256, 0, stream>>>(kept_idx, total, cap, n_kept, v_scale);
+            ea_count_launches(ctx, 1);
+            st = EA_CHECK_LAUNCH();
+        }
+    } else {
+        st = ea_launch_select(ctx, *shape, scores, n_kept, kept_idx, stream);
+        if (st == EA_OK) st = ea_launch_compact_inplace(ctx, *shape, n_kept, kept_idx, k_q8, v_q8, stream, true);
+        if (st == EA_OK) {
+            scale_inplace_kernel<<<(unsigned)heads, kScaleThreads, 0, stream>>>(kept_idx, cap, n_kept, v_scale);
+            ea_count_launches(ctx, 1);
+            st = EA_CHECK_LAUNCH();
+        }
+    }
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

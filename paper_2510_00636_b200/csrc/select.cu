@@ -737,13 +737,15 @@ ea_status ea_launch_gather(const ea_ctx* ctx, const ea_shape& s, int n_kept, con
 }
 
 ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* kept_idx,
-                                    __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st) {
+                                    void* k, void* v, cudaStream_t st, bool codes) {
     if (n_kept <= 0) return EA_OK;
     ea_count_launches(ctx, 1);
     const dim3 grid((unsigned)(s.n_units * s.n_kv_heads), 2);
     uint4* k4 = reinterpret_cast<uint4*>(k);
     uint4* v4 = reinterpret_cast<uint4*>(v);
-    switch (s.head_dim) {
+    // the kernels count rows in 16-byte pieces of bf16: a row of d one-byte codes is a bf16 row of d / 2
+    switch (codes ? s.head_dim / 2 : s.head_dim) {
+        case 32: compact_inplace_kernel<32><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
         case 64: compact_inplace_kernel<64><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
         case 128: compact_inplace_kernel<128><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
         case 256: compact_inplace_kernel<256><<<grid, kIpThreads, 0, st>>>(kept_idx, ea_kv_cap(s), n_kept, k4, v4); break;
@@ -753,7 +755,7 @@ ea_status ea_launch_compact_inplace(const ea_ctx* ctx, const ea_shape& s, int n_
 }
 
 ea_status ea_launch_compact_fill(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* sel,
-                                 int32_t* where, __nv_bfloat16* k, __nv_bfloat16* v, cudaStream_t st) {
+                                 int32_t* where, void* k, void* v, cudaStream_t st, bool codes) {
     if (n_kept <= 0) return EA_OK;
     const size_t smem = 2 * (size_t)n_kept * sizeof(int32_t);
     if (smem > 200 * 1024) return EA_ERR_UNSUPPORTED;
@@ -761,7 +763,11 @@ ea_status ea_launch_compact_fill(const ea_ctx* ctx, const ea_shape& s, int n_kep
     uint4* k4 = reinterpret_cast<uint4*>(k);
     uint4* v4 = reinterpret_cast<uint4*>(v);
     const int cap = ea_kv_cap(s);
-    switch (s.head_dim) {
+    switch (codes ? s.head_dim / 2 : s.head_dim) {
+        case 32:
+            EA_CUDA_TRY(cudaFuncSetAttribute(compact_fill_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            compact_fill_kernel<32><<<grid, kFillThreads, smem, st>>>(sel, cap, n_kept, where, k4, v4);
+            break;
         case 64:
             EA_CUDA_TRY(cudaFuncSetAttribute(compact_fill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             compact_fill_kernel<64><<<grid, kFillThreads, smem, st>>>(sel, cap, n_kept, where, k4, v4);

@@ -44,6 +44,14 @@ __global__ void window_push_kernel(const uint4* __restrict__ q_new, long long pi
     }
 }
 
+// the value scales of appended code rows: scale_new[head, j] -> scale[head * cap + n_old + j]
+__global__ void scale_append_kernel(const float* __restrict__ scale_new, long long total, int n_new, int n_old, int cap,
+                                    float* __restrict__ scale) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride)
+        scale[(t / n_new) * cap + n_old + t % n_new] = scale_new[t];
+}
+
 __global__ void window_bump_kernel(long long* __restrict__ pushed, int n_units, int n_new) {
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
     if (u < n_units) pushed[u] += n_new;
@@ -88,6 +96,32 @@ ea_status ea_cache_append(ea_ctx* ctx, const ea_shape* shape, void* k, void* v, 
         static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), pieces, n_new, shape->n_keys, cap, lpr,
         static_cast<uint4*>(k), static_cast<uint4*>(v));
     ea_count_launches(ctx, 1);
+    st = EA_CHECK_LAUNCH();
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_cache_append_q8(ea_ctx* ctx, const ea_shape* shape, void* k_q8, void* v_q8, float* v_scale,
+                             const void* k_new, const void* v_new, const float* v_scale_new, int32_t n_new,
+                             void* cuda_stream) {
+    ea_status st = check_common(ctx, shape);
+    if (st != EA_OK) return st;
+    const int cap = ea_kv_cap(*shape);
+    if (n_new < 0 || (long long)shape->n_keys + n_new > cap) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0 || n_new == 0) return EA_OK;
+    if (!k_q8 || !v_q8 || !v_scale || !k_new || !v_new || !v_scale_new) return EA_ERR_INVALID_ARG;
+    if (!aligned16(k_q8) || !aligned16(v_q8) || !aligned16(k_new) || !aligned16(v_new)) return EA_ERR_INVALID_ARG;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int lpr = shape->head_dim / 16;                       // a row of codes is head_dim bytes
+    const long long rows = (long long)shape->n_units * shape->n_kv_heads * n_new, pieces = rows * lpr;
+    cache_append_kernel<<<grid_for(ctx, pieces), 256, 0, stream>>>(
+        static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), pieces, n_new, shape->n_keys, cap, lpr,
+        static_cast<uint4*>(k_q8), static_cast<uint4*>(v_q8));
+    scale_append_kernel<<<grid_for(ctx, rows), 256, 0, stream>>>(v_scale_new, rows, n_new, shape->n_keys, cap, v_scale);
+    ea_count_launches(ctx, 2);
     st = EA_CHECK_LAUNCH();
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;

@@ -170,14 +170,17 @@ def generate_layer(cfg: EAConfig, layer: int = 0, device="cpu", n_keys: int | No
     return q, k, v, torch.full((B,), p, dtype=torch.int64)
 
 
-def quantize_e4m3(k: torch.Tensor, v: torch.Tensor):
+def quantize_e4m3(k: torch.Tensor, v: torch.Tensor, k_scale: torch.Tensor | None = None):
     """Manufactures a quantised cache from bf16 ``k, v`` [B,Hkv,n,d]: FP8 E4M3 codes (uint8) with one fp32
     scale per key channel and one per value token, each scale mapping the largest magnitude to 448.
-    Returns ``(k_q8, k_scale [B,Hkv,d], v_q8, v_scale [B,Hkv,n])``.  Rounding is torch's cast."""
+    Returns ``(k_q8, k_scale [B,Hkv,d], v_q8, v_scale [B,Hkv,n])``.  Rounding is torch's cast.  With
+    ``k_scale`` given (pairs appended to an existing cache) the keys are coded against those scales,
+    saturating at the largest finite code."""
     kf, vf = k.float(), v.float()
-    k_scale = (kf.abs().amax(dim=2) / 448.0).clamp_min(1e-30)
+    if k_scale is None:
+        k_scale = (kf.abs().amax(dim=2) / 448.0).clamp_min(1e-30)
     v_scale = (vf.abs().amax(dim=3) / 448.0).clamp_min(1e-30)
-    k_q8 = (kf / k_scale[:, :, None, :]).to(torch.float8_e4m3fn).view(torch.uint8)
+    k_q8 = (kf / k_scale[:, :, None, :]).clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
     v_q8 = (vf / v_scale[..., None]).to(torch.float8_e4m3fn).view(torch.uint8)
     return k_q8.contiguous(), k_scale.contiguous(), v_q8.contiguous(), v_scale.contiguous()
 

@@ -105,11 +105,15 @@ def test_quantised_calls_validate_their_arguments(ea):
     ctx = ea.Context.for_shape(shape)
     mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
     sc = ea.ea_score_q8(ctx, shape, kq, ks, vq, vs, mu, sig, cfg.eps)
-    strided = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window,
-                            kv_capacity=cfg.n_keys + 8)
-    with pytest.raises(ea.EAError) as e:
-        ea.ea_score_q8(ctx, strided, kq, ks, vq, vs, mu, sig, cfg.eps)
-    assert e.value.status == 2
+    full = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_keys, cfg.window,
+                         kv_capacity=cfg.n_keys)
+    with pytest.raises(ea.EAError) as e:                 # no room behind the cached rows
+        ea.ea_cache_append_q8(ctx, full, kq, vq, vs, kq[:, :, :4].contiguous(), vq[:, :, :4].contiguous(),
+                              vs[:, :, :4].contiguous())
+    assert e.value.status == 1
+    with pytest.raises(ea.EAError) as e:                 # K and V must be distinct buffers
+        ea.ea_select_compact_inplace_q8(ctx, shape, sc, 8, kq, kq, vs)
+    assert e.value.status == 1
     with pytest.raises(ea.EAError) as e:
         ea.ea_select_compact_q8(ctx, shape, sc, cfg.n_keys + 1, kq, vq, vs)
     assert e.value.status == 1
@@ -117,3 +121,76 @@ def test_quantised_calls_validate_their_arguments(ea):
         ea.ea_score_q8(ea.Context(0, 256), shape, kq, ks, vq, vs, mu, sig, cfg.eps)
     assert e.value.status == 3
     ctx.sync_status()
+
+
+@pytest.mark.parametrize("unordered", [False, True])
+def test_quantised_cache_carried_through_consecutive_events(ea, oracle, unordered):
+    """Streaming decode on ONE buffer of codes: every event appends new code rows (coded against the cache's
+    key scales) with their value scales, pushes queries into the window ring, scores the cache inside its
+    larger buffer and compacts codes and value scales in place, in temporal order or with the evicted
+    positions filled.  Event by event against the oracle's quantised streaming driver on the same codes:
+    log-scores and scores within the tolerance protocol (scores to relative 1e-2 directly), the kept set against
+    the oracle's ranges and bit-exactly against the oracle's selection on the GPU's own scores, then codes and
+    scales of the cache bit-exactly.  The oracle's cache continues from the rows the GPU kept, in the GPU's
+    order."""
+    from oracle.ea_stream import QuantStreamOracle, fill_holes
+    base = inputs.CONFIGS[4].tempered(2.0)
+    budget, every, n0 = 1024, 384, 640
+    cap = budget + every
+    cfg = dataclasses.replace(base, n_layers=1, batch=2, n_keys=n0, n_kept=budget)
+    U, Hq, Hkv, d, W = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
+    dev = torch.device("cuda")
+    _, k0, v0, _ = inputs.generate_layer(cfg, layer=5, device=dev, n_keys=n0, draw=1)
+    kq0, ks, vq0, vs0 = inputs.quantize_e4m3(k0, v0)
+    kq = torch.zeros((U, Hkv, cap, d), dtype=torch.uint8, device=dev)
+    vq = torch.zeros_like(kq)
+    vs = torch.zeros((U, Hkv, cap), dtype=torch.float32, device=dev)
+    kq[:, :, :n0], vq[:, :, :n0], vs[:, :, :n0] = kq0, vq0, vs0
+    ring = torch.zeros((U, Hq, W, d), dtype=torch.bfloat16, device=dev)
+    pushed = torch.zeros((U,), dtype=torch.int64, device=dev)
+    st = QuantStreamOracle(_np(kq0), _np(ks), _np(vq0), _np(vs0), window=W, budget=budget)
+    ctx = ea.Context.for_shape(ea.make_shape(U, Hq, Hkv, d, cap, W, kv_capacity=cap))
+    n_cur, position = n0, n0
+    for e, m in enumerate((100, 200, 384, 384)):
+        n = n_cur + every
+        n_kept = min(n, budget)
+        position += every
+        _, kn, vn, _ = inputs.generate_layer(cfg, layer=5, device=dev, n_keys=every, draw=2 + e,
+                                             key_positions=torch.arange(position - every, position))
+        kqn, _, vqn, vsn = inputs.quantize_e4m3(kn, vn, k_scale=ks)
+        qn, _, _, _ = inputs.generate_layer(dataclasses.replace(cfg, window=m), layer=5, device=dev, n_keys=1,
+                                            draw=100 + e, q_phase=0.1 * e)
+        pos = torch.full((U,), position, dtype=torch.int64, device=dev)
+        shape_old = ea.make_shape(U, Hq, Hkv, d, n_cur, W, kv_capacity=cap)
+        shape = ea.make_shape(U, Hq, Hkv, d, n, W, kv_capacity=cap)
+        ea.ea_cache_append_q8(ctx, shape_old, kq, vq, vs, kqn, vqn, vsn)
+        ea.ea_window_push(ctx, shape, ring, pushed, qn)
+        mu, sigma = ea.ea_query_stats_ring(ctx, shape, ring, pushed, pos, cfg.n_future, cfg.rope_base)
+        sc_t, lg_t = ea.ea_score_q8(ctx, shape, kq, ks, vq, vs, mu, sigma, cfg.eps, want_logits=True)
+        idx = ea.ea_select_compact_inplace_q8(ctx, shape, sc_t, n_kept, kq, vq, vs, unordered=unordered)
+        ctx.sync_status()
+
+        st.append(_np(kqn), _np(vqn), _np(vsn))
+        st.push_queries(inputs.bits(qn))
+        ref = st.compress(np.full((U,), position), cfg.n_future, cfg.rope_base, cfg.eps)
+        from oracle import ea_quant
+        k_real, v_real = ea_quant.dequant_k(st.k, st.k_scale), ea_quant.dequant_v(st.v, st.v_scale)
+        delta = parity.logit_error_bound(None, ref["mu_bar"], ref["sigma_bar"], 16, k_values=k_real)
+        bad, _ = parity.check_logits(_np(lg_t), ref["logits"], delta)
+        assert bad == 0, f"event {e}: {bad} log-scores off"
+        lo, hi = parity.score_range(ref["logits"], delta, None, cfg.eps, 0, v_values=v_real)
+        sc = _np(sc_t)
+        bad, unstable = parity.check_scores(sc, lo, hi)
+        assert bad == 0 and unstable == 0, f"event {e}"
+        np.testing.assert_allclose(sc, ref["scores"], rtol=1e-2, atol=0.0)
+        got = _np(idx)
+        sel = oracle.select(sc.astype(np.float64), n_kept)                 # ascending kept positions
+        missing, present, _ = parity.check_kept(np.sort(got, axis=-1), lo, hi, n_kept)
+        assert missing == 0 and present == 0, f"event {e}"
+        want = fill_holes(sel, n_kept) if unordered else sel
+        assert np.array_equal(got, want), f"event {e}"
+        st.keep(got)
+        assert np.array_equal(_np(kq[:, :, :n_kept]), st.k), f"event {e}: key codes differ"
+        assert np.array_equal(_np(vq[:, :, :n_kept]), st.v), f"event {e}: value codes differ"
+        assert np.array_equal(_np(vs[:, :, :n_kept]), st.v_scale), f"event {e}: value scales differ"
+        n_cur = n_kept

@@ -16,7 +16,9 @@ gathering are the integer routines of ``ea_oracle`` applied to codes and scales.
 
 Parity status: pinned (``tests/test_oracle_pins.py``): the decoder against a library conversion of all
 256 codes; dequantise-then-score against scoring with the key scales folded into the statistics (an
-exact identity); unit scales and representable values against the pinned bf16 oracle.
+exact identity); unit scales and representable values against the pinned bf16 oracle; the ragged gather
+of head-adaptive eviction against the pinned C routine on the same bytes and, where every head keeps
+the same count, against plain indexing.
 """
 from __future__ import annotations
 
@@ -97,3 +99,22 @@ def compress(q_win_bits, k_q8, k_scale, v_q8, v_scale, pos_next, n_future, rope_
                 k_out=np.take_along_axis(np.asarray(k_q8), i64[..., None], axis=2),
                 v_out=np.take_along_axis(np.asarray(v_q8), i64[..., None], axis=2),
                 v_scale_out=np.take_along_axis(np.asarray(v_scale), i64, axis=2))
+
+
+def gather_adaptive(k_q8, v_q8, v_scale, idx, offsets):
+    """Compaction after head-adaptive eviction (``ea_oracle.select_adaptive``) of a quantised cache: head g of
+    unit u owns ``idx[u, offsets[u, g]:offsets[u, g + 1]]``; returns the kept code rows ``[U, B, d]`` (keys,
+    values) and the value scales ``[U, B]`` of their tokens, heads one after the other."""
+    k_q8, v_q8, v_scale = np.asarray(k_q8), np.asarray(v_q8), np.asarray(v_scale)
+    idx, offsets = np.asarray(idx), np.asarray(offsets)
+    U, Hkv, n, d = k_q8.shape
+    B = idx.shape[1]
+    k_out = np.zeros((U, B, d), k_q8.dtype)
+    v_out = np.zeros((U, B, d), v_q8.dtype)
+    s_out = np.zeros((U, B), v_scale.dtype)
+    for u in range(U):
+        for g in range(Hkv):
+            for j in range(int(offsets[u, g]), int(offsets[u, g + 1])):
+                i = int(idx[u, j])
+                k_out[u, j], v_out[u, j], s_out[u, j] = k_q8[u, g, i], v_q8[u, g, i], v_scale[u, g, i]
+    return k_out, v_out, s_out

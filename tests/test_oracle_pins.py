@@ -726,3 +726,27 @@ def test_quantised_stream_with_unit_scales_walks_with_the_bf16_stream(oracle):
         bs.keep(b["kept_idx"])
         assert np.array_equal(to_bf16(qs.k), bs.k) and np.array_equal(to_bf16(qs.v), bs.v)
         assert (qs.v_scale == 1.0).all() and qs.v_scale.shape == (1, 2, qs.n_keys)
+
+
+def test_quantised_adaptive_gather_against_the_c_routine_and_plain_indexing(oracle):
+    """Codes are bytes: the ragged gather of code rows must equal the pinned C gather on the same bytes read as
+    16-bit words, the scales must be the scales of the same tokens, and with the safeguard at the whole budget
+    (every head keeps n_kept) the result is plain per-head indexing."""
+    from oracle import ea_quant
+    q, kq, ks, vq, vs = _quant_case(31, U=2, n=80)
+    rng = np.random.default_rng(7)
+    sc = rng.random((2, 2, 80)) * np.array([1.0, 4.0])[None, :, None]
+    idx, off = oracle.select_adaptive(sc, 30, 6)
+    assert (off[:, -1] == 60).all() and (np.diff(off, axis=1) != 30).any()          # genuinely ragged
+    ko, vo, so = ea_quant.gather_adaptive(kq, vq, vs, idx, off)
+    assert np.array_equal(ko.view(np.uint16), oracle.gather_adaptive(kq.view(np.uint16), idx, off))
+    assert np.array_equal(vo.view(np.uint16), oracle.gather_adaptive(vq.view(np.uint16), idx, off))
+    for u in range(2):
+        for g in range(2):
+            sl = slice(off[u, g], off[u, g + 1])
+            assert np.array_equal(so[u, sl], vs[u, g][idx[u, sl]])
+    idx_f, off_f = oracle.select_adaptive(sc, 30, 30)
+    ko, vo, so = ea_quant.gather_adaptive(kq, vq, vs, idx_f, off_f)
+    per_head = oracle.select(sc, 30).astype(np.int64)
+    assert np.array_equal(ko.reshape(2, 2, 30, -1), np.take_along_axis(kq, per_head[..., None], axis=2))
+    assert np.array_equal(so.reshape(2, 2, 30), np.take_along_axis(vs, per_head, axis=2))

@@ -302,6 +302,18 @@ ea_status ea_select_compact_q8(ea_ctx* ctx, const ea_shape* shape, const float* 
                                const float* v_scale, int32_t* kept_idx, void* k_out, void* v_out,
                                float* v_scale_out, void* cuda_stream);
 /*
+ * ea_select_compact_adaptive (head-adaptive eviction, same arguments and
+ * errors) on a quantised cache: ragged outputs k_out, v_out uint8
+ * [n_units, Hkv * n_kept, d] and v_scale_out fp32 [n_units, Hkv * n_kept],
+ * head g of unit u owning the rows head_offsets[u, g] .. head_offsets[u, g + 1].
+ * The outputs are always gathered (all three required when n_kept > 0).
+ */
+ea_status ea_select_compact_adaptive_q8(ea_ctx* ctx, const ea_shape* shape, const float* scores,
+                                        int32_t n_kept, int32_t n_floor, const void* k_q8,
+                                        const void* v_q8, const float* v_scale, int32_t* kept_idx,
+                                        int32_t* head_offsets, void* k_out, void* v_out,
+                                        float* v_scale_out, void* cuda_stream);
+/*
  * Streaming decode on a quantised cache (the decoding set-up of Sec. 4 with
  * the format above): the two calls that let one buffer of codes live through
  * consecutive compression events, beside ea_window_push / ea_query_stats_ring

@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_cache_append_q8", "ea_select_compact_inplace_q8", "ea_select_compact_inplace_unordered",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_cache_append_q8", "ea_select_compact_inplace_q8", "ea_select_compact_adaptive_q8", "ea_select_compact_inplace_unordered",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -99,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.ea_cache_append_q8.argtypes = [vp, sp, vp, vp, vp, vp, vp, vp, i32, vp]
         L.ea_select_compact_inplace_q8.argtypes = [vp, sp, vp, i32, vp, vp, vp, vp, i32, vp]
         L.ea_cache_append_q8.restype = L.ea_select_compact_inplace_q8.restype = ctypes.c_int
+        L.ea_select_compact_adaptive_q8.argtypes = [vp, sp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.ea_select_compact_adaptive_q8.restype = ctypes.c_int
         L.ea_score_q8_scratch_bytes.restype = ctypes.c_int
         L.ea_set_fused_stats.argtypes = [vp, i32]
         L.ea_set_fused_stats.restype = ctypes.c_int
@@ -514,6 +516,27 @@ def ea_select_compact_adaptive(ctx: Context, shape: Shape, scores, n_kept: int, 
                                             _ptr(k), _ptr(v), _ptr(kept_idx), _ptr(head_offsets), _ptr(k_out),
                                             _ptr(v_out), _stream(ctx.device)), "ea_select_compact_adaptive")
     return kept_idx, head_offsets, k_out, v_out
+
+
+def ea_select_compact_adaptive_q8(ctx: Context, shape: Shape, scores, n_kept: int, n_floor: int, k_q8, v_q8, v_scale):
+    """Head-adaptive eviction on a quantised cache -> (kept_idx [U,Hkv*n_kept], head_offsets [U,Hkv+1],
+    k_out, v_out uint8 [U,Hkv*n_kept,d], v_scale_out fp32 [U,Hkv*n_kept])."""
+    _dev_tensor(scores, torch.float32, "scores")
+    _dev_tensor(k_q8, torch.uint8, "k_q8")
+    _dev_tensor(v_q8, torch.uint8, "v_q8")
+    _dev_tensor(v_scale, torch.float32, "v_scale")
+    U, Hkv, d = shape.n_units, shape.n_kv_heads, shape.head_dim
+    B, dev = Hkv * max(n_kept, 0), scores.device
+    kept_idx = torch.empty((U, B), dtype=torch.int32, device=dev)
+    head_offsets = torch.empty((U, Hkv + 1), dtype=torch.int32, device=dev)
+    k_out = torch.empty((U, B, d), dtype=torch.uint8, device=dev)
+    v_out = torch.empty((U, B, d), dtype=torch.uint8, device=dev)
+    v_scale_out = torch.empty((U, B), dtype=torch.float32, device=dev)
+    _check(lib().ea_select_compact_adaptive_q8(ctx._h, ctypes.byref(shape), _ptr(scores), int(n_kept), int(n_floor),
+                                               _ptr(k_q8), _ptr(v_q8), _ptr(v_scale), _ptr(kept_idx),
+                                               _ptr(head_offsets), _ptr(k_out), _ptr(v_out), _ptr(v_scale_out),
+                                               _stream(ctx.device)), "ea_select_compact_adaptive_q8")
+    return kept_idx, head_offsets, k_out, v_out, v_scale_out
 
 
 @dataclass

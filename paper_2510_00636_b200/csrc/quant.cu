@@ -117,6 +117,34 @@ __global__ void gather_q8_kernel(const int32_t* __restrict__ kept_idx, long long
     }
 }
 
+// gather_q8_kernel after head-adaptive eviction: output row j of unit u belongs to the head whose range
+// [head_off[g], head_off[g + 1]) holds j
+__global__ void gather_adaptive_q8_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ head_off,
+                                          long long n_rows_out, int cap, int Hkv, int unit_stride, int lpr,
+                                          const uint4* __restrict__ k, const uint4* __restrict__ v,
+                                          const float* __restrict__ v_scale, uint4* __restrict__ k_out,
+                                          uint4* __restrict__ v_out, float* __restrict__ v_scale_out) {
+    const long long total = n_rows_out * lpr;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
+        const long long row = t / lpr;
+        const int piece = (int)(t % lpr);
+        const long long u = row / unit_stride;
+        const int j = (int)(row % unit_stride);
+        const int32_t* off = head_off + u * (Hkv + 1);
+        int lo = 0, hi = Hkv - 1;                      // the last g with off[g] <= j
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) / 2;
+            if (off[mid] <= j) lo = mid;
+            else hi = mid - 1;
+        }
+        const long long src = (u * Hkv + lo) * cap + kept_idx[row];
+        k_out[t] = __ldg(k + src * lpr + piece);
+        v_out[t] = __ldg(v + src * lpr + piece);
+        if (piece == 0) v_scale_out[row] = v_scale[src];
+    }
+}
+
 // The value scales of a head follow their rows through an in-place compaction.  Ordered form: position j
 // receives the scale of row idx[j] >= j; one CTA per head walks the kept rows in chunks, a chunk's sources
 // in registers before its destinations are written; a later chunk reads at or behind its own first
@@ -311,6 +339,54 @@ ea_status ea_select_compact_q8(ea_ctx* ctx, const ea_shape* shape, const float* 
         st = ea_launch_gather_q8(ctx, *shape, n_kept, kept_idx, static_cast<const uint8_t*>(k_q8),
                                  static_cast<const uint8_t*>(v_q8), v_scale, static_cast<uint8_t*>(k_out),
                                  static_cast<uint8_t*>(v_out), v_scale_out, stream);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_select_compact_adaptive_q8(ea_ctx* ctx, const ea_shape* shape, const float* scores, int32_t n_kept,
+                                        int32_t n_floor, const void* k_q8, const void* v_q8, const float* v_scale,
+                                        int32_t* kept_idx, int32_t* head_offsets, void* k_out, void* v_out,
+                                        float* v_scale_out, void* cuda_stream) {
+    if (!ctx || !shape) return EA_ERR_INVALID_ARG;
+    size_t need = 0;
+    ea_status st = ea_workspace_bytes(shape, &need);
+    if (st != EA_OK) return st;
+    if (n_kept < 0 || n_kept > shape->n_keys || n_floor < 0 || n_floor > n_kept) return EA_ERR_INVALID_ARG;
+    if ((long long)shape->n_kv_heads * n_kept > 0x7fffffffLL) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0) return EA_OK;
+    if (!head_offsets) return EA_ERR_INVALID_ARG;
+    if (n_kept > 0 && (!scores || !kept_idx || !k_q8 || !v_q8 || !v_scale || !k_out || !v_out || !v_scale_out))
+        return EA_ERR_INVALID_ARG;
+    if (!aligned16(scores) || !aligned16(k_q8) || !aligned16(v_q8) || !aligned16(k_out) || !aligned16(v_out))
+        return EA_ERR_INVALID_ARG;
+    if (n_kept > 0) {
+        const size_t in_bytes = (size_t)shape->n_units * shape->n_kv_heads * ea_kv_cap(*shape) * shape->head_dim;
+        const size_t out_bytes = (size_t)shape->n_units * shape->n_kv_heads * n_kept * shape->head_dim;
+        const char* ins[2] = {static_cast<const char*>(k_q8), static_cast<const char*>(v_q8)};
+        const char* outs[2] = {static_cast<const char*>(k_out), static_cast<const char*>(v_out)};
+        for (const char* o : outs)
+            for (const char* i : ins)
+                if (o < i + in_bytes && i < o + out_bytes) return EA_ERR_INVALID_ARG;
+    }
+    if (ctx->workspace_bytes < need) return EA_ERR_WORKSPACE;
+    const ea_ws_plan plan = ea_plan_workspace(*shape);
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = ea_launch_select_adaptive(ctx, *shape, scores, n_kept, n_floor,
+                                   static_cast<char*>(ctx->workspace) + plan.adaptive, kept_idx, head_offsets, stream);
+    if (st == EA_OK && n_kept > 0) {
+        const int lpr = shape->head_dim / 16, unit_stride = shape->n_kv_heads * n_kept;
+        const long long rows = (long long)shape->n_units * unit_stride;
+        const long long want = (rows * lpr + 255) / 256, lim = (long long)ctx->sm_count * 16;
+        gather_adaptive_q8_kernel<<<(unsigned)(want < lim ? want : lim), 256, 0, stream>>>(
+            kept_idx, head_offsets, rows, ea_kv_cap(*shape), shape->n_kv_heads, unit_stride, lpr,
+            static_cast<const uint4*>(k_q8), static_cast<const uint4*>(v_q8), v_scale, static_cast<uint4*>(k_out),
+            static_cast<uint4*>(v_out), v_scale_out);
+        ea_count_launches(ctx, 1);
+        st = EA_CHECK_LAUNCH();
+    }
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

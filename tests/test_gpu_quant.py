@@ -194,3 +194,31 @@ def test_quantised_cache_carried_through_consecutive_events(ea, oracle, unordere
         assert np.array_equal(_np(vq[:, :, :n_kept]), st.v), f"event {e}: value codes differ"
         assert np.array_equal(_np(vs[:, :, :n_kept]), st.v_scale), f"event {e}: value scales differ"
         n_cur = n_kept
+
+
+@pytest.mark.parametrize("cfg_id,floor_share,cap_extra", [(1, 0.2, 0), (0, 0.0, 24), (3, 0.5, 0)])
+def test_head_adaptive_eviction_on_a_quantised_cache(ea, oracle, cfg_id, floor_share, cap_extra):
+    """Scores of the quantised cache from the CUDA path, then head-adaptive eviction on the code rows: offsets,
+    indices, gathered codes and value scales bit-exact against the oracle's routines on the GPU's own scores
+    (also with the cache inside a larger buffer)."""
+    from oracle import ea_quant
+    cfg = inputs.CONFIGS[cfg_id].tempered(2.0, 0.02)
+    if cfg_id == 3:
+        cfg = dataclasses.replace(cfg, n_layers=1, n_keys=3000, n_kept=700)
+    q, k, v, pos = inputs.generate_layer(cfg, device="cuda")
+    kq, ks, vq, vs = inputs.quantize_e4m3(k, v)
+    n, cap = cfg.n_keys, cfg.n_keys + cap_extra
+    if cap_extra:
+        grow = lambda t: torch.cat([t, torch.zeros_like(t[:, :, :cap_extra])], dim=2).contiguous()
+        kq, vq, vs = grow(kq), grow(vq), grow(vs)
+    shape = ea.make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, n, cfg.window, kv_capacity=cap if cap_extra else 0)
+    ctx = ea.Context.for_shape(shape)
+    mu, sig = ea.ea_query_stats(ctx, shape, q, pos.cuda(), cfg.n_future, cfg.rope_base)
+    sc = ea.ea_score_q8(ctx, shape, kq, ks, vq, vs, mu, sig, cfg.eps)
+    n_floor = ea.ea_n_floor(cfg.n_kept, floor_share)
+    idx, off, ko, vo, so = ea.ea_select_compact_adaptive_q8(ctx, shape, sc, cfg.n_kept, n_floor, kq, vq, vs)
+    ctx.sync_status()
+    want_idx, want_off = oracle.select_adaptive(_np(sc).astype(np.float64), cfg.n_kept, n_floor)
+    assert np.array_equal(_np(off), want_off) and np.array_equal(_np(idx), want_idx)
+    wk, wv, ws = ea_quant.gather_adaptive(_np(kq)[:, :, :n], _np(vq)[:, :, :n], _np(vs)[:, :, :n], want_idx, want_off)
+    assert np.array_equal(_np(ko), wk) and np.array_equal(_np(vo), wv) and np.array_equal(_np(so), ws)

@@ -47,6 +47,12 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
+// two such matrices (lanes 0-15 give the row addresses)
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t (&r)[2]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
+                 : "=r"(r[0]), "=r"(r[1])
+                 : "r"(addr));
+}
 // eight consecutive channels of a window row
 __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
     const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
@@ -124,17 +130,53 @@ __device__ __forceinline__ void lds8(const float* p, float (&v)[8]) {
     v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 
+// Where the accumulator tiles (16 channel rows x 8 channel columns, one mma.m16n8k16 each) of a warp lie in
+// the CTA's BM x BM block.
+//   full block (TRI = false): the warps form a 2 x 4 grid of (BM/2) x (BM/4) warp tiles.
+//   upper triangle of a diagonal block of 128 (TRI = true): the block has 8 strips of 16 rows; strip i needs
+//   the column tiles j >= 2 i (the two that straddle the diagonal included): 72 of the 128 tiles, nine per
+//   warp.  Warp 2p takes strip p, columns 2p .. 2p+8; warp 2p+1 the rest of strip p (columns 2p+9 .. 15)
+//   and all of strip 7-p (columns 14-2p .. 15).  A warp's tile 0 is the single odd column tile, tiles 1 .. 8
+//   are four pairs of neighbouring column tiles, so that one ldmatrix.x4 serves a pair.
+template <int BM, bool TRI>
+struct StatsTiles {
+    static constexpr int TM = BM / 32, TN = BM / 32;      // full block: mma tiles per warp along rows, columns
+    static constexpr int NT = TRI ? 9 : TM * TN;
+    int p, q;                                             // TRI: warp = 2p + q
+    int wm, wn;                                           // full: warp position
+    __device__ __forceinline__ explicit StatsTiles(int warp) : p(warp / 2), q(warp % 2), wm(warp / 4), wn(warp % 4) {}
+    // TRI: the strip (0: strip p, 1: strip 7-p) and first column tile of pair r
+    __device__ __forceinline__ int pair_second_strip(int r) const { return q && r >= 3 - p; }
+    __device__ __forceinline__ int pair_col(int r) const {
+        if (!q) return 2 * p + 2 * r;
+        return r < 3 - p ? 2 * p + 10 + 2 * r : 14 - 2 * p + 2 * (r - (3 - p));
+    }
+    __device__ __forceinline__ int row0(int t) const {    // first channel row of tile t within the block
+        if (!TRI) return wm * (BM / 2) + (t / TN) * 16;
+        return 16 * ((t > 0 && pair_second_strip((t - 1) / 2)) ? 7 - p : p);
+    }
+    __device__ __forceinline__ int col0(int t) const {    // first channel column of tile t within the block
+        if (!TRI) return wn * (BM / 4) + (t % TN) * 8;
+        if (t == 0) return 8 * (q ? 2 * p + 9 : 2 * p + 8);
+        return 8 * (pair_col((t - 1) / 2) + (t - 1) % 2);
+    }
+};
+
 // QT: the window queries as bf16 (what a model's query projection emits) or fp32 (from project_kernel).
-template <int D, typename QT>
-__global__ void __launch_bounds__(256, 2)
+// TRI: the CTA computes the upper triangle of diagonal block blockIdx.y (blocks of 128 only); otherwise the
+// whole block (0, 0) (head_dim 64) or (0, 1) (head_dim 256).
+template <int D, typename QT, bool TRI>
+__global__ void __launch_bounds__(256, TRI ? 3 : 2)
 stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, int Hq, int W,
                  int layout, float inv_norm, float* __restrict__ mu_bar, float* __restrict__ sigma_bar,
                  int w_cap, const long long* __restrict__ pushed, int cov_sample, const StatsImage img) {
     using SG = StatsGeo<D>;
     constexpr int HALF = D / 2;
     constexpr int BM = SG::BM, NB1 = SG::NB1, P = SG::PITCH;
-    constexpr int WM = BM / 2, WN = BM / 4;        // warp tile: 2 x 4 warps
-    constexpr int TM = WM / 16, TN = WN / 8;       // mma tiles per warp
+    using TL = StatsTiles<BM, TRI>;
+    constexpr int WM = BM / 2, WN = BM / 4;        // full block: warp tile of the 2 x 4 warps
+    constexpr int TM = TL::TM, TN = TL::TN, NT = TL::NT;
+    static_assert(!TRI || BM == 128, "the triangular tiling is laid out for blocks of 128");
     extern __shared__ __align__(16) unsigned char stats_smem[];
     // [hi / lo][w in chunk][channel: BM channels of the block's rows, then (off the diagonal) of its columns]
     float* mu_s = reinterpret_cast<float*>(stats_smem + SG::REGION);                        // [D]
@@ -144,10 +186,11 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
 
     const int uh = blockIdx.x;
     const int u = uh / Hq;
-    // blockIdx.y -> (bi <= bj)
-    const int bi = NB1 == 1 ? 0 : (blockIdx.y == 2 ? 1 : 0);
-    const int bj = NB1 == 1 ? 0 : (blockIdx.y == 0 ? 0 : 1);
+    // the block (bi <= bj) of this CTA
+    const int bi = TRI ? (int)blockIdx.y : 0;
+    const int bj = TRI ? (int)blockIdx.y : NB1 - 1;
     const bool diag = bi == bj;
+    const bool first_block = (TRI || NB1 == 1) && blockIdx.y == 0;      // writes mu_bar
     const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
     // A window kept as a ring of w_cap rows (pushed != nullptr): the rows written so far, at most
     // w_cap of them, are the window; mean and covariance do not depend on their order, so a
@@ -198,7 +241,7 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
         }
     }
     __syncthreads();
-    if (blockIdx.y == 0) {
+    if (first_block) {
         for (int m = tid; m < HALF; m += 256) {
             const int a = layout == EA_ROPE_INTERLEAVED ? 2 * m : m;
             const int b = layout == EA_ROPE_INTERLEAVED ? 2 * m + 1 : m + HALF;
@@ -211,15 +254,14 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
         }
     }
 
-    float acc[TM][TN][4];
+    float acc[NT][4];
 #pragma unroll
-    for (int i = 0; i < TM; ++i)
+    for (int t = 0; t < NT; ++t)
 #pragma unroll
-        for (int j = 0; j < TN; ++j)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+        for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
 
-    const int wm = warp / 4, wn = warp % 4;        // warp position in the block
+    const TL tiles(warp);
+    const int wm = tiles.wm, wn = tiles.wn;
     const int n_ch = diag ? BM : 2 * BM;           // channels staged per chunk
     const uint32_t xs_hi = static_cast<uint32_t>(__cvta_generic_to_shared(stats_smem));
     const uint32_t xs_lo = xs_hi + kKC * P * 2;
@@ -286,33 +328,81 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
         __syncthreads();
 #pragma unroll
         for (int k0 = 0; k0 < kKC; k0 += 16) {
-            uint32_t a_hi[TM][4], a_lo[TM][4];
+            if constexpr (TRI) {
+                // A fragments of the warp's one or two strips; matrices (channels +0, w +0), (+8, +0), (+0, +8), (+8, +8)
+                uint32_t a_hi[2][4], a_lo[2][4];
+                const int kr_a = k0 + (lane % 8) + 8 * (lane / 16);
 #pragma unroll
-            for (int i = 0; i < TM; ++i) {
-                // matrices: (channels +0, w +0), (channels +8, w +0), (channels +0, w +8), (channels +8, w +8)
-                const int kr = k0 + (lane % 8) + 8 * (lane / 16);
-                const int mc = wm * WM + i * 16 + 8 * ((lane / 8) % 2);
-                const uint32_t off = (uint32_t)((kr * P + mc) * 2);
-                ldmatrix_x4_trans(xs_hi + off, a_hi[i]);
-                ldmatrix_x4_trans(xs_lo + off, a_lo[i]);
-            }
+                for (int i = 0; i < 2; ++i) {
+                    const int mc = 16 * (i ? (tiles.q ? 7 - tiles.p : tiles.p) : tiles.p) + 8 * ((lane / 8) % 2);
+                    const uint32_t off = (uint32_t)((kr_a * P + mc) * 2);
+                    ldmatrix_x4_trans(xs_hi + off, a_hi[i]);
+                    ldmatrix_x4_trans(xs_lo + off, a_lo[i]);
+                }
+                {   // tile 0: the single column tile, always in strip p; matrices (w +0), (w +8)
+                    uint32_t b_hi[2], b_lo[2];
+                    const int kr = k0 + (lane % 8) + 8 * ((lane / 8) % 2);
+                    const uint32_t off = (uint32_t)((kr * P + tiles.col0(0)) * 2);
+                    ldmatrix_x2_trans(xs_hi + off, b_hi);
+                    ldmatrix_x2_trans(xs_lo + off, b_lo);
+                    mma_bf16_16816(acc[0], a_hi[0], b_hi[0], b_hi[1]);
+                    mma_bf16_16816(acc[0], a_hi[0], b_lo[0], b_lo[1]);
+                    mma_bf16_16816(acc[0], a_lo[0], b_hi[0], b_hi[1]);
+                }
 #pragma unroll
-            for (int j2 = 0; j2 < TN; j2 += 2) {
-                // two 8-channel column tiles per load: (tile 0, w +0), (tile 0, w +8), (tile 1, w +0), (tile 1, w +8)
-                uint32_t b_hi[4], b_lo[4];
-                const int kr = k0 + (lane % 8) + 8 * ((lane / 8) % 2);
-                const int nc = (diag ? 0 : BM) + wn * WN + j2 * 8 + 8 * (lane / 16);
-                const uint32_t off = (uint32_t)((kr * P + nc) * 2);
-                ldmatrix_x4_trans(xs_hi + off, b_hi);
-                ldmatrix_x4_trans(xs_lo + off, b_lo);
+                for (int r = 0; r < 4; ++r) {
+                    // a pair of column tiles: (tile 0, w +0), (tile 0, w +8), (tile 1, w +0), (tile 1, w +8)
+                    uint32_t b_hi[4], b_lo[4];
+                    const int kr = k0 + (lane % 8) + 8 * ((lane / 8) % 2);
+                    const int nc = 8 * tiles.pair_col(r) + 8 * (lane / 16);
+                    const uint32_t off = (uint32_t)((kr * P + nc) * 2);
+                    ldmatrix_x4_trans(xs_hi + off, b_hi);
+                    ldmatrix_x4_trans(xs_lo + off, b_lo);
+                    if (tiles.pair_second_strip(r)) {          // warp-uniform
 #pragma unroll
-                for (int i = 0; i < TM; ++i)
+                        for (int jj = 0; jj < 2; ++jj) {
+                            mma_bf16_16816(acc[1 + 2 * r + jj], a_hi[1], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                            mma_bf16_16816(acc[1 + 2 * r + jj], a_hi[1], b_lo[2 * jj], b_lo[2 * jj + 1]);
+                            mma_bf16_16816(acc[1 + 2 * r + jj], a_lo[1], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                        }
+                    } else {
 #pragma unroll
-                    for (int jj = 0; jj < 2; ++jj) {
-                        mma_bf16_16816(acc[i][j2 + jj], a_hi[i], b_hi[2 * jj], b_hi[2 * jj + 1]);
-                        mma_bf16_16816(acc[i][j2 + jj], a_hi[i], b_lo[2 * jj], b_lo[2 * jj + 1]);
-                        mma_bf16_16816(acc[i][j2 + jj], a_lo[i], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                        for (int jj = 0; jj < 2; ++jj) {
+                            mma_bf16_16816(acc[1 + 2 * r + jj], a_hi[0], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                            mma_bf16_16816(acc[1 + 2 * r + jj], a_hi[0], b_lo[2 * jj], b_lo[2 * jj + 1]);
+                            mma_bf16_16816(acc[1 + 2 * r + jj], a_lo[0], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                        }
                     }
+                }
+            } else {
+                uint32_t a_hi[TM][4], a_lo[TM][4];
+#pragma unroll
+                for (int i = 0; i < TM; ++i) {
+                    // matrices: (channels +0, w +0), (channels +8, w +0), (channels +0, w +8), (channels +8, w +8)
+                    const int kr = k0 + (lane % 8) + 8 * (lane / 16);
+                    const int mc = wm * WM + i * 16 + 8 * ((lane / 8) % 2);
+                    const uint32_t off = (uint32_t)((kr * P + mc) * 2);
+                    ldmatrix_x4_trans(xs_hi + off, a_hi[i]);
+                    ldmatrix_x4_trans(xs_lo + off, a_lo[i]);
+                }
+#pragma unroll
+                for (int j2 = 0; j2 < TN; j2 += 2) {
+                    // two 8-channel column tiles per load: (tile 0, w +0), (tile 0, w +8), (tile 1, w +0), (tile 1, w +8)
+                    uint32_t b_hi[4], b_lo[4];
+                    const int kr = k0 + (lane % 8) + 8 * ((lane / 8) % 2);
+                    const int nc = (diag ? 0 : BM) + wn * WN + j2 * 8 + 8 * (lane / 16);
+                    const uint32_t off = (uint32_t)((kr * P + nc) * 2);
+                    ldmatrix_x4_trans(xs_hi + off, b_hi);
+                    ldmatrix_x4_trans(xs_lo + off, b_lo);
+#pragma unroll
+                    for (int i = 0; i < TM; ++i)
+#pragma unroll
+                        for (int jj = 0; jj < 2; ++jj) {
+                            mma_bf16_16816(acc[i * TN + j2 + jj], a_hi[i], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                            mma_bf16_16816(acc[i * TN + j2 + jj], a_hi[i], b_lo[2 * jj], b_lo[2 * jj + 1]);
+                            mma_bf16_16816(acc[i * TN + j2 + jj], a_lo[i], b_hi[2 * jj], b_hi[2 * jj + 1]);
+                        }
+                }
             }
         }
     }
@@ -321,19 +411,17 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
     if (sigma_bar) {
         float* out = sigma_bar + (size_t)uh * D * D;
 #pragma unroll
-        for (int i = 0; i < TM; ++i)
+        for (int t = 0; t < NT; ++t)
 #pragma unroll
-            for (int j = 0; j < TN; ++j)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int a = bi * BM + wm * WM + i * 16 + lane / 4 + 8 * (e / 2);
-                    const int c = bj * BM + wn * WN + j * 8 + 2 * (lane % 4) + (e % 2);
-                    if (a <= c) {
-                        const float v = acc[i][j][e] * inv_norm;
-                        out[(size_t)a * D + c] = v;
-                        out[(size_t)c * D + a] = v;
-                    }
+            for (int e = 0; e < 4; ++e) {
+                const int a = bi * BM + tiles.row0(t) + lane / 4 + 8 * (e / 2);
+                const int c = bj * BM + tiles.col0(t) + 2 * (lane % 4) + (e % 2);
+                if (a <= c) {
+                    const float v = acc[t][e] * inv_norm;
+                    out[(size_t)a * D + c] = v;
+                    out[(size_t)c * D + a] = v;
                 }
+            }
     }
     if constexpr (NB1 == 1) {
         if (img.image) {
@@ -354,14 +442,12 @@ stats_mma_kernel(const QT* __restrict__ q_win, const float* __restrict__ coef, i
                                                         ((((k % 64) / 8) ^ (r & 7)) << 4) + (k % 8) * 2);
             };
 #pragma unroll
-            for (int i = 0; i < TM; ++i)
-#pragma unroll
-                for (int j = 0; j < TN; ++j)
+            for (int t = 0; t < NT; ++t)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const int a = wm * WM + i * 16 + lane / 4 + 8 * (e / 2);
-                        const int c = wn * WN + j * 8 + 2 * (lane % 4) + (e % 2);
-                        const float v = acc[i][j][e] * inv_norm;
+                        const int a = tiles.row0(t) + lane / 4 + 8 * (e / 2);
+                        const int c = tiles.col0(t) + 2 * (lane % 4) + (e % 2);
+                        const float v = acc[t][e] * inv_norm;
                         if (a < c) {
                             // the two mirrored entries together carry (S_ca + S_ac) / (2 d), split into a bf16
                             // and the bf16 rounding of its remainder
@@ -421,6 +507,7 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
         1.0f / (float)(s.cov_norm == EA_COV_SAMPLE ? s.window - 1 : s.window);
     const unsigned heads = (unsigned)(s.n_units * s.n_q_heads);
     const StatsImage img = {static_cast<uint8_t*>(image), vec, s.n_kv_heads, 1.0f / sqrtf((float)d), 0.5f / (float)d};
+    int n_launches = 2;
     auto launch = [&](auto kern, int smem, unsigned blocks_y) {
         if (smem > 48 * 1024 &&
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
@@ -433,13 +520,18 @@ static ea_status launch_stats(const ea_ctx* ctx, const ea_shape& s, const QT* q_
     };
     bool ok;
     switch (d) {
-        case 64: ok = launch(stats_mma_kernel<64, QT>, StatsGeo<64>::SMEM, 1); break;
-        case 128: ok = launch(stats_mma_kernel<128, QT>, StatsGeo<128>::SMEM, 1); break;
-        case 256: ok = launch(stats_mma_kernel<256, QT>, StatsGeo<256>::SMEM, 3); break;
+        case 64: ok = launch(stats_mma_kernel<64, QT, false>, StatsGeo<64>::SMEM, 1); break;
+        case 128: ok = launch(stats_mma_kernel<128, QT, true>, StatsGeo<128>::SMEM, 1); break;
+        case 256:
+            // the two diagonal blocks (upper triangles), then the block above the diagonal
+            ok = launch(stats_mma_kernel<256, QT, true>, StatsGeo<256>::SMEM, 2) &&
+                 launch(stats_mma_kernel<256, QT, false>, StatsGeo<256>::SMEM, 1);
+            n_launches = 3;
+            break;
         default: return EA_ERR_UNSUPPORTED;
     }
     if (!ok) return EA_ERR_CUDA;
-    if (ctx) ea_count_launches(ctx, 2);
+    if (ctx) ea_count_launches(ctx, n_launches);
     return EA_CHECK_LAUNCH();
 }
 

@@ -506,7 +506,10 @@ ea_status ea_set_sm_budget(ea_ctx* ctx, int32_t n_sms);
  * not EA_GROUP_MEAN_LOGIT, workspace of ea_workspace_bytes(shape); otherwise
  * the statistics call behaves as without the flag (and then needs sigma_bar),
  * and ea_score with NULL statistics returns EA_ERR_INVALID_ARG.  Any later
- * statistics call of the context replaces the operand.
+ * statistics call of the context replaces the operand; a scoring call that is
+ * given statistics (ea_score with sigma_bar, ea_score_wo, ea_score_q8) builds
+ * its own operand in the same place, after which ea_score with NULL statistics
+ * is refused until the next statistics call.
  */
 ea_status ea_set_fused_stats(ea_ctx* ctx, int32_t on);
 

@@ -293,6 +293,7 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
     const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
     const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
     const ea_quad_form eq7 = ea_eq7_form(*shape, from_image ? nullptr : mu_bar, sigma_bar);
+    if (!from_image) ctx->image_ready = false;       // the images are rebuilt from the statistics given here
     if (ea_mma_path_supported(*shape) && shape->group_mode != EA_GROUP_MEAN_LOGIT) {
         // tensor-core log-scores with the log-sum-exp partials from their epilogue
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
@@ -365,6 +366,7 @@ ea_status ea_score_wo(ea_ctx* ctx, const ea_shape* shape, const void* k, const v
     if (n_weight_sets < 1 || shape->n_units % n_weight_sets != 0) return EA_ERR_INVALID_ARG;
     const ea_ws_plan plan = ea_plan_workspace(*shape);
     if (ctx->workspace_bytes < plan.total) return EA_ERR_WORKSPACE;
+    ctx->image_ready = false;                         // this call writes its own images into the workspace
     int prev = 0;
     EA_CUDA_TRY(cudaGetDevice(&prev));
     if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));

@@ -267,6 +267,7 @@ ea_status ea_score_q8(ea_ctx* ctx, const ea_shape* shape, const void* k_q8, cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     __nv_bfloat16* codes = static_cast<__nv_bfloat16*>(k_scratch);
     ea_quad_form eq7 = ea_eq7_form(*shape, mu_bar, sigma_bar);
+    ctx->image_ready = false;                         // this call writes its own (scaled) images into the workspace
     eq7.ch_scale = k_scale;
     bool lse_ready = false;
     if (ea_mma_q8_supported(*shape)) {

@@ -322,6 +322,12 @@ def test_fused_statistics_give_the_same_scores_bit_for_bit(ea, d, Hq, Hkv, n, ri
         sc2, lg2 = ea.ea_score(ctx, shape, k, v, None, None, cfg.eps, want_logits=True)
         ctx.sync_status()
         assert torch.equal(lg2, lg0) and torch.equal(sc2, sc0)
+    # a scoring call with explicit statistics rebuilds the images: the fused ones no longer stand
+    stats()
+    ea.ea_score(ctx, shape, k, v, mu, sig, cfg.eps)
+    with pytest.raises(ea.EAError) as e:
+        ea.ea_score(ctx, shape, k, v, None, None, cfg.eps)
+    assert e.value.status == 1
     # without a matching operand the call is refused
     other = ea.make_shape(U, Hq, Hkv, d, n - 1 if n > 129 else n + 1, W)
     big = ea.Context.for_shape(ea.make_shape(U, Hq, Hkv, d, n + 1, W))

@@ -250,10 +250,13 @@ class DecodeWorkload:
     by the previous step: synthetic rows of the same distribution)."""
 
     def __init__(self, cfg: inputs.EAConfig, device, ea, n_phases: int = 4, use_graph: bool = False,
-                 unordered: bool = False, fused: bool = False, fp8: bool = False):
+                 unordered: bool = False, fused: bool = False, fp8: bool = False, carry_norms: bool = False):
         import dataclasses
         self.cfg, self.device, self.ea = cfg, device, ea
         self.fp8 = fp8                      # the carried cache holds FP8 E4M3 codes with scales (the _q8 calls)
+        self.carry_norms = carry_norms      # ||v|| carried beside the cache: norms of the appended rows only per event
+        if fp8 and carry_norms:
+            raise SystemExit("--carry-norms is for the bf16 cache")
         if fp8 and fused:
             raise SystemExit("--fused-stats builds the image without key scales: not with --kv-dtype fp8")
         self.fused = fused                  # ea_set_fused_stats: no sigma_bar round trip, no image kernel
@@ -300,6 +303,12 @@ class DecodeWorkload:
             self.new_k.append(nk), self.new_v.append(nv), self.new_q.append(nq), self.new_vs.append(nvs)
         self.ring = torch.zeros((U, Hq, W, d), dtype=bf, device=device)
         self.pushed = torch.zeros((U,), dtype=torch.int64, device=device)
+        self.v_norm = None
+        if carry_norms:
+            self.v_norm = torch.empty((U, Hkv, self.cap), dtype=f32, device=device)
+            full = ea.make_shape(U, Hq, Hkv, d, self.cap, W, kv_capacity=self.cap)
+            ea.ea_value_norms(ea.Context.for_shape(full, device.index), full, self.v, 0, self.cap, self.v_norm)
+            torch.cuda.synchronize()
         self.pos = [torch.full((U,), pos, dtype=torch.int64, device=device) for pos, _, _ in self.events]
         self.mu = torch.empty((U, Hq, d), dtype=f32, device=device)
         self.sigma = torch.empty((U, Hq, d, d), dtype=f32, device=device)
@@ -332,16 +341,24 @@ class DecodeWorkload:
                                             unordered=self.unordered)
             return
         ea.ea_cache_append(ctx, self._shape(n - self.every), self.k, self.v, self.new_k[ph], self.new_v[ph])
+        if self.carry_norms:
+            ea.ea_value_norms(ctx, shape, self.v, n - self.every, self.every, self.v_norm)
         ea.ea_window_push(ctx, shape, self.ring, self.pushed, self.new_q[ph])
         if self.fused:
             ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu,
                                    want_sigma=False)
-            ea.ea_score(ctx, shape, self.k, self.v, None, None, cfg.eps, scores)
+            mu, sigma = None, None
         else:
             ea.ea_query_stats_ring(ctx, shape, self.ring, self.pushed, pos, cfg.n_future, cfg.rope_base, self.mu, self.sigma)
-            ea.ea_score(ctx, shape, self.k, self.v, self.mu, self.sigma, cfg.eps, scores)
+            mu, sigma = self.mu, self.sigma
+        if self.carry_norms:
+            ea.ea_score_vnorm(ctx, shape, self.k, self.v_norm, mu, sigma, cfg.eps, scores)
+        else:
+            ea.ea_score(ctx, shape, self.k, self.v, mu, sigma, cfg.eps, scores)
         compact = ea.ea_select_compact_inplace_unordered if self.unordered else ea.ea_select_compact_inplace
         compact(ctx, shape, scores, kept, self.k, self.v, idx)
+        if self.carry_norms:
+            ea.ea_carry_f32_inplace(ctx, shape, idx, kept, self.v_norm)
 
     def step(self, ctx, units_per_call):
         for e, (pos, n, kept) in enumerate(self.events):
@@ -498,7 +515,7 @@ def measure(args, cfg, ea, device, world, local, peaks, steps, warmup, keep_work
         torch.cuda.empty_cache()
     decode = cfg.cfg_id == 4
     wl = DecodeWorkload(cfg, device, ea, use_graph=args.graph, unordered=args.unordered, fused=args.fused_stats,
-                        fp8=args.kv_dtype == "fp8") if decode else Workload(cfg, device, ea, args.head_adaptive,
+                        fp8=args.kv_dtype == "fp8", carry_norms=args.carry_norms) if decode else Workload(cfg, device, ea, args.head_adaptive,
                                                                  args.hidden_stats, args.with_wo, args.kv_dtype == "fp8")
     upc = wl.n_units if decode else (args.units_per_call or wl.n_units)
     ctx = wl.make_ctx(upc)
@@ -621,6 +638,8 @@ def main():
                     help="prefill configs: cache held as FP8 E4M3 codes with scales (ea_score_q8, ea_select_compact_q8); "
                          "the device-resident line only, with the algorithmic bytes of that format")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--carry-norms", action="store_true",
+                    help="config 4: carry the value norms beside the cache (ea_value_norms / ea_score_vnorm / ea_carry_f32_inplace)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -678,6 +697,7 @@ def main():
         result["config"]["cache"] = "one carried buffer per sequence, compacted in place (%s), 512 pairs appended per event" % (
             "unordered: the tail's kept rows fill the evicted positions" if args.unordered else "temporal order kept")
         result["config"]["fused_statistics"] = bool(args.fused_stats)
+        result["config"]["carried_value_norms"] = bool(args.carry_norms)
 
     # end to end from host buffers through ea_compress_host (rank-local; max over ranks)
     if not args.skip_e2e:
@@ -697,12 +717,15 @@ def main():
                                  "kernel_frac": om["roofline"]["frac"], "kernel_ms": om["roofline"]["kernel_ms"],
                                  "kernel_mcycles": om["roofline"]["kernel_mcycles"], "sm_mhz": om["clocks"]["sm_mhz"],
                                  "gpu_launches": om["gpu_launches"]}
-        args.unordered = args.fused_stats = True
+        # the streaming shortcuts: only the appended tail's kept rows move, the statistics kernel writes the
+        # tensor-core operand itself, the value norms travel with the cache
+        args.unordered = args.fused_stats = args.carry_norms = True
         om = measure(args, inputs.CONFIGS[4], ea, device, world, local, peaks, max(5, args.steps // 2), 3, keep_workload=False)
-        args.unordered = args.fused_stats = False
-        others[inputs.CONFIGS[4].name]["unordered_compaction_fused_statistics"] = {
+        args.unordered = args.fused_stats = args.carry_norms = False
+        others[inputs.CONFIGS[4].name]["unordered_compaction_fused_statistics_carried_value_norms"] = {
             "ms_per_step": om["ms"], "value": om["slots"] / (om["ms"] * 1e-3) / 1e9,
-            "path_roofline_frac": om["path_roofline"]["frac"]}
+            "path_roofline_frac": om["path_roofline"]["frac"], "kernel_ms": om["roofline"]["kernel_ms"],
+            "sm_mhz": om["clocks"]["sm_mhz"], "gpu_launches": om["gpu_launches"]}
         # the headline shapes with the cache held as FP8 E4M3 codes (its own algorithmic bytes)
         args.kv_dtype = "fp8"
         om = measure(args, cfg, ea, device, world, local, peaks, max(5, args.steps // 2), 3, keep_workload=False)

@@ -398,6 +398,39 @@ ea_status ea_select_compact_inplace_unordered(ea_ctx* ctx, const ea_shape* shape
                                               int32_t* kept_idx, void* cuda_stream);
 
 /*
+ * Carried value norms (streaming decode, Sec. 4's set-up; the paper has no
+ * counterpart).  ||v_i|| of Eq. 9 does not change while pair i stays in the
+ * cache, so a cache that lives through consecutive compression events can
+ * carry the norms with it: v_norm fp32 [n_units, Hkv, capacity] (capacity =
+ * kv_capacity, or n_keys when that is 0), entry i of a head's range = ||v||
+ * of the head's row i.  Scoring then reads 4 bytes per cached pair in place
+ * of its value row.
+ *
+ * ea_value_norms: v_norm[u, g, i] = ||v[u, g, i, :]|| (fp32 accumulation) for
+ * first_row <= i < first_row + n_rows of every head; the rows need not lie
+ * below n_keys (first_row + n_rows <= capacity, else EA_ERR_INVALID_ARG).
+ * After ea_cache_append: first_row = the old n_keys, n_rows = n_new.
+ *
+ * ea_score_vnorm: ea_score with v_norm in place of v; every other argument,
+ * the fused form with NULL statistics included, as for ea_score.  The scores
+ * agree with ea_score's to fp32 rounding of the sum of squares.
+ *
+ * ea_carry_f32_inplace: values[u, g, j] <- values[u, g, kept_idx[u, g, j]] for
+ * j < n_kept, for a per-token fp32 array [n_units, Hkv, capacity] such as
+ * v_norm: what ea_select_compact_inplace or
+ * ea_select_compact_inplace_unordered did to the rows, given the kept_idx that
+ * call returned (both satisfy kept_idx[j] >= j, which the move relies on).
+ * Device pointers; asynchronous on cuda_stream.
+ */
+ea_status ea_value_norms(ea_ctx* ctx, const ea_shape* shape, const void* v, int32_t first_row,
+                         int32_t n_rows, float* v_norm, void* cuda_stream);
+ea_status ea_score_vnorm(ea_ctx* ctx, const ea_shape* shape, const void* k, const float* v_norm,
+                         const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
+                         float* logits_opt, void* cuda_stream);
+ea_status ea_carry_f32_inplace(ea_ctx* ctx, const ea_shape* shape, const int32_t* kept_idx,
+                               int32_t n_kept, float* values, void* cuda_stream);
+
+/*
  * Streaming decode: one cache buffer and one window buffer carried through
  * consecutive compression events (the decoding set-up of the "Implementation
  * details" paragraph: a buffer of the most recent 128 states, compression

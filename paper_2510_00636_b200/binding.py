@@ -25,7 +25,7 @@ EXPORTS = (
     "ea_query_stats", "ea_score", "ea_select_compact", "ea_sync_status", "ea_profile_begin",
     "ea_profile_end", "ea_host_workspace_bytes", "ea_compress_host", "ea_query_stats_static",
     "ea_select_compact_adaptive", "ea_n_floor", "ea_query_stats_hidden", "ea_wo_gram", "ea_score_wo",
-    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_cache_append_q8", "ea_select_compact_inplace_q8", "ea_select_compact_adaptive_q8", "ea_select_compact_inplace_unordered",
+    "ea_select_compact_inplace", "ea_selftest_wait_timeout", "ea_last_cuda_error", "ea_set_sm_budget", "ea_set_side_sms", "ea_set_fused_stats", "ea_cache_append", "ea_window_push", "ea_query_stats_ring", "ea_score_q8", "ea_score_q8_scratch_bytes", "ea_select_compact_q8", "ea_cache_append_q8", "ea_select_compact_inplace_q8", "ea_select_compact_adaptive_q8", "ea_value_norms", "ea_score_vnorm", "ea_carry_f32_inplace", "ea_select_compact_inplace_unordered",
 )
 STATIC_MAX_ROPE_PAIRS = 16384
 
@@ -101,6 +101,10 @@ def lib() -> ctypes.CDLL:
         L.ea_cache_append_q8.restype = L.ea_select_compact_inplace_q8.restype = ctypes.c_int
         L.ea_select_compact_adaptive_q8.argtypes = [vp, sp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.ea_select_compact_adaptive_q8.restype = ctypes.c_int
+        L.ea_value_norms.argtypes = [vp, sp, vp, i32, i32, vp, vp]
+        L.ea_score_vnorm.argtypes = [vp, sp, vp, vp, vp, vp, f32, vp, vp, vp]
+        L.ea_carry_f32_inplace.argtypes = [vp, sp, vp, i32, vp, vp]
+        L.ea_value_norms.restype = L.ea_score_vnorm.restype = L.ea_carry_f32_inplace.restype = ctypes.c_int
         L.ea_score_q8_scratch_bytes.restype = ctypes.c_int
         L.ea_set_fused_stats.argtypes = [vp, i32]
         L.ea_set_fused_stats.restype = ctypes.c_int
@@ -344,6 +348,39 @@ def ea_score(ctx: Context, shape: Shape, k, v, mu_bar, sigma_bar, epsilon: float
     _check(lib().ea_score(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(mu_bar), _ptr(sigma_bar),
                           float(epsilon), _ptr(scores), _ptr(logits), _stream(ctx.device)), "ea_score")
     return (scores, logits) if (want_logits or logits is not None) else scores
+
+
+def ea_value_norms(ctx: Context, shape: Shape, v, first_row: int, n_rows: int, v_norm):
+    """``v_norm[u,g,i] = ||v[u,g,i]||`` for ``first_row <= i < first_row + n_rows``; v bf16 [U,Hkv,cap,d], v_norm fp32
+    [U,Hkv,cap] (written in place)."""
+    _dev_tensor(v, torch.bfloat16, "v")
+    _dev_tensor(v_norm, torch.float32, "v_norm")
+    _check(lib().ea_value_norms(ctx._h, ctypes.byref(shape), _ptr(v), int(first_row), int(n_rows), _ptr(v_norm),
+                                _stream(ctx.device)), "ea_value_norms")
+
+
+def ea_score_vnorm(ctx: Context, shape: Shape, k, v_norm, mu_bar, sigma_bar, epsilon: float, scores=None, logits=None,
+                   want_logits: bool = False):
+    """``ea_score`` with the carried value norms ``v_norm`` fp32 [U,Hkv,cap] in place of the value rows."""
+    _dev_tensor(k, torch.bfloat16, "k")
+    _dev_tensor(v_norm, torch.float32, "v_norm")
+    U, Hq, Hkv, n = shape.n_units, shape.n_q_heads, shape.n_kv_heads, shape.n_keys
+    if scores is None:
+        scores = torch.empty((U, Hkv, n), dtype=torch.float32, device=k.device)
+    if logits is None and want_logits:
+        logits = torch.empty((U, Hq, n), dtype=torch.float32, device=k.device)
+    _check(lib().ea_score_vnorm(ctx._h, ctypes.byref(shape), _ptr(k), _ptr(v_norm), _ptr(mu_bar), _ptr(sigma_bar),
+                                float(epsilon), _ptr(scores), _ptr(logits), _stream(ctx.device)), "ea_score_vnorm")
+    return (scores, logits) if (want_logits or logits is not None) else scores
+
+
+def ea_carry_f32_inplace(ctx: Context, shape: Shape, kept_idx, n_kept: int, values):
+    """``values[u,g,j] <- values[u,g,kept_idx[u,g,j]]`` for ``j < n_kept`` (in place), with the ``kept_idx`` an in-place
+    compaction returned."""
+    _dev_tensor(kept_idx, torch.int32, "kept_idx")
+    _dev_tensor(values, torch.float32, "values")
+    _check(lib().ea_carry_f32_inplace(ctx._h, ctypes.byref(shape), _ptr(kept_idx), int(n_kept), _ptr(values),
+                                      _stream(ctx.device)), "ea_carry_f32_inplace")
 
 
 def score_q8_scratch_bytes(shape: Shape) -> int:

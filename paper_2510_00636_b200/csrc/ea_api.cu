@@ -259,14 +259,16 @@ ea_status ea_query_stats_hidden(ea_ctx* ctx, const ea_shape* shape, const void* 
     return st;
 }
 
-ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
-                   const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
-                   float* logits_opt, void* cuda_stream) {
+// ea_score and ea_score_vnorm: exactly one of v (the value rows) and v_norm (their norms, carried with the
+// cache, [units, Hkv, capacity]) is given.
+static ea_status score_impl(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v, const float* v_norm,
+                            const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
+                            float* logits_opt, void* cuda_stream) {
     if (!ctx) return EA_ERR_INVALID_ARG;
     ea_status st = check_shape(shape);
     if (st != EA_OK) return st;
     if (shape->n_units == 0 || shape->n_keys == 0) return EA_OK;
-    if (!k || !v || !scores) return EA_ERR_INVALID_ARG;
+    if (!k || (!v && !v_norm) || !scores) return EA_ERR_INVALID_ARG;
     // sigma_bar == NULL: the images the last statistics call of this context wrote for this very shape
     // (ea_set_fused_stats) stand in for mu_bar and sigma_bar
     const bool from_image = sigma_bar == nullptr;
@@ -299,7 +301,7 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
         float* lse_part = reinterpret_cast<float*>(ws + plan.lse_part);
         float* vnorm = reinterpret_cast<float*>(ws + plan.vnorm);
         int n_chunks = 0;
-        const bool side = ctx->side_sms > 0 && ea_kv_cap(*shape) == shape->n_keys;   // the side pass streams a dense V
+        const bool side = v && ctx->side_sms > 0 && ea_kv_cap(*shape) == shape->n_keys;   // the side pass streams a dense V
         if (side) {
             // the value norms do not depend on the log-scores: their pass over V goes to a few SMs of its
             // own, on a second stream, and is launched first so that it is resident when the log-score
@@ -316,7 +318,9 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
         if (side) {
             // always rejoin, whatever happened in between: the caller's stream must not run ahead of the side pass
             EA_CUDA_TRY(cudaStreamWaitEvent(stream, ctx->ev_join, 0));
-            if (st == EA_OK) st = ea_launch_weight(ctx, *shape, logits, lse, vnorm, epsilon, scores, stream);
+            if (st == EA_OK) st = ea_launch_weight(ctx, *shape, logits, lse, vnorm, shape->n_keys, epsilon, scores, stream);
+        } else if (st == EA_OK && v_norm) {
+            st = ea_launch_weight(ctx, *shape, logits, lse, v_norm, ea_kv_cap(*shape), epsilon, scores, stream);
         } else if (st == EA_OK) {
             st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, true, scores, stream);
         }
@@ -329,8 +333,63 @@ ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void
         } else {
             st = ea_launch_logits_simt(ctx, *shape, kb, eq7, logits, stream);
         }
-        if (st == EA_OK) st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, false, scores, stream);
+        if (st == EA_OK && v_norm) {
+            // one softmax row per query head, or per KV head for the mean of the log-scores
+            st = shape->group_mode == EA_GROUP_MEAN_LOGIT ? ea_launch_lse_grouped(ctx, *shape, logits, lse, stream)
+                                                          : ea_launch_lse(ctx, *shape, logits, lse, stream);
+            if (st == EA_OK)
+                st = ea_launch_weight(ctx, *shape, logits, lse, v_norm, ea_kv_cap(*shape), epsilon, scores, stream);
+        } else if (st == EA_OK) {
+            st = ea_launch_finalize(ctx, *shape, logits, vb, epsilon, lse, false, scores, stream);
+        }
     }
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
+                   const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
+                   float* logits_opt, void* cuda_stream) {
+    if (!v) return EA_ERR_INVALID_ARG;
+    return score_impl(ctx, shape, k, v, nullptr, mu_bar, sigma_bar, epsilon, scores, logits_opt, cuda_stream);
+}
+
+ea_status ea_score_vnorm(ea_ctx* ctx, const ea_shape* shape, const void* k, const float* v_norm,
+                         const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
+                         float* logits_opt, void* cuda_stream) {
+    if (!v_norm) return EA_ERR_INVALID_ARG;
+    return score_impl(ctx, shape, k, nullptr, v_norm, mu_bar, sigma_bar, epsilon, scores, logits_opt, cuda_stream);
+}
+
+ea_status ea_value_norms(ea_ctx* ctx, const ea_shape* shape, const void* v, int32_t first_row, int32_t n_rows,
+                         float* v_norm, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (first_row < 0 || n_rows < 0 || (long long)first_row + n_rows > ea_kv_cap(*shape)) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0 || n_rows == 0) return EA_OK;
+    if (!v || !v_norm || !aligned16(v)) return EA_ERR_INVALID_ARG;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    st = ea_launch_vnorm_rows(ctx, *shape, static_cast<const __nv_bfloat16*>(v), first_row, n_rows, v_norm,
+                              static_cast<cudaStream_t>(cuda_stream));
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return st;
+}
+
+ea_status ea_carry_f32_inplace(ea_ctx* ctx, const ea_shape* shape, const int32_t* kept_idx, int32_t n_kept,
+                               float* values, void* cuda_stream) {
+    if (!ctx) return EA_ERR_INVALID_ARG;
+    ea_status st = check_shape(shape);
+    if (st != EA_OK) return st;
+    if (n_kept < 0 || n_kept > shape->n_keys) return EA_ERR_INVALID_ARG;
+    if (shape->n_units == 0 || n_kept == 0) return EA_OK;
+    if (!kept_idx || !values) return EA_ERR_INVALID_ARG;
+    int prev = 0;
+    EA_CUDA_TRY(cudaGetDevice(&prev));
+    if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
+    st = ea_launch_carry_f32(ctx, *shape, n_kept, kept_idx, values, static_cast<cudaStream_t>(cuda_stream));
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;
 }

@@ -162,8 +162,15 @@ ea_status ea_launch_lse_combine(const ea_ctx* ctx, const ea_shape& s, const floa
 // ||v|| of every value row on n_ctas SMs (bulk-copy-fed stream), and the weighting that uses them.
 ea_status ea_launch_vnorm(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* v, int n_ctas, float* vnorm,
                           cudaStream_t st);
+// (vn_stride: floats between the norms of consecutive heads)
 ea_status ea_launch_weight(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
-                           const float* vnorm, float epsilon, float* scores, cudaStream_t st);
+                           const float* vnorm, int vn_stride, float epsilon, float* scores, cudaStream_t st);
+// ||v|| of rows first_row .. first_row + n_rows - 1 of every head, into v_norm [units, Hkv, capacity]
+ea_status ea_launch_vnorm_rows(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* v, int first_row,
+                               int n_rows, float* v_norm, cudaStream_t st);
+// values[head][j] <- values[head][idx[head][j]] for j < n_kept (idx[j] >= j), values [units, Hkv, capacity]
+ea_status ea_launch_carry_f32(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* idx, float* values,
+                              cudaStream_t st);
 
 ea_status ea_launch_finalize(const ea_ctx* ctx, const ea_shape& s, const float* logits,
                              const __nv_bfloat16* v, float epsilon, float* lse, bool lse_ready, float* scores,

@@ -242,7 +242,7 @@ vnorm_stream_kernel(const __nv_bfloat16* __restrict__ v, long long n_rows, float
 // score = (group reduction of the attention + eps) * ||v|| with the norms already computed; one thread per key.
 __global__ void __launch_bounds__(256)
 weight_kernel(const float* __restrict__ logits, const float* __restrict__ lse, const float* __restrict__ vnorm,
-              int Hq, int Hkv, int n, int group_mode, float epsilon, float* __restrict__ scores) {
+              int vn_stride, int Hq, int Hkv, int n, int group_mode, float epsilon, float* __restrict__ scores) {
     const int G = Hq / Hkv;
     const int ug = blockIdx.y;
     const int u = ug / Hkv, g = ug % Hkv;
@@ -261,7 +261,38 @@ weight_kernel(const float* __restrict__ logits, const float* __restrict__ lse, c
         }
         if (group_mode == EA_GROUP_MEAN_PROB) a *= 1.0f / (float)G;
     }
-    scores[(size_t)ug * n + key] = (a + epsilon) * vnorm[(size_t)ug * n + key];
+    scores[(size_t)ug * n + key] = (a + epsilon) * vnorm[(size_t)ug * vn_stride + key];
+}
+
+// ||v|| of a range of rows of every head: lane groups of D / 8 lanes read one row each (128-bit loads), the
+// partial sums of squares meet by shuffles, the group's first lane stores the norm.
+template <int D>
+__global__ void __launch_bounds__(256)
+vnorm_rows_kernel(const __nv_bfloat16* __restrict__ v, int cap, int first_row, int n_rows, long long total_rows,
+                  float* __restrict__ v_norm) {
+    constexpr int LPR = D / 8;                     // lanes per row
+    const long long stride = (long long)gridDim.x * blockDim.x / LPR;
+    const int lane = threadIdx.x % 32, piece = lane % LPR;
+    // the loop bound is the warp's, so that every lane takes part in the shuffles
+    for (long long r0 = ((long long)blockIdx.x * blockDim.x + (threadIdx.x - lane)) / LPR; r0 < total_rows; r0 += stride) {
+        const long long r = r0 + lane / LPR;
+        const bool valid = r < total_rows;
+        const long long row = valid ? (r / n_rows) * cap + first_row + r % n_rows : 0;
+        float ss = 0.f;
+        if (valid) {
+            const uint4 x = __ldg(reinterpret_cast<const uint4*>(v + row * D) + piece);
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float a = __uint_as_float(w[q] << 16), b = __uint_as_float(w[q] & 0xffff0000u);
+                ss = fmaf(a, a, ss);
+                ss = fmaf(b, b, ss);
+            }
+        }
+#pragma unroll
+        for (int off = LPR / 2; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        if (valid && piece == 0) v_norm[row] = sqrtf(ss);
+    }
 }
 
 // score = group reduction of (a_hat_h + eps) * sqrt(wo_norm2_h) over the query heads of the KV head
@@ -403,10 +434,28 @@ ea_status ea_launch_vnorm(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloa
 }
 
 ea_status ea_launch_weight(const ea_ctx* ctx, const ea_shape& s, const float* logits, const float* lse,
-                           const float* vnorm, float epsilon, float* scores, cudaStream_t st) {
+                           const float* vnorm, int vn_stride, float epsilon, float* scores, cudaStream_t st) {
     dim3 grid((unsigned)((s.n_keys + 255) / 256), (unsigned)(s.n_units * s.n_kv_heads));
-    weight_kernel<<<grid, 256, 0, st>>>(logits, lse, vnorm, s.n_q_heads, s.n_kv_heads, s.n_keys, s.group_mode,
-                                        epsilon, scores);
+    weight_kernel<<<grid, 256, 0, st>>>(logits, lse, vnorm, vn_stride, s.n_q_heads, s.n_kv_heads, s.n_keys,
+                                        s.group_mode, epsilon, scores);
+    ea_count_launches(ctx, 1);
+    return EA_CHECK_LAUNCH();
+}
+
+ea_status ea_launch_vnorm_rows(const ea_ctx* ctx, const ea_shape& s, const __nv_bfloat16* v, int first_row,
+                               int n_rows, float* v_norm, cudaStream_t st) {
+    const long long total = (long long)s.n_units * s.n_kv_heads * n_rows;
+    if (total <= 0) return EA_OK;
+    const int lpr = s.head_dim / 8;
+    const long long want = (total * lpr + 255) / 256, lim = (long long)ctx->sm_count * 16;
+    const unsigned grid = (unsigned)(want < lim ? want : lim);
+    const int cap = ea_kv_cap(s);
+    switch (s.head_dim) {
+        case 64: vnorm_rows_kernel<64><<<grid, 256, 0, st>>>(v, cap, first_row, n_rows, total, v_norm); break;
+        case 128: vnorm_rows_kernel<128><<<grid, 256, 0, st>>>(v, cap, first_row, n_rows, total, v_norm); break;
+        case 256: vnorm_rows_kernel<256><<<grid, 256, 0, st>>>(v, cap, first_row, n_rows, total, v_norm); break;
+        default: return EA_ERR_UNSUPPORTED;
+    }
     ea_count_launches(ctx, 1);
     return EA_CHECK_LAUNCH();
 }

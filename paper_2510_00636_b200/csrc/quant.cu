@@ -145,35 +145,6 @@ __global__ void gather_adaptive_q8_kernel(const int32_t* __restrict__ kept_idx, 
     }
 }
 
-// The value scales of a head follow their rows through an in-place compaction.  Ordered form: position j
-// receives the scale of row idx[j] >= j; one CTA per head walks the kept rows in chunks, a chunk's sources
-// in registers before its destinations are written; a later chunk reads at or behind its own first
-// destination, which earlier chunks never write.
-constexpr int kScaleThreads = 256;
-__global__ void __launch_bounds__(kScaleThreads)
-scale_inplace_kernel(const int32_t* __restrict__ kept_idx, int cap, int n_kept, float* v_scale) {
-    const long long head = blockIdx.x;
-    float* vs = v_scale + head * (long long)cap;
-    const int32_t* idx = kept_idx + head * (long long)n_kept;
-    for (int j0 = 0; j0 < n_kept; j0 += kScaleThreads) {
-        const int j = j0 + threadIdx.x;
-        const int src = j < n_kept ? idx[j] : -1;
-        const float x = src >= 0 ? vs[src] : 0.f;
-        __syncthreads();
-        if (src >= 0) vs[j] = x;
-    }
-}
-// Unordered form: where[p] is the original row now at p; the movers come from at or beyond n_kept and
-// land below it, so no move can disturb another.
-__global__ void scale_fill_kernel(const int32_t* __restrict__ where, long long total, int cap, int n_kept, float* v_scale) {
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
-        const long long head = t / n_kept;
-        const int p = (int)(t % n_kept), w = where[t];
-        if (w != p) v_scale[head * cap + p] = v_scale[head * cap + w];
-    }
-}
-
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -415,28 +386,18 @@ ea_status ea_select_compact_inplace_q8(ea_ctx* ctx, const ea_shape* shape, const
     EA_CUDA_TRY(cudaGetDevice(&prev));
     if (prev != ctx->device) EA_CUDA_TRY(cudaSetDevice(ctx->device));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const int cap = ea_kv_cap(*shape);
-    const long long heads = (long long)shape->n_units * shape->n_kv_heads;
     if (unordered) {
         // the ascending selection goes to the workspace (the log-score region: nothing of a compaction reads it)
         const ea_ws_plan plan = ea_plan_workspace(*shape);
         int32_t* sel = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + plan.logits);
         st = ea_launch_select(ctx, *shape, scores, n_kept, sel, stream);
         if (st == EA_OK) st = ea_launch_compact_fill(ctx, *shape, n_kept, sel, kept_idx, k_q8, v_q8, stream, true);
-        if (st == EA_OK) {
-            const long long total = heads * n_kept, want = (total + 255) / 256, lim = (long long)ctx->sm_count * 16;
-            scale_fill_kernel<<<(unsigned)(want < lim ? want : lim), 256, 0, stream>>>(kept_idx, total, cap, n_kept, v_scale);
-            ea_count_launches(ctx, 1);
-            st = EA_CHECK_LAUNCH();
-        }
+        // the value scales follow their rows (kept_idx now names the original row at each position)
+        if (st == EA_OK) st = ea_launch_carry_f32(ctx, *shape, n_kept, kept_idx, v_scale, stream);
     } else {
         st = ea_launch_select(ctx, *shape, scores, n_kept, kept_idx, stream);
         if (st == EA_OK) st = ea_launch_compact_inplace(ctx, *shape, n_kept, kept_idx, k_q8, v_q8, stream, true);
-        if (st == EA_OK) {
-            scale_inplace_kernel<<<(unsigned)heads, kScaleThreads, 0, stream>>>(kept_idx, cap, n_kept, v_scale);
-            ea_count_launches(ctx, 1);
-            st = EA_CHECK_LAUNCH();
-        }
+        if (st == EA_OK) st = ea_launch_carry_f32(ctx, *shape, n_kept, kept_idx, v_scale, stream);
     }
     if (prev != ctx->device) cudaSetDevice(prev);
     return st;

@@ -599,7 +599,35 @@ compact_fill_kernel(const int32_t* __restrict__ sel, int cap, int n_kept, int32_
     }
 }
 
+// A per-token fp32 array of a head follows its rows through an in-place compaction: position j receives the
+// value of row idx[j] >= j (ascending kept positions, or the original row now at j after the unordered form,
+// where movers come from beyond n_kept).  One CTA per head walks the positions in chunks, a chunk's sources
+// in registers before its destinations are written; a later chunk reads at or behind its own first
+// destination, which earlier chunks never write.
+constexpr int kCarryThreads = 256;
+__global__ void __launch_bounds__(kCarryThreads)
+carry_f32_kernel(const int32_t* __restrict__ idx_all, int cap, int n_kept, float* values) {
+    const long long head = blockIdx.x;
+    float* vs = values + head * (long long)cap;
+    const int32_t* idx = idx_all + head * (long long)n_kept;
+    for (int j0 = 0; j0 < n_kept; j0 += kCarryThreads) {
+        const int j = j0 + threadIdx.x;
+        const int src = j < n_kept ? idx[j] : -1;
+        const float x = src >= 0 ? vs[src] : 0.f;
+        __syncthreads();
+        if (src >= 0) vs[j] = x;
+    }
+}
+
 }  // namespace
+
+ea_status ea_launch_carry_f32(const ea_ctx* ctx, const ea_shape& s, int n_kept, const int32_t* idx, float* values,
+                              cudaStream_t st) {
+    if (n_kept <= 0) return EA_OK;
+    carry_f32_kernel<<<(unsigned)(s.n_units * s.n_kv_heads), kCarryThreads, 0, st>>>(idx, ea_kv_cap(s), n_kept, values);
+    ea_count_launches(ctx, 1);
+    return EA_CHECK_LAUNCH();
+}
 
 static ea_status launch_select(const ea_ctx* ctx, const ea_shape& s, const float* scores, int n_kept,
                                const HeadPlan& plan, int32_t* kept_idx, cudaStream_t st) {

@@ -375,3 +375,75 @@ def test_streaming_calls_validate_their_arguments(ea):
     ea.ea_window_push(ctx, shape, ring, pushed, ring[:, :, :0].contiguous())
     ctx.sync_status()
     assert int(pushed[0]) == 0
+
+
+@pytest.mark.parametrize("unordered", [False, True])
+def test_value_norms_carried_with_the_cache(ea, oracle, unordered):
+    """Streaming decode with the value norms carried beside the cache: norms of the appended rows only
+    (ea_value_norms), scores from the norms (ea_score_vnorm), the norms moved like the rows
+    (ea_carry_f32_inplace).  Every event: scores within the tolerance protocol of the oracle's streaming driver
+    (and to relative 1e-2 directly), equal to ea_score's on the same cache up to the rounding of the sum of
+    squares, the kept set exact on the GPU's own scores, and afterwards every carried norm equal to the norm of
+    the row it sits beside."""
+    import dataclasses
+    import parity
+    from oracle.ea_stream import StreamOracle, fill_holes
+    base = inputs.CONFIGS[4].tempered(2.0)
+    budget, every, n0 = 1024, 384, 640
+    cap = budget + every
+    cfg = dataclasses.replace(base, n_layers=1, batch=2, n_keys=n0, n_kept=budget)
+    U, Hq, Hkv, d, W = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window
+    dev = torch.device("cuda")
+    _, k0, v0, _ = inputs.generate_layer(cfg, layer=7, device=dev, n_keys=n0, draw=1)
+    k = torch.zeros((U, Hkv, cap, d), dtype=torch.bfloat16, device=dev)
+    v = torch.zeros_like(k)
+    k[:, :, :n0], v[:, :, :n0] = k0, v0
+    v_norm = torch.full((U, Hkv, cap), float("nan"), device=dev)          # nothing may read a norm never written
+    ring = torch.zeros((U, Hq, W, d), dtype=torch.bfloat16, device=dev)
+    pushed = torch.zeros((U,), dtype=torch.int64, device=dev)
+    st = StreamOracle(inputs.bits(k0), inputs.bits(v0), window=W, budget=budget)
+    ctx = ea.Context.for_shape(ea.make_shape(U, Hq, Hkv, d, cap, W, kv_capacity=cap))
+    ea.ea_value_norms(ctx, ea.make_shape(U, Hq, Hkv, d, n0, W, kv_capacity=cap), v, 0, n0, v_norm)
+    n_cur, position = n0, n0
+    for e, m in enumerate((100, 200, 384, 384)):
+        n = n_cur + every
+        n_kept = min(n, budget)
+        position += every
+        _, kn, vn, _ = inputs.generate_layer(cfg, layer=7, device=dev, n_keys=every, draw=2 + e,
+                                             key_positions=torch.arange(position - every, position))
+        qn, _, _, _ = inputs.generate_layer(dataclasses.replace(cfg, window=m), layer=7, device=dev, n_keys=1,
+                                            draw=100 + e, q_phase=0.1 * e)
+        pos = torch.full((U,), position, dtype=torch.int64, device=dev)
+        shape_old = ea.make_shape(U, Hq, Hkv, d, n_cur, W, kv_capacity=cap)
+        shape = ea.make_shape(U, Hq, Hkv, d, n, W, kv_capacity=cap)
+        ea.ea_cache_append(ctx, shape_old, k, v, kn, vn)
+        ea.ea_value_norms(ctx, shape, v, n_cur, every, v_norm)
+        ea.ea_window_push(ctx, shape, ring, pushed, qn)
+        mu, sigma = ea.ea_query_stats_ring(ctx, shape, ring, pushed, pos, cfg.n_future, cfg.rope_base)
+        sc_t, lg_t = ea.ea_score_vnorm(ctx, shape, k, v_norm, mu, sigma, cfg.eps, want_logits=True)
+        sc_v = ea.ea_score(ctx, shape, k, v, mu, sigma, cfg.eps)
+        torch.testing.assert_close(sc_t, sc_v, rtol=1e-5, atol=0.0)
+        compact = ea.ea_select_compact_inplace_unordered if unordered else ea.ea_select_compact_inplace
+        idx = compact(ctx, shape, sc_t, n_kept, k, v)
+        ea.ea_carry_f32_inplace(ctx, shape, idx, n_kept, v_norm)
+        ctx.sync_status()
+
+        st.append(inputs.bits(kn), inputs.bits(vn))
+        st.push_queries(inputs.bits(qn))
+        ref = st.compress(np.full((U,), position), cfg.n_future, cfg.rope_base, cfg.eps)
+        delta = parity.logit_error_bound(st.k, ref["mu_bar"], ref["sigma_bar"], 16)
+        bad, _ = parity.check_logits(lg_t.cpu().numpy(), ref["logits"], delta)
+        assert bad == 0, f"event {e}"
+        lo, hi = parity.score_range(ref["logits"], delta, st.v, cfg.eps, 0)
+        sc = sc_t.cpu().numpy()
+        bad, unstable = parity.check_scores(sc, lo, hi)
+        assert bad == 0 and unstable == 0, f"event {e}"
+        np.testing.assert_allclose(sc, ref["scores"], rtol=1e-2, atol=0.0)
+        got = idx.cpu().numpy()
+        sel = oracle.select(sc.astype(np.float64), n_kept)
+        assert np.array_equal(got, fill_holes(sel, n_kept) if unordered else sel), f"event {e}"
+        st.keep(got)
+        assert np.array_equal(inputs.bits(v[:, :, :n_kept]), st.v), f"event {e}: value cache differs"
+        want_norm = v[:, :, :n_kept].float().square().sum(-1).sqrt()
+        torch.testing.assert_close(v_norm[:, :, :n_kept], want_norm, rtol=2e-6, atol=0.0)
+        n_cur = n_kept

@@ -350,14 +350,12 @@ static ea_status score_impl(ea_ctx* ctx, const ea_shape* shape, const void* k, c
 ea_status ea_score(ea_ctx* ctx, const ea_shape* shape, const void* k, const void* v,
                    const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
                    float* logits_opt, void* cuda_stream) {
-    if (!v) return EA_ERR_INVALID_ARG;
     return score_impl(ctx, shape, k, v, nullptr, mu_bar, sigma_bar, epsilon, scores, logits_opt, cuda_stream);
 }
 
 ea_status ea_score_vnorm(ea_ctx* ctx, const ea_shape* shape, const void* k, const float* v_norm,
                          const float* mu_bar, const float* sigma_bar, float epsilon, float* scores,
                          float* logits_opt, void* cuda_stream) {
-    if (!v_norm) return EA_ERR_INVALID_ARG;
     return score_impl(ctx, shape, k, nullptr, v_norm, mu_bar, sigma_bar, epsilon, scores, logits_opt, cuda_stream);
 }
 
